@@ -1,0 +1,123 @@
+"""Pins for the k-bit linear quantiser (Eq. 9), bit-planes and the bit-plane product (Eq. 8)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1609_07061_b200 import workloads
+
+
+def _read(golden_dir, name):
+    with open(os.path.join(golden_dir, name)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def test_linear_quant_golden(golden_dir):
+    rows = _read(golden_dir, "linear_quant_2bit.txt")
+    x = np.array([float(r[0]) for r in rows], np.float32)
+    want = np.array([int(r[1]) for r in rows], np.int32)
+    np.testing.assert_array_equal(oracle.linear_quant_codes(x, 2, 0.0, 1.0), want)
+
+
+@pytest.mark.parametrize("bits", [1, 2, 4, 8])
+@pytest.mark.parametrize("lo,hi", [(0.0, 1.0), (-1.0, 1.0), (-3.0, 5.0)])
+def test_level_centres_are_fixed_points(bits, lo, hi):
+    L = (1 << bits) - 1
+    q = np.arange(L + 1)
+    centres = (lo + q.astype(np.float64) * (hi - lo) / L).astype(np.float32)
+    np.testing.assert_array_equal(oracle.linear_quant_codes(centres, bits, lo, hi), q)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_monotone_clipped_and_bounded(bits):
+    x = np.linspace(-2.0, 2.0, 20001).astype(np.float32)
+    q = oracle.linear_quant_codes(x, bits, -1.0, 1.0)
+    assert np.all(np.diff(q) >= 0)
+    assert q.min() == 0 and q.max() == (1 << bits) - 1
+    assert np.all(q[x <= -1.0] == 0) and np.all(q[x >= 1.0] == (1 << bits) - 1)
+    assert len(np.unique(q)) == 1 << bits
+
+
+def test_ties_go_to_even():
+    # lo=0, hi=15 with 4 bits makes the step exactly 1, so j+0.5 is an exact tie
+    x = np.arange(0, 15, dtype=np.float32) + 0.5
+    q = oracle.linear_quant_codes(x, 4, 0.0, 15.0)
+    want = np.array([0, 2, 2, 4, 4, 6, 6, 8, 8, 10, 10, 12, 12, 14, 14], np.int32)
+    np.testing.assert_array_equal(q, want)
+
+
+@pytest.mark.parametrize("bits,lo,hi", [(2, 0.0, 1.0), (4, -1.0, 1.0), (8, 0.0, 1.0)])
+def test_against_torch_round_on_same_quotient(bits, lo, hi):
+    """torch.round is also round-half-to-even: an independent library witness on the same fp32 steps."""
+    g = torch.Generator().manual_seed(11)
+    x = (torch.randn(50000, generator=g) * 0.8).to(torch.float32)
+    inv = torch.tensor(float(oracle.inv_step(bits, lo, hi)), dtype=torch.float32)
+    t = torch.clamp(x, lo, hi)
+    u = (t - torch.tensor(lo, dtype=torch.float32)) * inv
+    want = torch.round(u).to(torch.int32).clamp(0, (1 << bits) - 1).numpy()
+    np.testing.assert_array_equal(oracle.linear_quant_codes(x.numpy(), bits, lo, hi), want)
+
+
+def test_nan_and_infinities():
+    x = np.array([np.nan, np.inf, -np.inf], np.float32)
+    np.testing.assert_array_equal(oracle.linear_quant_codes(x, 4, -1.0, 1.0), [0, 15, 0])
+
+
+@pytest.mark.parametrize("bits", [1, 2, 4, 8])
+def test_bit_plane_reconstruction(bits):
+    q = np.arange(1 << bits, dtype=np.int32)
+    rec = sum((1 << i) * oracle.bit_plane(q, i).astype(np.int64) for i in range(bits))
+    np.testing.assert_array_equal(rec, q)
+    # symmetric reading: 2q - (2^k - 1) = sum_i 2^i s_i, s_i = +-1 from bit i
+    sym = sum((1 << i) * (2 * oracle.bit_plane(q, i).astype(np.int64) - 1) for i in range(bits))
+    np.testing.assert_array_equal(oracle.codes_to_symmetric(q, bits), sym)
+
+
+def test_eq8_golden(golden_dir):
+    rows = _read(golden_dir, "eq8_bitplanes.txt")
+    x = np.array([[int(v) for v in r[1:]] for r in rows if r[0] == "x"], np.int32)
+    w = np.array([[int(v) for v in r[1:]] for r in rows if r[0] == "w"], np.int32).T
+    s = int([r for r in rows if r[0] == "s"][0][1])
+    for r in rows:
+        if r[0] == "plane":
+            n = int(r[1])
+            np.testing.assert_array_equal(oracle.bit_plane(x[0], n - 1), [int(v) for v in r[2:5]])
+            dot = oracle.int_gemm(oracle.bit_plane(x, n - 1).astype(np.int32), w)
+            assert int(dot[0, 0]) == int(r[5])
+    assert int(oracle.int_gemm(x, w)[0, 0]) == s
+    assert int(oracle.planewise_gemm(x, 8, w)[0, 0]) == s
+
+
+@pytest.mark.parametrize("M,N,K,ka", [(3, 4, 5, 8), (7, 3, 33, 2), (2, 9, 100, 4)])
+def test_planewise_equals_integer_product_and_float64(M, N, K, ka):
+    rng = np.random.default_rng(M + N + K)
+    Q = rng.integers(0, 1 << ka, (M, K)).astype(np.int32)
+    B = np.where(rng.uniform(-1, 1, (K, N)) >= 0, 1, -1).astype(np.int32)
+    got = oracle.int_gemm(Q, B)
+    np.testing.assert_array_equal(got, oracle.planewise_gemm(Q, ka, B))
+    np.testing.assert_array_equal(got, (Q.astype(np.float64) @ B.astype(np.float64)).astype(np.int32))
+
+
+def test_one_bit_symmetric_case_reduces_to_xnor():
+    rng = np.random.default_rng(5)
+    X = rng.standard_normal((6, 70)).astype(np.float32)
+    W = rng.standard_normal((70, 5)).astype(np.float32)
+    qa = oracle.linear_quant_codes(np.where(X >= 0, 1.0, -1.0), 1, -1.0, 1.0)
+    qb = oracle.linear_quant_codes(np.where(W >= 0, 1.0, -1.0), 1, -1.0, 1.0)
+    got = oracle.int_gemm(oracle.codes_to_symmetric(qa, 1), oracle.codes_to_symmetric(qb, 1))
+    np.testing.assert_array_equal(got, oracle.xnor_gemm(X, W))
+
+
+def test_lstm_levels_roundtrip_and_real_product():
+    wl = workloads.lstm_gate(M=9, K=64, N=7, seed=4)
+    qa = oracle.linear_quant_codes(wl.X.numpy(), 4, -1.0, 1.0)
+    qb = oracle.linear_quant_codes(wl.W.numpy(), 4, -1.0, 1.0)
+    va = oracle.codes_to_symmetric(qa, 4)
+    vb = oracle.codes_to_symmetric(qb, 4)
+    # the generator's real values are exactly v/15
+    np.testing.assert_allclose(va / 15.0, wl.X.numpy().astype(np.float64), atol=1e-6)
+    got = oracle.int_gemm(va, vb)
+    real = wl.X.numpy().astype(np.float64) @ wl.W.numpy().astype(np.float64)
+    np.testing.assert_allclose(got / 225.0, real, atol=1e-4)
