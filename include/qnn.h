@@ -1,0 +1,278 @@
+/*
+ * qnn.h -- C ABI of the B200 (sm_100a) quantised-network forward library.
+ *
+ * The library implements the inference hot path of quantised / binarised
+ * neural networks: sign and k-bit linear quantisation of real tensors,
+ * bit-packing along the reduction dimension K, the 1-bit x 1-bit
+ * XNOR-popcount matrix product, k-bit operands as weighted sums of bit-plane
+ * products, batch-norm + sign folded to a per-channel integer threshold that
+ * emits packed bits for the next layer, and binary convolution through a
+ * packed im2col matrix.
+ *
+ * Conventions (all entry points):
+ *  - Every function returns an int status (QNN_OK = 0 or a QNN_ERR_* code),
+ *    never throws, aborts or traps.  qnn_last_error() returns a thread-local
+ *    text for the last failure.  Arguments are validated on the host BEFORE
+ *    anything is launched: a call that returns an error launched nothing.
+ *  - Unless a parameter says "host", every data pointer is a DEVICE pointer
+ *    owned by the caller; the library keeps no reference after the call.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    Calls are asynchronous on that stream and never synchronise it, except
+ *    the *_host entry points, which synchronise the stream before returning.
+ *  - The library allocates no device memory.  Calls that need scratch take a
+ *    caller workspace (`ws`, `ws_bytes`, 256-byte aligned) whose size is given
+ *    by qnn_workspace_bytes(); passing too little returns QNN_ERR_WORKSPACE.
+ *  - Leading dimensions are in elements (floats, int32, bytes) or, for packed
+ *    data, in 32-bit words.
+ *
+ * Canonical packed format (crosses the ABI between calls):
+ *    row-major uint32_t [rows, ld_words]; element k of a row is bit (k mod 32)
+ *    of word (k div 32), least significant bit = lowest k.  Bit 1 means +1
+ *    (sign data) or "plane bit set" (bit-plane data).  All pad bits of the
+ *    last used word (positions k >= K) are ZERO.  Words at index
+ *    >= ceil(K/32) of a row are ignored on input and untouched on output.
+ *    A k-bit tensor is `bits` such matrices, `plane_stride_words` apart;
+ *    plane i holds bit i of the integer code (i = 0 least significant, the
+ *    paper's plane n = i + 1 in Eq. 8).
+ *
+ * Operand value modes for bit-plane tensors:
+ *    QNN_MODE_U01  planes are {0,1}; the value is the unsigned code q = sum_i 2^i p_i
+ *    QNN_MODE_PM1  planes are {-1,+1}; the value is sum_i 2^i s_i = 2q - (2^bits - 1)
+ */
+#ifndef QNN_H_
+#define QNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define QNN_API __attribute__((visibility("default")))
+#else
+#define QNN_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QNN_VERSION 100
+
+/* status codes */
+#define QNN_OK 0
+#define QNN_ERR_INVALID_ARG 1 /* NULL pointer, negative size, bad enum, ld too small      */
+#define QNN_ERR_ALIGNMENT 2   /* pointer or leading dimension not aligned as documented   */
+#define QNN_ERR_UNSUPPORTED 3 /* valid request this build does not implement              */
+#define QNN_ERR_OVERFLOW 4    /* K * max|a| * max|b| does not fit int32                   */
+#define QNN_ERR_WORKSPACE 5   /* workspace missing, misaligned or too small               */
+#define QNN_ERR_CUDA 6        /* a CUDA runtime call failed (text in qnn_last_error)      */
+#define QNN_ERR_TIMEOUT 7     /* a bounded device-side wait ran out (see qnn_device_status) */
+
+/* matrix-product algorithms */
+#define QNN_ALGO_AUTO 0   /* library picks per shape                                      */
+#define QNN_ALGO_POPC 1   /* xor/and + popc on the CUDA cores (Eq. 11 as written)          */
+#define QNN_ALGO_TC_I8 2  /* values expanded to int8, tcgen05 kind::i8, TMEM accumulators */
+#define QNN_ALGO_B1_MMA 3 /* 1-bit mma.sync and/xor-popc (legacy tensor-core path)        */
+
+#define QNN_MODE_U01 0
+#define QNN_MODE_PM1 1
+
+/* operations, for qnn_workspace_bytes */
+#define QNN_OP_XNOR_GEMM 1
+#define QNN_OP_BITPLANE_GEMM 2
+#define QNN_OP_CONV2D 3
+#define QNN_OP_MLP 4
+
+QNN_API int qnn_version(void);
+QNN_API const char *qnn_status_string(int status);
+/* Thread-local description of the last error returned on this thread ("" if none). */
+QNN_API const char *qnn_last_error(void);
+
+/* ------------------------------------------------------------------------- */
+/* Quantise + pack                                                            */
+/* ------------------------------------------------------------------------- */
+
+/* Eq. 1 (deterministic binarisation) + the 32-per-word concatenation of Sec. 6.
+ * x: fp32 [rows, K] row-major, leading dimension ldx >= K.
+ * out: uint32 [rows, ld_words], ld_words >= ceil(K/32); bit = (x >= 0), so
+ * +0.0 and -0.0 give 1 and NaN gives 0.
+ * row_popc: optional int32 [rows], receives the number of set bits per row. */
+QNN_API int qnn_quantize_pack_sign(const float *x, int64_t rows, int64_t K, int64_t ldx, uint32_t *out,
+                           int64_t ld_words, int32_t *row_popc, void *stream);
+
+/* Same binarisation for a weight matrix stored as the paper writes it, W[K, N]
+ * row-major (ldw >= N): packs along K for every output unit n, producing
+ * out[N, ld_words] -- the "B" operand layout of the matrix products below. */
+QNN_API int qnn_quantize_pack_sign_t(const float *w, int64_t K, int64_t N, int64_t ldw, uint32_t *out,
+                             int64_t ld_words, int32_t *row_popc, void *stream);
+
+/* Eq. 1 for an NCHW activation tensor x[B,C,H,W] (dense): packs along the
+ * channel dimension into out[B,H,W,ceil(C/32)] words (dense NHWC bits), the
+ * input layout of qnn_binary_conv2d. */
+QNN_API int qnn_quantize_pack_sign_nchw(const float *x, int B, int C, int H, int W, uint32_t *out,
+                                void *stream);
+
+/* Eq. 9 read as a uniform quantiser with 2^bits levels on [lo, hi]
+ * (bits in 1..8): t = clip(x, lo, hi); code q = round_half_even((t - lo) * inv_step),
+ * inv_step = (2^bits - 1) / (hi - lo) evaluated in fp32; all steps are single
+ * IEEE fp32 operations (no fused multiply-add).  NaN gives code 0.
+ * Writes `bits` planes: planes + i * plane_stride_words is uint32 [rows, ld_words].
+ * row_sum_q: optional int32 [rows] = sum_k q[row, k]. */
+QNN_API int qnn_quantize_pack_kbit(const float *x, int64_t rows, int64_t K, int64_t ldx, int bits, float lo,
+                           float hi, uint32_t *planes, int64_t ld_words, int64_t plane_stride_words,
+                           int32_t *row_sum_q, void *stream);
+
+/* Transposed twin for weights W[K, N] row-major: planes are [N, ld_words], packed along K. */
+QNN_API int qnn_quantize_pack_kbit_t(const float *w, int64_t K, int64_t N, int64_t ldw, int bits, float lo,
+                             float hi, uint32_t *planes, int64_t ld_words, int64_t plane_stride_words,
+                             int32_t *row_sum_q, void *stream);
+
+/* Eq. 8 / Algorithm 4 first layer: splits unsigned fixed-point inputs x
+ * (uint8 [rows, K], ldx >= K bytes) into their `bits` (1..8) low bit-planes. */
+QNN_API int qnn_pack_planes_u8(const uint8_t *x, int64_t rows, int64_t K, int64_t ldx, int bits,
+                       uint32_t *planes, int64_t ld_words, int64_t plane_stride_words,
+                       int32_t *row_sum_q, void *stream);
+
+/* Section 5 binary convolution weights: w fp32 [Cout, C, KH, KW] (dense) is
+ * binarised with Eq. 1 and laid out as out[Cout, KH*KW*ceil(C/32)] words, the
+ * reduction ordered (kh, kw, channel word) to match the packed im2col rows. */
+QNN_API int qnn_pack_conv_weights(const float *w, int Cout, int C, int KH, int KW, uint32_t *out, void *stream);
+
+/* ------------------------------------------------------------------------- */
+/* Matrix products                                                            */
+/* ------------------------------------------------------------------------- */
+
+/* Algorithm 4 "XnorDotProduct" / Eq. 11:
+ * out[m, n] = sum_{k<K} a[m,k] * b[n,k] over +-1 values = K - 2 * popc(a XOR b).
+ * a: packed [M, lda], b: packed [N, ldb] (both packed along K, pad bits zero),
+ * out: int32 [M, ldo], ldo >= N.  K < 2^31.
+ * algo: QNN_ALGO_*; ws/ws_bytes: see qnn_workspace_bytes (may be NULL/0 for POPC). */
+QNN_API int qnn_xnor_gemm(const uint32_t *a, int64_t lda, const uint32_t *b, int64_t ldb, int64_t M,
+                  int64_t N, int64_t K, int32_t *out, int64_t ldo, int algo, void *ws,
+                  size_t ws_bytes, void *stream);
+
+/* The same product with Algorithm 4's Sign(BatchNorm(.)) folded in (see
+ * qnn_fold_bn): out_bits[m, n] = (dot[m,n] >= thr[n]) XOR flip[n], packed
+ * along n into uint32 [M, ld_words] -- the next layer's "a" operand.
+ * thr: int32 [N]; flip: uint8 [N] or NULL (all zero). */
+QNN_API int qnn_xnor_gemm_threshold(const uint32_t *a, int64_t lda, const uint32_t *b, int64_t ldb, int64_t M,
+                            int64_t N, int64_t K, const int32_t *thr, const uint8_t *flip,
+                            uint32_t *out_bits, int64_t ld_words, int algo, void *ws,
+                            size_t ws_bytes, void *stream);
+
+/* Eq. 8 generalised (Sec. 3: k-bit operands cost ka*kb binary products):
+ * out[m,n] = sum_k A[m,k] * B[n,k], where A, B are the integer values of the
+ * ka- and kb-plane tensors under their modes (QNN_MODE_*).
+ * a: ka planes of [M, lda], a_plane_stride words apart; b likewise [N, ldb].
+ * Requires K * (2^ka - 1) * (2^kb - 1) < 2^31, else QNN_ERR_OVERFLOW. */
+QNN_API int qnn_bitplane_gemm(const uint32_t *a, int ka, int a_mode, int64_t lda, int64_t a_plane_stride,
+                      const uint32_t *b, int kb, int b_mode, int64_t ldb, int64_t b_plane_stride,
+                      int64_t M, int64_t N, int64_t K, int32_t *out, int64_t ldo, int algo, void *ws,
+                      size_t ws_bytes, void *stream);
+
+QNN_API int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, int64_t lda,
+                                int64_t a_plane_stride, const uint32_t *b, int kb, int b_mode,
+                                int64_t ldb, int64_t b_plane_stride, int64_t M, int64_t N, int64_t K,
+                                const int32_t *thr, const uint8_t *flip, uint32_t *out_bits,
+                                int64_t ld_words, int algo, void *ws, size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------- */
+/* Threshold, rescale                                                         */
+/* ------------------------------------------------------------------------- */
+
+/* Algorithm 4, a^b = Sign(BatchNorm(a)): standalone form on an int32 matrix
+ * s[M, lds]: out[m, n] = (s[m,n] >= thr[n]) XOR flip[n], packed along n. */
+QNN_API int qnn_threshold_pack(const int32_t *s, int64_t M, int64_t N, int64_t lds, const int32_t *thr,
+                       const uint8_t *flip, uint32_t *out, int64_t ld_words, void *stream);
+
+/* HOST helper (host pointers, no GPU work): folds inference-time batch norm
+ * y = gamma * (s - mean) / sqrt(var + eps) + beta followed by Eq. 1 (y >= 0)
+ * into integers, in double precision:
+ *   gamma > 0: thr = ceil(tau),      flip = 0,  tau = mean - beta * sigma / gamma
+ *   gamma < 0: thr = floor(tau) + 1, flip = 1
+ *   gamma = 0: thr = INT32_MIN,      flip = (beta < 0)
+ * thr is clamped to the int32 range. */
+QNN_API int qnn_fold_bn(const double *gamma, const double *beta, const double *mean, const double *var,
+                double eps, int64_t N, int32_t *thr_host, uint8_t *flip_host);
+
+/* Algorithm 4 output layer (affine batch norm of the integer scores) and
+ * de-quantisation of affine codes:
+ * y[m,n] = alpha * p[m,n] + row_off[m] + col_off[n] + delta in fp32
+ * (row_off, col_off optional).  Evaluated as ((alpha*p + row) + col) + delta
+ * with separate roundings. */
+QNN_API int qnn_rescale_f32(const int32_t *p, int64_t M, int64_t N, int64_t ldp, float alpha,
+                    const float *row_off, const float *col_off, float delta, float *y, int64_t ldy,
+                    void *stream);
+
+/* ------------------------------------------------------------------------- */
+/* Binary convolution                                                         */
+/* ------------------------------------------------------------------------- */
+
+/* Section 5: out[b,co,y,x] = sum_{c,kh,kw} X[b,c,y*stride+kh-pad,x*stride+kw-pad] * Wt[co,c,kh,kw]
+ * over +-1 values (cross-correlation); a tap outside the image reads +1 when
+ * pad_bit = 1, -1 when pad_bit = 0.
+ * x: packed NHWC bits [B,H,W,ceil(C/32)] (qnn_quantize_pack_sign_nchw);
+ * w: [Cout, KH*KW*ceil(C/32)] (qnn_pack_conv_weights).
+ * Outputs (either may be NULL, not both): out_nchw int32 [B,Cout,Ho,Wo];
+ * out_bits packed NHWC [B,Ho,Wo,ceil(Cout/32)] = (out >= thr[co]) XOR flip[co]
+ * (thr required when out_bits is given).
+ * The packed im2col matrix [B*Ho*Wo, KH*KW*ceil(C/32)] lives in the workspace. */
+QNN_API int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint32_t *w, int Cout,
+                      int KH, int KW, int stride, int pad, int pad_bit, int32_t *out_nchw,
+                      const int32_t *thr, const uint8_t *flip, uint32_t *out_bits, int algo, void *ws,
+                      size_t ws_bytes, void *stream);
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 4 runner                                                         */
+/* ------------------------------------------------------------------------- */
+
+/* One layer of the MLP (a HOST struct; the pointers inside are device pointers). */
+typedef struct qnn_mlp_layer {
+    const uint32_t *w;   /* packed weights [N, ldw], packed along K           */
+    int64_t ldw;         /* words                                             */
+    int64_t K;           /* inputs of this layer                              */
+    int64_t N;           /* units of this layer                               */
+    const int32_t *thr;  /* int32 [N]; ignored for the last layer             */
+    const uint8_t *flip; /* uint8 [N] or NULL; ignored for the last layer     */
+} qnn_mlp_layer;
+
+/* Algorithm 4 "Running a BNN with L layers" on device buffers:
+ * layer 1 is the bit-plane product of the in_bits-bit input (Eq. 8), hidden
+ * layers are XNOR products with folded thresholds, the last layer returns
+ * int32 scores[M, layers[L-1].N] (its affine batch norm is qnn_rescale_f32).
+ * x: uint8 [M, layers[0].K] dense.  layers: HOST array of L structs. */
+QNN_API int qnn_mlp_forward(const uint8_t *x, int64_t M, int in_bits, const qnn_mlp_layer *layers, int L,
+                    int32_t *scores, int algo, void *ws, size_t ws_bytes, void *stream);
+
+/* Same, for callers holding HOST buffers: copies x_host (pinned memory
+ * recommended) to the device, runs the layers, copies the scores back to
+ * scores_host and synchronises `stream`.  The workspace must also hold the
+ * input and the scores: size it with qnn_mlp_workspace_bytes(..., 1). */
+QNN_API int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, const qnn_mlp_layer *layers,
+                         int L, int32_t *scores_host, int algo, void *ws, size_t ws_bytes,
+                         void *stream);
+
+QNN_API size_t qnn_mlp_workspace_bytes(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int algo,
+                               int host_io);
+
+/* ------------------------------------------------------------------------- */
+/* Workspace, status                                                          */
+/* ------------------------------------------------------------------------- */
+
+/* Scratch bytes for one call of `op` (QNN_OP_XNOR_GEMM, QNN_OP_BITPLANE_GEMM:
+ * M,N,K,ka,kb; QNN_OP_CONV2D: M = B*Ho*Wo, N = Cout, K = KH*KW*32*ceil(C/32),
+ * ka = kb = 1) under `algo`.  0 means no workspace is needed. */
+QNN_API size_t qnn_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int ka, int kb, int algo);
+
+/* Which algorithm QNN_ALGO_AUTO resolves to for a shape (never returns AUTO). */
+QNN_API int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int a_mode, int b_mode);
+
+/* Tensor-core kernels bound every device-side wait; when one runs out the
+ * kernel records it in a per-process device status word and exits cleanly.
+ * This call synchronises `stream`, reads and clears that word and returns
+ * QNN_OK or QNN_ERR_TIMEOUT. */
+QNN_API int qnn_device_status(void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QNN_H_ */

@@ -1,0 +1,236 @@
+"""ctypes binding of libqnn.so: argument marshalling only.
+
+Every function mirrors the C entry point of the same name (see include/qnn.h).
+Tensors are torch CUDA tensors; the binding passes their data pointers, sizes
+and the current CUDA stream, raises ``QnnError`` on a non-zero status and does
+no arithmetic of its own.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqnn.so")
+
+QNN_OK = 0
+QNN_ERR_INVALID_ARG, QNN_ERR_ALIGNMENT, QNN_ERR_UNSUPPORTED, QNN_ERR_OVERFLOW = 1, 2, 3, 4
+QNN_ERR_WORKSPACE, QNN_ERR_CUDA, QNN_ERR_TIMEOUT = 5, 6, 7
+QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA = 0, 1, 2, 3
+QNN_MODE_U01, QNN_MODE_PM1 = 0, 1
+QNN_OP_XNOR_GEMM, QNN_OP_BITPLANE_GEMM, QNN_OP_CONV2D, QNN_OP_MLP = 1, 2, 3, 4
+
+
+class QnnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({_lib.qnn_status_string(status).decode()}): "
+                         f"{_lib.qnn_last_error().decode()}")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_1609_07061_b200.build` "
+        "(nvcc, sm_100a).  There is no CPU fallback.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+i64, i32, vp, f32, sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
+
+
+class qnn_mlp_layer(ctypes.Structure):
+    _fields_ = [("w", vp), ("ldw", i64), ("K", i64), ("N", i64), ("thr", vp), ("flip", vp)]
+
+
+_SIGS = {
+    "qnn_version": (i32, []),
+    "qnn_status_string": (ctypes.c_char_p, [i32]),
+    "qnn_last_error": (ctypes.c_char_p, []),
+    "qnn_quantize_pack_sign": (i32, [vp, i64, i64, i64, vp, i64, vp, vp]),
+    "qnn_quantize_pack_sign_t": (i32, [vp, i64, i64, i64, vp, i64, vp, vp]),
+    "qnn_quantize_pack_sign_nchw": (i32, [vp, i32, i32, i32, i32, vp, vp]),
+    "qnn_quantize_pack_kbit": (i32, [vp, i64, i64, i64, i32, f32, f32, vp, i64, i64, vp, vp]),
+    "qnn_quantize_pack_kbit_t": (i32, [vp, i64, i64, i64, i32, f32, f32, vp, i64, i64, vp, vp]),
+    "qnn_pack_planes_u8": (i32, [vp, i64, i64, i64, i32, vp, i64, i64, vp, vp]),
+    "qnn_pack_conv_weights": (i32, [vp, i32, i32, i32, i32, vp, vp]),
+    "qnn_xnor_gemm": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
+    "qnn_xnor_gemm_threshold": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, vp, vp, i64, i32, vp, sz, vp]),
+    "qnn_bitplane_gemm": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
+    "qnn_bitplane_gemm_threshold": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, vp, vp,
+                                          i64, i32, vp, sz, vp]),
+    "qnn_threshold_pack": (i32, [vp, i64, i64, i64, vp, vp, vp, i64, vp]),
+    "qnn_fold_bn": (i32, [vp, vp, vp, vp, ctypes.c_double, i64, vp, vp]),
+    "qnn_rescale_f32": (i32, [vp, i64, i64, i64, f32, vp, vp, f32, vp, i64, vp]),
+    "qnn_binary_conv2d": (i32, [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, vp, sz, vp]),
+    "qnn_mlp_forward": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
+    "qnn_mlp_forward_host": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
+    "qnn_mlp_workspace_bytes": (sz, [i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
+    "qnn_workspace_bytes": (sz, [i32, i64, i64, i64, i32, i32, i32]),
+    "qnn_select_algo": (i32, [i64, i64, i64, i32, i32, i32, i32]),
+    "qnn_device_status": (i32, [vp]),
+}
+for _name, (_res, _args) in _SIGS.items():
+    _fn = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+EXPORTED = tuple(_SIGS.keys())
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream():
+    # without a CUDA device only host-side validation can succeed; any launch then returns QNN_ERR_CUDA
+    return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+
+
+def _ck(status: int, where: str):
+    if status != QNN_OK:
+        raise QnnError(status, where)
+
+
+def _ws(ws: Optional[torch.Tensor]):
+    return (None, 0) if ws is None else (ws.data_ptr(), ws.numel() * ws.element_size())
+
+
+def qnn_version() -> int:
+    return _lib.qnn_version()
+
+
+def qnn_status_string(status: int) -> str:
+    return _lib.qnn_status_string(status).decode()
+
+
+def qnn_last_error() -> str:
+    return _lib.qnn_last_error().decode()
+
+
+def qnn_quantize_pack_sign(x, rows, K, ldx, out, ld_words, row_popc=None):
+    _ck(_lib.qnn_quantize_pack_sign(_p(x), rows, K, ldx, _p(out), ld_words, _p(row_popc), _stream()),
+        "qnn_quantize_pack_sign")
+
+
+def qnn_quantize_pack_sign_t(w, K, N, ldw, out, ld_words, row_popc=None):
+    _ck(_lib.qnn_quantize_pack_sign_t(_p(w), K, N, ldw, _p(out), ld_words, _p(row_popc), _stream()),
+        "qnn_quantize_pack_sign_t")
+
+
+def qnn_quantize_pack_sign_nchw(x, B, C, H, W, out):
+    _ck(_lib.qnn_quantize_pack_sign_nchw(_p(x), B, C, H, W, _p(out), _stream()), "qnn_quantize_pack_sign_nchw")
+
+
+def qnn_quantize_pack_kbit(x, rows, K, ldx, bits, lo, hi, planes, ld_words, plane_stride_words, row_sum_q=None):
+    _ck(_lib.qnn_quantize_pack_kbit(_p(x), rows, K, ldx, bits, lo, hi, _p(planes), ld_words, plane_stride_words,
+                                    _p(row_sum_q), _stream()), "qnn_quantize_pack_kbit")
+
+
+def qnn_quantize_pack_kbit_t(w, K, N, ldw, bits, lo, hi, planes, ld_words, plane_stride_words, row_sum_q=None):
+    _ck(_lib.qnn_quantize_pack_kbit_t(_p(w), K, N, ldw, bits, lo, hi, _p(planes), ld_words, plane_stride_words,
+                                      _p(row_sum_q), _stream()), "qnn_quantize_pack_kbit_t")
+
+
+def qnn_pack_planes_u8(x, rows, K, ldx, bits, planes, ld_words, plane_stride_words, row_sum_q=None):
+    _ck(_lib.qnn_pack_planes_u8(_p(x), rows, K, ldx, bits, _p(planes), ld_words, plane_stride_words, _p(row_sum_q),
+                                _stream()), "qnn_pack_planes_u8")
+
+
+def qnn_pack_conv_weights(w, Cout, C, KH, KW, out):
+    _ck(_lib.qnn_pack_conv_weights(_p(w), Cout, C, KH, KW, _p(out), _stream()), "qnn_pack_conv_weights")
+
+
+def qnn_xnor_gemm(a, lda, b, ldb, M, N, K, out, ldo, algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_xnor_gemm(_p(a), lda, _p(b), ldb, M, N, K, _p(out), ldo, algo, wp, wb, _stream()), "qnn_xnor_gemm")
+
+
+def qnn_xnor_gemm_threshold(a, lda, b, ldb, M, N, K, thr, flip, out_bits, ld_words, algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_xnor_gemm_threshold(_p(a), lda, _p(b), ldb, M, N, K, _p(thr), _p(flip), _p(out_bits), ld_words, algo,
+                                     wp, wb, _stream()), "qnn_xnor_gemm_threshold")
+
+
+def qnn_bitplane_gemm(a, ka, a_mode, lda, a_plane_stride, b, kb, b_mode, ldb, b_plane_stride, M, N, K, out, ldo,
+                      algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_bitplane_gemm(_p(a), ka, a_mode, lda, a_plane_stride, _p(b), kb, b_mode, ldb, b_plane_stride, M, N, K,
+                               _p(out), ldo, algo, wp, wb, _stream()), "qnn_bitplane_gemm")
+
+
+def qnn_bitplane_gemm_threshold(a, ka, a_mode, lda, a_plane_stride, b, kb, b_mode, ldb, b_plane_stride, M, N, K, thr,
+                                flip, out_bits, ld_words, algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_bitplane_gemm_threshold(_p(a), ka, a_mode, lda, a_plane_stride, _p(b), kb, b_mode, ldb,
+                                         b_plane_stride, M, N, K, _p(thr), _p(flip), _p(out_bits), ld_words, algo, wp,
+                                         wb, _stream()), "qnn_bitplane_gemm_threshold")
+
+
+def qnn_threshold_pack(s, M, N, lds, thr, flip, out, ld_words):
+    _ck(_lib.qnn_threshold_pack(_p(s), M, N, lds, _p(thr), _p(flip), _p(out), ld_words, _stream()),
+        "qnn_threshold_pack")
+
+
+def qnn_fold_bn(gamma, beta, mean, var, eps, thr_host, flip_host):
+    """All arguments are CPU tensors (float64 in, int32 / uint8 out)."""
+    N = gamma.numel()
+    _ck(_lib.qnn_fold_bn(_p(gamma), _p(beta), _p(mean), _p(var), float(eps), N, _p(thr_host), _p(flip_host)),
+        "qnn_fold_bn")
+
+
+def qnn_rescale_f32(p, M, N, ldp, alpha, row_off, col_off, delta, y, ldy):
+    _ck(_lib.qnn_rescale_f32(_p(p), M, N, ldp, alpha, _p(row_off), _p(col_off), delta, _p(y), ldy, _stream()),
+        "qnn_rescale_f32")
+
+
+def qnn_binary_conv2d(x, B, C, H, W, w, Cout, KH, KW, stride, pad, pad_bit, out_nchw, thr, flip, out_bits,
+                      algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_binary_conv2d(_p(x), B, C, H, W, _p(w), Cout, KH, KW, stride, pad, pad_bit, _p(out_nchw), _p(thr),
+                               _p(flip), _p(out_bits), algo, wp, wb, _stream()), "qnn_binary_conv2d")
+
+
+def make_mlp_layers(ws: Sequence[torch.Tensor], ldws: Sequence[int], Ks: Sequence[int], Ns: Sequence[int],
+                    thrs: Sequence[Optional[torch.Tensor]], flips: Sequence[Optional[torch.Tensor]]):
+    """Builds the host array of qnn_mlp_layer structs (pointer marshalling only)."""
+    L = len(ws)
+    arr = (qnn_mlp_layer * L)()
+    for l in range(L):
+        arr[l].w = _p(ws[l])
+        arr[l].ldw = ldws[l]
+        arr[l].K = Ks[l]
+        arr[l].N = Ns[l]
+        arr[l].thr = _p(thrs[l]) if l < len(thrs) else None
+        arr[l].flip = _p(flips[l]) if l < len(flips) else None
+    return arr
+
+
+def qnn_mlp_workspace_bytes(M, in_bits, layers, algo=QNN_ALGO_AUTO, host_io=0) -> int:
+    return int(_lib.qnn_mlp_workspace_bytes(M, in_bits, layers, len(layers), algo, host_io))
+
+
+def qnn_mlp_forward(x, M, in_bits, layers, scores, algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_mlp_forward(_p(x), M, in_bits, layers, len(layers), _p(scores), algo, wp, wb, _stream()),
+        "qnn_mlp_forward")
+
+
+def qnn_mlp_forward_host(x_host, M, in_bits, layers, scores_host, algo=QNN_ALGO_AUTO, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_mlp_forward_host(_p(x_host), M, in_bits, layers, len(layers), _p(scores_host), algo, wp, wb,
+                                  _stream()), "qnn_mlp_forward_host")
+
+
+def qnn_workspace_bytes(op, M, N, K, ka=1, kb=1, algo=QNN_ALGO_AUTO) -> int:
+    return int(_lib.qnn_workspace_bytes(op, M, N, K, ka, kb, algo))
+
+
+def qnn_select_algo(M, N, K, ka=1, kb=1, a_mode=QNN_MODE_PM1, b_mode=QNN_MODE_PM1) -> int:
+    return int(_lib.qnn_select_algo(M, N, K, ka, kb, a_mode, b_mode))
+
+
+def qnn_device_status() -> int:
+    return int(_lib.qnn_device_status(_stream()))

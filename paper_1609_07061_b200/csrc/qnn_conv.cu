@@ -1,0 +1,144 @@
+// Binary convolution (Sec. 5) as a packed im2col followed by the XNOR matrix
+// product, plus the weight re-layout and the fp32 affine rescale.
+#include "qnn_internal.cuh"
+
+namespace qnn {
+namespace {
+
+// One thread per word of the im2col matrix col[m, (kh*KW + kw)*Cw + cw],
+// m = (b, yo, xo).  A tap outside the image reads the pad word: all valid
+// channel bits set for +1 padding, zero for -1 padding; bits of channels
+// >= C stay zero in every word so they cancel against the weights' zero pads.
+__global__ void __launch_bounds__(256) im2col_bits_kernel(const uint32_t *__restrict__ x, int B, int C, int H, int W,
+                                                          int KH, int KW, int stride, int pad, int pad_bit, int Ho,
+                                                          int Wo, uint32_t *__restrict__ col, int64_t total)
+{
+    const int Cw = (C + 31) >> 5;
+    const uint32_t tail_mask = (C & 31) ? ((1u << (C & 31)) - 1u) : 0xffffffffu;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int cw = (int)(e % Cw);
+        int64_t t = e / Cw;
+        const int kw = (int)(t % KW); t /= KW;
+        const int kh = (int)(t % KH); t /= KH;
+        const int xo = (int)(t % Wo); t /= Wo;
+        const int yo = (int)(t % Ho); t /= Ho;
+        const int b = (int)t;
+        const int yi = yo * stride + kh - pad;
+        const int xi = xo * stride + kw - pad;
+        uint32_t v;
+        if (yi >= 0 && yi < H && xi >= 0 && xi < W)
+            v = __ldg(x + (((int64_t)b * H + yi) * W + xi) * Cw + cw);
+        else
+            v = pad_bit ? ((cw == Cw - 1) ? tail_mask : 0xffffffffu) : 0u;
+        col[e] = v;
+    }
+}
+
+// One thread per output word out[co, (kh*KW + kw)*Cw + cw]: gathers 32 channels of one filter tap.
+__global__ void __launch_bounds__(256) conv_weight_pack_kernel(const float *__restrict__ w, int Cout, int C, int KH,
+                                                               int KW, uint32_t *__restrict__ out, int64_t total)
+{
+    const int Cw = (C + 31) >> 5;
+    const int taps = KH * KW;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int cw = (int)(e % Cw);
+        int64_t t = e / Cw;
+        const int tap = (int)(t % taps);
+        const int co = (int)(t / taps);
+        uint32_t word = 0;
+        for (int j = 0; j < 32; ++j) {
+            const int c = cw * 32 + j;
+            if (c < C) word |= (uint32_t)(__ldg(w + ((int64_t)co * C + c) * taps + tap) >= 0.0f) << j;
+        }
+        out[e] = word;
+    }
+}
+
+__global__ void __launch_bounds__(256) rescale_kernel(const int32_t *__restrict__ p, int64_t M, int64_t N, int64_t ldp,
+                                                      float alpha, const float *__restrict__ row_off,
+                                                      const float *__restrict__ col_off, float delta,
+                                                      float *__restrict__ y, int64_t ldy)
+{
+    const int64_t total = M * N;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t m = e / N, n = e - m * N;
+        float v = __fmul_rn(alpha, (float)p[m * ldp + n]);
+        if (row_off) v = __fadd_rn(v, row_off[m]);
+        if (col_off) v = __fadd_rn(v, col_off[n]);
+        v = __fadd_rn(v, delta);
+        y[m * ldy + n] = v;
+    }
+}
+
+inline int grid_for(int64_t total)
+{
+    const int64_t need = ceil_div(total, 256);
+    const int64_t cap = (int64_t)sm_count() * 16;
+    return (int)(need < cap ? need : cap);
+}
+
+}  // namespace
+}  // namespace qnn
+
+using namespace qnn;
+
+extern "C" {
+
+int qnn_pack_conv_weights(const float *w, int Cout, int C, int KH, int KW, uint32_t *out, void *stream)
+{
+    QNN_REQUIRE(Cout >= 0 && C >= 0 && KH >= 1 && KW >= 1, QNN_ERR_INVALID_ARG, "qnn_pack_conv_weights: bad sizes");
+    if (Cout == 0 || C == 0) return QNN_OK;
+    QNN_REQUIRE(w && out, QNN_ERR_INVALID_ARG, "qnn_pack_conv_weights: NULL pointer");
+    const int64_t total = (int64_t)Cout * KH * KW * ceil_div(C, 32);
+    conv_weight_pack_kernel<<<grid_for(total), 256, 0, as_stream(stream)>>>(w, Cout, C, KH, KW, out, total);
+    return check_launch("qnn_pack_conv_weights");
+}
+
+int qnn_rescale_f32(const int32_t *p, int64_t M, int64_t N, int64_t ldp, float alpha, const float *row_off,
+                    const float *col_off, float delta, float *y, int64_t ldy, void *stream)
+{
+    QNN_REQUIRE(M >= 0 && N >= 0, QNN_ERR_INVALID_ARG, "qnn_rescale_f32: negative size");
+    if (M == 0 || N == 0) return QNN_OK;
+    QNN_REQUIRE(p && y, QNN_ERR_INVALID_ARG, "qnn_rescale_f32: NULL pointer");
+    QNN_REQUIRE(ldp >= N && ldy >= N, QNN_ERR_INVALID_ARG, "qnn_rescale_f32: leading dimension too small");
+    rescale_kernel<<<grid_for(M * N), 256, 0, as_stream(stream)>>>(p, M, N, ldp, alpha, row_off, col_off, delta, y, ldy);
+    return check_launch("qnn_rescale_f32");
+}
+
+int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint32_t *w, int Cout, int KH, int KW,
+                      int stride, int pad, int pad_bit, int32_t *out_nchw, const int32_t *thr, const uint8_t *flip,
+                      uint32_t *out_bits, int algo, void *ws, size_t ws_bytes, void *stream)
+{
+    QNN_REQUIRE(B >= 0 && C >= 0 && H >= 0 && W >= 0 && Cout >= 0, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: negative size");
+    QNN_REQUIRE(KH >= 1 && KW >= 1 && stride >= 1 && pad >= 0 && (pad_bit == 0 || pad_bit == 1), QNN_ERR_INVALID_ARG,
+                "qnn_binary_conv2d: bad kernel, stride, pad or pad_bit");
+    if (B == 0 || C == 0 || Cout == 0 || H == 0 || W == 0) return QNN_OK;
+    QNN_REQUIRE(H + 2 * pad >= KH && W + 2 * pad >= KW, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: kernel larger than padded image");
+    QNN_REQUIRE(x && w, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: NULL operand");
+    QNN_REQUIRE(out_nchw || out_bits, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: no output buffer");
+    QNN_REQUIRE(!out_bits || thr, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: thresholds required for packed-bit output");
+    const int Ho = (H + 2 * pad - KH) / stride + 1;
+    const int Wo = (W + 2 * pad - KW) / stride + 1;
+    const int64_t Cw = ceil_div(C, 32);
+    const int64_t M = (int64_t)B * Ho * Wo;
+    const int64_t kwords = (int64_t)KH * KW * Cw;
+    const size_t col_bytes = round_up(sizeof(uint32_t) * (size_t)M * (size_t)kwords, 256);
+    QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= col_bytes, QNN_ERR_WORKSPACE,
+                "qnn_binary_conv2d: workspace of at least %zu bytes (256-byte aligned) required", col_bytes);
+    cudaStream_t st = as_stream(stream);
+    uint32_t *col = static_cast<uint32_t *>(ws);
+
+    GemmArgs g{};
+    g.a = col; g.lda = kwords; g.b = w; g.ldb = kwords; g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;
+    g.M = M; g.N = Cout; g.K = (int64_t)KH * KW * C; g.kwords = kwords;
+    g.epilogue = EPI_NCHW; g.out = out_nchw; g.hw = (int64_t)Ho * Wo;
+    g.thr = thr; g.flip = flip; g.out_bits = out_bits; g.ld_bits = ceil_div(Cout, 32);
+    if (int rc = validate_gemm(g)) return rc;
+
+    const int64_t total = M * kwords;
+    im2col_bits_kernel<<<grid_for(total), 256, 0, st>>>(x, B, C, H, W, KH, KW, stride, pad, pad_bit, Ho, Wo, col, total);
+    if (int rc = check_launch("qnn_binary_conv2d im2col")) return rc;
+    return run_gemm(g, algo, static_cast<char *>(ws) + col_bytes, ws_bytes - col_bytes, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,246 @@
+"""GPU parity on the paper-shaped workloads: convolution, the Algorithm-4 MLP, k-bit FC layers, big squares."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1609_07061_b200 import workloads
+from util import Guarded, as_i32_words, dev, pack_bits_ref, unpack_words, words_np, words_per_row
+
+pytestmark = pytest.mark.gpu
+
+ALGOS = [1, 2, 0]          # POPC, TC_I8, AUTO
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_1609_07061_b200.binding as b
+    return b
+
+
+def _skip_unsupported(q, e):
+    if e.status == q.QNN_ERR_UNSUPPORTED:
+        pytest.skip(str(e))
+    raise e
+
+
+def _conv_gpu(q, X, Wt, T, flip, stride, pad, pad_bit, algo, want_int=True, want_bits=True):
+    B, C, H, W = X.shape
+    Cout, _, KH, KW = Wt.shape
+    Ho = (H + 2 * pad - KH) // stride + 1
+    Wo = (W + 2 * pad - KW) // stride + 1
+    cw = words_per_row(C)
+    xb = torch.zeros(B, H, W, cw, dtype=torch.int32, device="cuda")
+    wb = torch.zeros(Cout, KH * KW * cw, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_sign_nchw(dev(X), B, C, H, W, xb)
+    q.qnn_pack_conv_weights(dev(Wt), Cout, C, KH, KW, wb)
+    out = Guarded((B, Cout, Ho, Wo), torch.int32, fill=-7) if want_int else None
+    bits = Guarded((B, Ho, Wo, words_per_row(Cout)), torch.int32, fill=0) if want_bits else None
+    n = q.qnn_workspace_bytes(q.QNN_OP_CONV2D, B * Ho * Wo, Cout, KH * KW * 32 * cw, 1, 1, algo)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    try:
+        q.qnn_binary_conv2d(xb, B, C, H, W, wb, Cout, KH, KW, stride, pad, pad_bit, out.t if out else None,
+                            dev(T) if want_bits else None, dev(flip) if (want_bits and flip is not None) else None,
+                            bits.t if bits else None, algo, ws)
+    except q.QnnError as e:
+        _skip_unsupported(q, e)
+    torch.cuda.synchronize()
+    if out: out.check()
+    if bits: bits.check()
+    return (out.t.cpu().numpy() if out else None), (words_np(bits.t) if bits else None)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("B,C,H,W,Co,KH,KW,stride,pad,pad_bit", [
+    (2, 3, 5, 6, 4, 3, 3, 1, 1, 1), (1, 33, 4, 4, 5, 3, 3, 1, 1, 1), (2, 64, 8, 8, 70, 3, 3, 1, 1, 1),
+    (2, 40, 7, 5, 33, 1, 1, 1, 0, 1), (1, 32, 9, 9, 16, 3, 3, 2, 1, 1), (1, 16, 6, 6, 8, 5, 3, 1, 2, 0),
+    (3, 256, 16, 16, 256, 3, 3, 1, 1, 1)])
+def test_conv2d(q, B, C, H, W, Co, KH, KW, stride, pad, pad_bit, algo):
+    rng = np.random.default_rng(B + C + H + Co)
+    X = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    Wt = rng.uniform(-1, 1, (Co, C, KH, KW)).astype(np.float32)
+    T = rng.integers(-16, 17, Co).astype(np.int32)
+    flip = rng.integers(0, 2, Co).astype(np.uint8)
+    want = oracle.conv2d(oracle.sign(X), oracle.sign(Wt), stride, pad, 1 if pad_bit else -1)
+    got, bits = _conv_gpu(q, X, Wt, T, flip, stride, pad, pad_bit, algo)
+    np.testing.assert_array_equal(got, want)
+    Bn, _, Ho, Wo = want.shape
+    rows = want.transpose(0, 2, 3, 1).reshape(-1, Co)
+    np.testing.assert_array_equal(unpack_words(bits.reshape(-1, words_per_row(Co)), Co), oracle.threshold(rows, T, flip))
+    # bits-only and int-only calls agree with the combined call
+    got2, _ = _conv_gpu(q, X, Wt, T, flip, stride, pad, pad_bit, algo, want_int=True, want_bits=False)
+    _, bits2 = _conv_gpu(q, X, Wt, T, flip, stride, pad, pad_bit, algo, want_int=False, want_bits=True)
+    np.testing.assert_array_equal(got2, want)
+    np.testing.assert_array_equal(bits2, bits)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_cifar_conv_config_sampled(q, algo):
+    """Config 4 at full size on the GPU; the oracle checks three whole images (first, middle, last)."""
+    wl = workloads.cifar_conv()
+    X, Wt, T = wl.X.numpy(), wl.W.numpy(), wl.T.numpy()
+    got, bits = _conv_gpu(q, X, Wt, T, None, 1, 1, 1, algo)
+    ws = oracle.sign(Wt)
+    for b in (0, 63, 127):
+        want = oracle.conv2d(oracle.sign(X[b:b + 1]), ws, 1, 1, 1)
+        np.testing.assert_array_equal(got[b:b + 1], want)
+        rows = want.transpose(0, 2, 3, 1).reshape(-1, 256)
+        np.testing.assert_array_equal(unpack_words(bits[b].reshape(-1, 8), 256), oracle.threshold(rows, T))
+    # property over the whole output: parity and bound of a +-1 sum of 2304 terms
+    assert np.all(np.abs(got) <= 2304) and np.all(got % 2 == 0)
+
+
+def _mlp_gpu(q, wl, M, algo, host=False, in_bits=8):
+    dims = wl.dims
+    packed, ldws = [], []
+    for W in wl.Ws:
+        K, N = W.shape
+        ld = (words_per_row(K) + 3) // 4 * 4
+        out = torch.zeros(N, ld, dtype=torch.int32, device="cuda")
+        q.qnn_quantize_pack_sign_t(W.cuda(), K, N, N, out, ld)
+        packed.append(out); ldws.append(ld)
+    thr = [t.cuda() for t in wl.Ts]
+    layers = q.make_mlp_layers(packed, ldws, dims[:-1], dims[1:], thr, [None] * len(thr))
+    n = q.qnn_mlp_workspace_bytes(M, in_bits, layers, algo, 1 if host else 0)
+    ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+    try:
+        if host:
+            xh = wl.X[:M].contiguous().pin_memory()
+            sh = torch.empty(M, dims[-1], dtype=torch.int32).pin_memory()
+            q.qnn_mlp_forward_host(xh, M, in_bits, layers, sh, algo, ws)
+            return sh.numpy().copy()
+        scores = Guarded((M, dims[-1]), torch.int32, fill=-7)
+        q.qnn_mlp_forward(wl.X[:M].cuda(), M, in_bits, layers, scores.t, algo, ws)
+        torch.cuda.synchronize()
+        scores.check()
+        return scores.t.cpu().numpy()
+    except q.QnnError as e:
+        _skip_unsupported(q, e)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("M,dims", [(1, (784, 64, 10)), (37, (50, 40, 24, 10)), (200, (784, 512, 256, 10)),
+                                    (130, (100, 300, 10)), (5, (33, 7))])
+def test_mlp_forward_small(q, M, dims, algo):
+    wl = workloads.mnist_mlp(M=M, dims=dims, seed=1)
+    want = oracle.mlp_forward(wl.X.numpy().astype(np.int32), [oracle.sign(w.numpy()) for w in wl.Ws],
+                              [t.numpy() for t in wl.Ts])
+    np.testing.assert_array_equal(_mlp_gpu(q, wl, M, algo), want)
+    np.testing.assert_array_equal(_mlp_gpu(q, wl, M, algo, host=True), want)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_mnist_mlp_config_sampled(q, algo):
+    """Config 2 at full size (batch 10000, the launch configuration bench.py times); batch rows are independent,
+    so the oracle runs the whole network on a sample of rows spread over several tiles and the ragged tail."""
+    wl = workloads.mnist_mlp()
+    got = _mlp_gpu(q, wl, 10000, algo)
+    rows = np.array([0, 1, 63, 64, 127, 128, 129, 255, 256, 1000, 4095, 4096, 5000, 7777, 9983, 9984, 9985, 9998, 9999])
+    want = oracle.mlp_forward(wl.X.numpy()[rows].astype(np.int32), [oracle.sign(w.numpy()) for w in wl.Ws],
+                              [t.numpy() for t in wl.Ts])
+    np.testing.assert_array_equal(got[rows], want)
+    # properties that hold for every row: scores have the parity of K = 4096 and are bounded by it
+    assert np.all(got % 2 == 0) and np.all(np.abs(got) <= 4096)
+    np.testing.assert_array_equal(_mlp_gpu(q, wl, 10000, algo, host=True), got)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("layer", [0, 1, 2])
+def test_alexnet_fc_config(q, layer, algo):
+    """Config 3: 2-bit activations on [0,1] x 1-bit weights, GPU quantisers + bit-plane product; oracle on sampled rows."""
+    wl = workloads.alexnet_fc()
+    X, W = wl.Xs[layer], wl.Ws[layer]
+    M, K = X.shape
+    N = W.shape[1]
+    ld = words_per_row(K)
+    ap = torch.zeros(2, M, ld, dtype=torch.int32, device="cuda")
+    bp = torch.zeros(N, ld, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_kbit(X.cuda(), M, K, K, 2, 0.0, 1.0, ap, ld, M * ld)
+    q.qnn_quantize_pack_sign_t(W.cuda(), K, N, N, bp, ld)
+    out = Guarded((M, N), torch.int32, fill=-7)
+    n = q.qnn_workspace_bytes(q.QNN_OP_BITPLANE_GEMM, M, N, K, 2, 1, algo)
+    ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
+    try:
+        q.qnn_bitplane_gemm(ap, 2, q.QNN_MODE_U01, ld, M * ld, bp, 1, q.QNN_MODE_PM1, ld, 0, M, N, K, out.t, N, algo, ws)
+    except q.QnnError as e:
+        _skip_unsupported(q, e)
+    torch.cuda.synchronize()
+    out.check()
+    rows = np.array([0, 1, 31, 64, 127, 128, 200, 255])
+    codes = oracle.linear_quant_codes(X.numpy()[rows], 2, 0.0, 1.0)
+    want = oracle.int_gemm(codes, oracle.sign(W.numpy()))
+    np.testing.assert_array_equal(out.t.cpu().numpy()[rows], want)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_lstm_gate_config(q, algo):
+    """Config 5, recurrent part: 4-bit x 4-bit signed levels, 700 x 4096 x 2048; oracle on sampled rows."""
+    wl = workloads.lstm_gate()
+    M, K = wl.X.shape
+    N = wl.W.shape[1]
+    ld = words_per_row(K)
+    ap = torch.zeros(4, M, ld, dtype=torch.int32, device="cuda")
+    bp = torch.zeros(4, N, ld, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_kbit(wl.X.cuda(), M, K, K, 4, -1.0, 1.0, ap, ld, M * ld)
+    q.qnn_quantize_pack_kbit_t(wl.W.cuda(), K, N, N, 4, -1.0, 1.0, bp, ld, N * ld)
+    out = Guarded((M, N), torch.int32, fill=-7)
+    n = q.qnn_workspace_bytes(q.QNN_OP_BITPLANE_GEMM, M, N, K, 4, 4, algo)
+    ws = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
+    try:
+        q.qnn_bitplane_gemm(ap, 4, q.QNN_MODE_PM1, ld, M * ld, bp, 4, q.QNN_MODE_PM1, ld, N * ld, M, N, K, out.t, N,
+                            algo, ws)
+    except q.QnnError as e:
+        _skip_unsupported(q, e)
+    torch.cuda.synchronize()
+    out.check()
+    rows = np.array([0, 1, 63, 64, 127, 128, 500, 639, 640, 698, 699])
+    va = oracle.codes_to_symmetric(oracle.linear_quant_codes(wl.X.numpy()[rows], 4, -1.0, 1.0), 4)
+    vb = oracle.codes_to_symmetric(oracle.linear_quant_codes(wl.W.numpy(), 4, -1.0, 1.0), 4)
+    np.testing.assert_array_equal(out.t.cpu().numpy()[rows], oracle.int_gemm(va, vb))
+
+
+def _square(q, n, algo):
+    wl = workloads.square_gemm(n)
+    ld = words_per_row(n)
+    a = torch.zeros(n, ld, dtype=torch.int32, device="cuda")
+    b = torch.zeros(n, ld, dtype=torch.int32, device="cuda")
+    Xd = wl.X.cuda()
+    q.qnn_quantize_pack_sign(Xd, n, n, n, a, ld)
+    del Xd
+    Wd = wl.W.cuda()
+    q.qnn_quantize_pack_sign_t(Wd, n, n, n, b, ld)
+    del Wd
+    out = torch.empty(n, n, dtype=torch.int32, device="cuda")
+    nws = q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, n, n, n, 1, 1, algo)
+    ws = torch.empty(max(nws, 256), dtype=torch.uint8, device="cuda")
+    try:
+        q.qnn_xnor_gemm(a, ld, b, ld, n, n, n, out, n, algo, ws)
+    except q.QnnError as e:
+        _skip_unsupported(q, e)
+    torch.cuda.synchronize()
+    return wl, out
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_square_1024_full(q, algo):
+    wl, out = _square(q, 1024, algo)
+    np.testing.assert_array_equal(out.cpu().numpy(), oracle.xnor_gemm(wl.X.numpy(), wl.W.numpy()))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_square_large_sampled_and_checksums(q, n, algo):
+    """Sizes where the scalar oracle cannot run whole: exact oracle on sampled full rows and full columns, plus
+    int64 row-sum and column-sum checksums that cover every output:
+      sum_n out[m,n] = a_m . (sum_n w_n)   and   sum_m out[m,n] = (sum_m a_m) . w_n ."""
+    wl, out = _square(q, n, algo)
+    X, W = wl.X.numpy(), wl.W.numpy()
+    got = out.cpu().numpy()
+    rows = np.array([0, 1, 127, 128, n // 2 + 1, n - 129, n - 2, n - 1])
+    cols = np.array([0, 5, 127, 128, 255, n // 2, n - 128, n - 1])
+    np.testing.assert_array_equal(got[rows], oracle.xnor_gemm(X[rows], W))
+    np.testing.assert_array_equal(got[:, cols], oracle.xnor_gemm(X, np.ascontiguousarray(W[:, cols])))
+    sa = oracle.sign(X).astype(np.int64)
+    sw = oracle.sign(W).astype(np.int64)
+    np.testing.assert_array_equal(got.sum(axis=1, dtype=np.int64), sa @ sw.sum(axis=1))
+    np.testing.assert_array_equal(got.sum(axis=0, dtype=np.int64), sa.sum(axis=0) @ sw)
