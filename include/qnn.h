@@ -272,6 +272,10 @@ QNN_API int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int
  * QNN_OK or QNN_ERR_TIMEOUT. */
 QNN_API int qnn_device_status(void *stream);
 
+/* Number of kernels this library has launched in this process so far (all
+ * threads, all streams); a monotonically increasing bookkeeping counter. */
+QNN_API uint64_t qnn_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

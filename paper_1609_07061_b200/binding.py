@@ -71,6 +71,7 @@ _SIGS = {
     "qnn_workspace_bytes": (sz, [i32, i64, i64, i64, i32, i32, i32]),
     "qnn_select_algo": (i32, [i64, i64, i64, i32, i32, i32, i32]),
     "qnn_device_status": (i32, [vp]),
+    "qnn_launch_count": (ctypes.c_uint64, []),
 }
 for _name, (_res, _args) in _SIGS.items():
     _fn = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
@@ -234,3 +235,7 @@ def qnn_select_algo(M, N, K, ka=1, kb=1, a_mode=QNN_MODE_PM1, b_mode=QNN_MODE_PM
 
 def qnn_device_status() -> int:
     return int(_lib.qnn_device_status(_stream()))
+
+
+def qnn_launch_count() -> int:
+    return int(_lib.qnn_launch_count())

@@ -3,12 +3,14 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <atomic>
 #include <climits>
 #include "qnn_internal.cuh"
 
 namespace qnn {
 
 static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_launches{0};
 
 int fail(int code, const char *fmt, ...)
 {
@@ -23,6 +25,7 @@ void clear_error() { g_err[0] = 0; }
 
 int check_launch(const char *what)
 {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(QNN_ERR_CUDA, "%s: launch failed: %s", what, cudaGetErrorString(e));
     return QNN_OK;
@@ -65,6 +68,8 @@ const char *qnn_status_string(int status)
 }
 
 const char *qnn_last_error(void) { return qnn::g_err; }
+
+uint64_t qnn_launch_count(void) { return qnn::g_launches.load(std::memory_order_relaxed); }
 
 int qnn_fold_bn(const double *gamma, const double *beta, const double *mean, const double *var,
                 double eps, int64_t N, int32_t *thr_host, uint8_t *flip_host)
