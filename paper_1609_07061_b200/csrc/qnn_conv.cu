@@ -131,6 +131,7 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
     GemmArgs g{};
     g.a = col; g.lda = kwords; g.b = w; g.ldb = kwords; g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;
     g.M = M; g.N = Cout; g.K = (int64_t)KH * KW * C; g.kwords = kwords;
+    g.pad_period = Cw; g.pad_tail = (int)(C - 32 * (Cw - 1));
     g.epilogue = EPI_NCHW; g.out = out_nchw; g.hw = (int64_t)Ho * Wo;
     g.thr = thr; g.flip = flip; g.out_bits = out_bits; g.ld_bits = ceil_div(Cout, 32);
     if (int rc = validate_gemm(g)) return rc;

@@ -45,6 +45,8 @@ struct GemmArgs {
     int ka, kb, a_mode, b_mode;
     int64_t M, N, K;        // K = number of real products per output (sets the constant term)
     int64_t kwords;         // words per row to reduce over; 0 = ceil(K/32) (conv rows carry interior pad bits)
+    int64_t pad_period;     // > 0: every pad_period-th word holds only pad_tail valid bits (conv: words per tap)
+    int pad_tail;
     int epilogue;           // Epilogue
     int32_t *out;           // EPI_ROWMAJOR / EPI_NCHW
     int64_t ldo;            // EPI_ROWMAJOR

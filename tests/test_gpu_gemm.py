@@ -41,6 +41,7 @@ def _run_xnor(q, X, W, algo, lda_pad=0, ldo_pad=0):
             pytest.skip(f"algo {algo} does not support this shape: {e}")
         raise
     torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
     out.check()
     res = out.t.cpu().numpy()
     if ldo_pad:
