@@ -62,7 +62,7 @@ def _ops(M):
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
 
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -76,12 +76,14 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(prefix="qnn_clocks_", suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.gpu)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Summarises the samples whose wall-clock timestamp lies in [t_begin, t_end] (all samples if none given)."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -98,6 +100,9 @@ class ClockSampler:
                     if len(c) < 9:
                         continue
                     try:
+                        ts = datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                        if t_begin is not None and not (t_begin - 0.05 <= ts <= t_end + 0.05):
+                            continue
                         sm.append(float(c[1])); mx.append(float(c[2]))
                     except ValueError:
                         continue
@@ -109,8 +114,7 @@ class ClockSampler:
         except Exception:
             pass
         if sm:
-            # under-load samples: the upper half of what was seen (idle samples sit at the low clock)
-            out["sm_mhz"] = statistics.median(sorted(sm)[len(sm) // 2:])
+            out["sm_mhz"] = statistics.median(sm)
             out["sm_max_mhz"] = max(mx)
             out["samples"] = len(sm)
         out["reasons"] = sorted(reasons)
@@ -178,11 +182,9 @@ class MlpBench:
                                       q.QNN_MODE_PM1, self.ldws[0], 0, M, DIMS[1], DIMS[0], self.thr[0], None,
                                       self.act[0], 128, self.algo, self.gws)
         if ev is not None:
-            ev[0].record()
+            q.qnn_set_kernel_events(ev[0], ev[1])        # recorded by the library right around the product kernel
         q.qnn_xnor_gemm_threshold(self.act[0], 128, self.packed[1], self.ldws[1], M, DIMS[2], DIMS[1], self.thr[1],
                                   None, self.act[1], 128, self.algo, self.gws)
-        if ev is not None:
-            ev[1].record()
         q.qnn_xnor_gemm_threshold(self.act[1], 128, self.packed[2], self.ldws[2], M, DIMS[3], DIMS[2], self.thr[2],
                                   None, self.act[0], 128, self.algo, self.gws)
         q.qnn_xnor_gemm(self.act[0], 128, self.packed[3], self.ldws[3], M, DIMS[4], DIMS[3], self.scores, DIMS[4],
@@ -196,7 +198,7 @@ def _cpu_baseline(sample_rows: int = 0, budget_s: float = 15.0):
     """The oracle as it stands, on the host cores, on a bounded sample of batch rows of the same workload."""
     import oracle
     from paper_1609_07061_b200 import workloads
-    wl = workloads.mnist_mlp(M=256, dims=DIMS, seed=1)
+    wl = workloads.mnist_mlp(M=BATCH if sample_rows <= 0 else sample_rows, dims=DIMS, seed=1)
     Ws = [oracle.sign(w.numpy()) for w in wl.Ws]
     Ts = [t.numpy() for t in wl.Ts]
     x = wl.X.numpy().astype(np.int32)
@@ -204,7 +206,7 @@ def _cpu_baseline(sample_rows: int = 0, budget_s: float = 15.0):
         t0 = time.perf_counter()
         oracle.mlp_forward(x[:8], Ws, Ts)
         t8 = time.perf_counter() - t0
-        sample_rows = int(max(8, min(256, 8 * budget_s / max(t8, 1e-3))))
+        sample_rows = int(max(8, min(BATCH, 8 * budget_s / max(t8, 1e-3))))
     t0 = time.perf_counter()
     oracle.mlp_forward(x[:sample_rows], Ws, Ts)
     dt = time.perf_counter() - t0
@@ -375,7 +377,7 @@ def run_extras(q, bench, peaks, algo):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--algo", default="auto", choices=["auto", "popc", "tc_i8", "b1_mma"])
@@ -405,11 +407,12 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident arm ----------------------------------------------------
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         bench.step_calls()
     barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
+    t_begin = time.time()
     launches0 = q.qnn_launch_count()
     step_ev, dom_ev = [], []
     barrier()
@@ -417,13 +420,13 @@ def main():
         bench.flush_l2()
         s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(); d1.record()                         # creates the underlying handles; re-recorded by the library
         s.record()
         bench.step_calls(ev=(d0, d1))
         e.record()
         step_ev.append((s, e)); dom_ev.append((d0, d1))
     barrier()
     launches = q.qnn_launch_count() - launches0
-    clocks = sampler.stop()
     total_ms = sum(s.elapsed_time(e) for s, e in step_ev)
     dom_ms = sum(a.elapsed_time(b) for a, b in dom_ev) / args.steps
     if q.qnn_device_status() != 0:
@@ -441,6 +444,8 @@ def main():
         e2e_ev.append((s, e))
     barrier()
     e2e_ms = sum(s.elapsed_time(e) for s, e in e2e_ev)
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end)
     same = bool(torch.equal(bench.scores_host, bench.scores.cpu()))
 
     if world > 1:
@@ -462,7 +467,7 @@ def main():
             # int8 tensor peak = measured bf16 peak x the nominal int8:bf16 ratio (2), sustained figure inside a step
             bound, peak = "tensor", 2.0 * peaks["bf16_tflops_sustained"]
             peak_note = f"2 x {peaks['source']} sustained bf16 ({peaks['bf16_tflops_sustained']} TF/s); one int8 MAC = one +-1 product"
-            kernel = "tcgen05 kind::i8 xnor product 10000x4096x4096 (+ int8 expansion)"
+            kernel = "tcgen05 kind::i8 xnor product 10000x4096x4096, threshold epilogue (gemm_i8_kernel)"
             dtype = "int8"
         else:
             # xor+popc+add on the CUDA cores: the popc unit issues 16 lanes/clk/SM -> 148 SM x 16 x 64 binary ops/clk

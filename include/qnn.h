@@ -272,6 +272,13 @@ QNN_API int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int
  * QNN_OK or QNN_ERR_TIMEOUT. */
 QNN_API int qnn_device_status(void *stream);
 
+/* Measurement aid: arms two cudaEvent_t handles (passed as void*) on the calling
+ * thread.  The next matrix-product call made by this thread records `start`
+ * immediately before and `stop` immediately after its product kernel (not
+ * around operand expansion or im2col), on that call's stream, and disarms
+ * them.  Pass NULLs to disarm. */
+QNN_API int qnn_set_kernel_events(void *start, void *stop);
+
 /* Number of kernels this library has launched in this process so far (all
  * threads, all streams); a monotonically increasing bookkeeping counter. */
 QNN_API uint64_t qnn_launch_count(void);

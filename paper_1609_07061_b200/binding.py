@@ -72,6 +72,7 @@ _SIGS = {
     "qnn_select_algo": (i32, [i64, i64, i64, i32, i32, i32, i32]),
     "qnn_device_status": (i32, [vp]),
     "qnn_launch_count": (ctypes.c_uint64, []),
+    "qnn_set_kernel_events": (i32, [vp, vp]),
 }
 for _name, (_res, _args) in _SIGS.items():
     _fn = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
@@ -239,3 +240,10 @@ def qnn_device_status() -> int:
 
 def qnn_launch_count() -> int:
     return int(_lib.qnn_launch_count())
+
+
+def qnn_set_kernel_events(start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]):
+    """Arms two torch CUDA events (already created, i.e. recorded once) around the next product kernel."""
+    a = None if start is None else start.cuda_event
+    b = None if stop is None else stop.cuda_event
+    _ck(_lib.qnn_set_kernel_events(a, b), "qnn_set_kernel_events")

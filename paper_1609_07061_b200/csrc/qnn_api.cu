@@ -22,6 +22,7 @@ int fail(int code, const char *fmt, ...)
 }
 
 void clear_error() { g_err[0] = 0; }
+void profile_arm(cudaEvent_t a, cudaEvent_t b);
 
 int check_launch(const char *what)
 {
@@ -30,6 +31,19 @@ int check_launch(const char *what)
     if (e != cudaSuccess) return fail(QNN_ERR_CUDA, "%s: launch failed: %s", what, cudaGetErrorString(e));
     return QNN_OK;
 }
+
+static thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+
+void profile_before(cudaStream_t st)
+{
+    if (g_ev_start) cudaEventRecord(g_ev_start, st);
+}
+void profile_after(cudaStream_t st)
+{
+    if (g_ev_stop) cudaEventRecord(g_ev_stop, st);
+    g_ev_start = g_ev_stop = nullptr;
+}
+void profile_arm(cudaEvent_t a, cudaEvent_t b) { g_ev_start = a; g_ev_stop = b; }
 
 int sm_count()
 {
@@ -51,6 +65,13 @@ int sm_count()
 extern "C" {
 
 int qnn_version(void) { return QNN_VERSION; }
+
+int qnn_set_kernel_events(void *start, void *stop)
+{
+    QNN_REQUIRE((start == nullptr) == (stop == nullptr), QNN_ERR_INVALID_ARG, "qnn_set_kernel_events: pass both events or neither");
+    qnn::profile_arm(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop));
+    return QNN_OK;
+}
 
 const char *qnn_status_string(int status)
 {

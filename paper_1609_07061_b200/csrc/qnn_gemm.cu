@@ -130,8 +130,14 @@ int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, int64_t l
 
 int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int a_mode, int b_mode)
 {
-    (void)M; (void)N; (void)K; (void)ka; (void)kb; (void)a_mode; (void)b_mode;
-    return QNN_ALGO_POPC;
+    // Measured on B200: the 1-bit mma.sync path never beats xor+popc on the CUDA cores, so it is never picked.
+    // The tcgen05 int8 path costs one pass whatever the plane counts and overtakes the CUDA-core path once the
+    // equivalent plane-pair work M*N*K*ka*kb reaches about 2^31; below that its expansion passes and launch
+    // latencies dominate.
+    if (M <= 0 || N <= 0 || K <= 0) return QNN_ALGO_POPC;
+    if ((a_mode == QNN_MODE_PM1 && ka > 7) || (b_mode == QNN_MODE_PM1 && kb > 7)) return QNN_ALGO_POPC;
+    const double work = (double)M * (double)N * (double)K * (double)ka * (double)kb;
+    return work >= 2147483648.0 ? QNN_ALGO_TC_I8 : QNN_ALGO_POPC;
 }
 
 size_t qnn_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int ka, int kb, int algo)

@@ -168,7 +168,9 @@ int launch_gemm_b1mma(const GemmArgs &g, cudaStream_t st)
     const int64_t gy = ceil_div(g.M, B1_BM);
     QNN_REQUIRE(gy <= 65535, QNN_ERR_UNSUPPORTED, "b1 mma path: M too large for the launch grid");
     dim3 grid((unsigned)ceil_div(g.N, B1_BN), (unsigned)gy);
+    profile_before(st);
     gemm_b1_kernel<<<grid, B1_THREADS, 0, st>>>(P);
+    profile_after(st);
     return check_launch("b1 mma gemm");
 }
 

@@ -229,7 +229,9 @@ int launch_cfg(const PopcParams &P, cudaStream_t st)
     const int64_t gx = ceil_div(g.N, BN), gy = ceil_div(g.M, BM);
     QNN_REQUIRE(gy <= 65535, QNN_ERR_UNSUPPORTED, "popc gemm: M too large for the launch grid");
     dim3 grid((unsigned)gx, (unsigned)gy);
+    profile_before(st);
     kern<<<grid, THREADS, smem, st>>>(P);
+    profile_after(st);
     return check_launch("popc gemm");
 }
 

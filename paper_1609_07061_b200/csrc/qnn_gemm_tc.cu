@@ -267,14 +267,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
                 uint32_t w = 0;
                 if (p.out_bits != nullptr && n0 < p.N) {
+                    // lane j fetches the threshold (and flip) of column n0 + j once; the row loop reads them by shuffle
+                    const bool ncol = (n0 + lane) < p.N;
+                    const int32_t tl = ncol ? __ldg(p.thr + n0 + lane) : 0;
+                    const uint32_t fl = (ncol && p.flip) ? (uint32_t)(__ldg(p.flip + n0 + lane) != 0) : 0u;
+                    const uint32_t fmask = __ballot_sync(0xffffffffu, fl != 0);
+                    const uint32_t nmask = __ballot_sync(0xffffffffu, ncol);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
-                        if (n0 + j < p.N) {
-                            uint32_t b = (int32_t)v[j] >= __ldg(p.thr + n0 + j);
-                            if (p.flip) b ^= (uint32_t)(__ldg(p.flip + n0 + j) != 0);
-                            w |= b << j;
-                        }
+                        const int32_t tj = __shfl_sync(0xffffffffu, tl, j);
+                        w |= (uint32_t)((int32_t)v[j] >= tj) << j;
                     }
+                    w = (w ^ fmask) & nmask;
                 }
                 words[c] = w;
             }
@@ -388,7 +392,9 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cuda
     p.idesc |= (uint32_t)(BN >> 3) << 17;
     const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    profile_before(st);
     kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, p);
+    profile_after(st);
     return check_launch("tc gemm");
 }
 

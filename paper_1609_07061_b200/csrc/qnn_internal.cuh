@@ -34,6 +34,10 @@ int check_launch(const char *what);
 
 int sm_count();
 
+// Armed measurement events (see qnn_set_kernel_events): call around the product kernel launch.
+void profile_before(cudaStream_t st);
+void profile_after(cudaStream_t st);
+
 // ---- internal launchers shared between translation units -------------------
 
 enum Epilogue { EPI_ROWMAJOR = 0, EPI_NCHW = 1, EPI_BITS = 2 };
