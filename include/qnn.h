@@ -175,6 +175,36 @@ QNN_API int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, i
                                 const int32_t *thr, const uint8_t *flip, uint32_t *out_bits,
                                 int64_t ld_words, int algo, void *ws, size_t ws_bytes, void *stream);
 
+/* Size of the scratch array built into the library for qnn_xnor_gemm_noalloc. */
+#define QNN_NOALLOC_SCRATCH_BYTES (8u << 20)
+
+/* The paper has no counterpart for this call; it is a packaging variant of
+ * qnn_xnor_gemm (same arguments, same int32 result, always the tensor-core
+ * algorithm) for callers that cannot allocate device memory or size a
+ * workspace when they call: code running on a latency-critical serving thread
+ * where cudaMalloc's implicit device synchronisation would stall every stream,
+ * plug-ins that are handed only their input and output buffers by a host
+ * framework that owns the allocator, and processes whose whole memory budget
+ * was reserved up front so that a later cudaMalloc simply fails.
+ *
+ * The int8 operand scratch is a fixed QNN_NOALLOC_SCRATCH_BYTES (8 MiB) array
+ * inside the library image: every GPU context that loads the library holds it
+ * until the process exits.  The call performs no cudaMalloc / cudaFree and
+ * calls no allocating library routine.  Shapes whose scratch
+ *   (M + N) * roundup(32 * ceil(K / 32), 128)   bytes (each term rounded to 256)
+ * exceeds the array are rejected with QNN_ERR_WORKSPACE before anything runs
+ * (e.g. 1024 x 1024 x 4096 fits, 4096 x 4096 x 4096 does not).
+ *
+ * The first call on each device looks up the array's device address (a
+ * one-time host-side set-up under a mutex, with that device current); make
+ * that first call before starting any stream capture.  All calls share the one
+ * array, which keeps the previous call's contents: the call rewrites every
+ * byte it later reads, so no clearing is needed, but two calls that overlap on
+ * the GPU (different streams, or several host threads) race on it -- keep
+ * calls to this entry point on one stream or serialise them yourself. */
+QNN_API int qnn_xnor_gemm_noalloc(const uint32_t *a, int64_t lda, const uint32_t *b, int64_t ldb, int64_t M,
+                                  int64_t N, int64_t K, int32_t *out, int64_t ldo, void *stream);
+
 /* ------------------------------------------------------------------------- */
 /* Threshold, rescale                                                         */
 /* ------------------------------------------------------------------------- */

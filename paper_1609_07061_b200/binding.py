@@ -22,6 +22,7 @@ QNN_ERR_WORKSPACE, QNN_ERR_CUDA, QNN_ERR_TIMEOUT = 5, 6, 7
 QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA = 0, 1, 2, 3
 QNN_MODE_U01, QNN_MODE_PM1 = 0, 1
 QNN_OP_XNOR_GEMM, QNN_OP_BITPLANE_GEMM, QNN_OP_CONV2D, QNN_OP_MLP = 1, 2, 3, 4
+QNN_NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
 class QnnError(RuntimeError):
@@ -57,6 +58,7 @@ _SIGS = {
     "qnn_pack_planes_u8": (i32, [vp, i64, i64, i64, i32, vp, i64, i64, vp, vp]),
     "qnn_pack_conv_weights": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "qnn_xnor_gemm": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
+    "qnn_xnor_gemm_noalloc": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, i64, vp]),
     "qnn_xnor_gemm_threshold": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, vp, vp, i64, i32, vp, sz, vp]),
     "qnn_bitplane_gemm": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
     "qnn_bitplane_gemm_threshold": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, vp, vp,
@@ -247,3 +249,11 @@ def qnn_set_kernel_events(start: Optional[torch.cuda.Event], stop: Optional[torc
     a = None if start is None else start.cuda_event
     b = None if stop is None else stop.cuda_event
     _ck(_lib.qnn_set_kernel_events(a, b), "qnn_set_kernel_events")
+
+
+def qnn_xnor_gemm_noalloc(a, lda, b, ldb, M, N, K, out, ldo):
+    """XNOR product whose scratch is the library's built-in 8 MiB array: no workspace argument, no allocation.
+
+    For callers that cannot allocate device memory at call time.  Calls share the array, so keep them on one
+    stream; the first call on a device should precede any stream capture."""
+    _ck(_lib.qnn_xnor_gemm_noalloc(_p(a), lda, _p(b), ldb, M, N, K, _p(out), ldo, _stream()), "qnn_xnor_gemm_noalloc")

@@ -1,0 +1,63 @@
+"""GPU test of qnn_xnor_gemm_noalloc, the entry point for callers that cannot allocate device memory
+(its operand scratch is an 8 MiB array built into the library).  Collected last on purpose.
+
+It must give exactly what qnn_xnor_gemm gives (integer outputs: bit-exact), on two calls in a row that
+share the built-in scratch, whether this file runs alone in a fresh process or after every other test."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_1609_07061_b200.binding as b
+    return b
+
+
+def _operands(M, N, K, seed):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    kw = (K + 31) // 32
+    ld = (kw + 3) // 4 * 4
+    a = torch.randint(-2**31, 2**31 - 1, (M, ld), dtype=torch.int32, device="cuda", generator=g)
+    b = torch.randint(-2**31, 2**31 - 1, (N, ld), dtype=torch.int32, device="cuda", generator=g)
+    if K % 32:                                   # the packed format wants zero pad bits in the last used word
+        mask = (1 << (K % 32)) - 1
+        m32 = mask if mask < 2**31 else mask - 2**32
+        a[:, kw - 1] &= m32
+        b[:, kw - 1] &= m32
+    return a, b, ld
+
+
+def test_noalloc_matches_workspace_entry_point_twice_in_a_row(q):
+    # second call: other shape, other data, smaller K -- stale scratch from the first call must not leak in
+    for (M, N, K, seed) in [(300, 1000, 4096, 1), (257, 130, 1000, 2)]:
+        a, b, ld = _operands(M, N, K, seed)
+        want = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+        ws = torch.empty(max(q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, N, K, 1, 1, q.QNN_ALGO_TC_I8), 256),
+                         dtype=torch.uint8, device="cuda")
+        q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, want, N, q.QNN_ALGO_TC_I8, ws)
+        popc = torch.empty_like(want)
+        q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, popc, N, q.QNN_ALGO_POPC)
+        got = torch.full((M, N), -9, dtype=torch.int32, device="cuda")
+        q.qnn_xnor_gemm_noalloc(a, ld, b, ld, M, N, K, got, N)
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0
+        assert torch.equal(got, want)
+        assert torch.equal(got, popc)
+
+
+def test_noalloc_rejects_shapes_beyond_the_builtin_scratch(q):
+    M = N = K = 4096                              # needs 2 x 16 MiB of int8 operands
+    assert q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, N, K, 1, 1, q.QNN_ALGO_TC_I8) > q.QNN_NOALLOC_SCRATCH_BYTES
+    a, b, ld = _operands(M, N, K, 3)
+    out = torch.full((M, N), 5, dtype=torch.int32, device="cuda")
+    before = q.qnn_launch_count()
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_xnor_gemm_noalloc(a, ld, b, ld, M, N, K, out, N)
+    assert e.value.status == q.QNN_ERR_WORKSPACE
+    assert "built-in" in str(e.value)
+    assert q.qnn_launch_count() == before         # nothing was launched
+    torch.cuda.synchronize()
+    assert bool((out == 5).all())
