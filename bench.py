@@ -170,9 +170,13 @@ class MlpBench:
                  q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, 4096, 4096, 1, 1, algo), 256)
         self.gws = torch.empty(gw, dtype=torch.uint8, device="cuda")
         self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        self.flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")
 
     def flush_l2(self):
+        """Writes a 256 MiB buffer (evicts every cached input), then reads another 256 MiB so that the dirty
+        lines of that write are written back BEFORE the timed region instead of inside it."""
         self.flush_buf.fill_(1)
+        self.flush_sink = self.flush_rd.sum()
 
     def step_calls(self, ev=None):
         """The Algorithm-4 pass as individual C-ABI calls; `ev` (optional) brackets the dominant product."""
@@ -464,9 +468,12 @@ def main():
         dom_ops = per_layer[1]
         achieved = dom_ops / (dom_ms / 1e3) / 1e12
         if resolved == q.QNN_ALGO_TC_I8:
-            # int8 tensor peak = measured bf16 peak x the nominal int8:bf16 ratio (2), sustained figure inside a step
-            bound, peak = "tensor", 2.0 * peaks["bf16_tflops_sustained"]
-            peak_note = f"2 x {peaks['source']} sustained bf16 ({peaks['bf16_tflops_sustained']} TF/s); one int8 MAC = one +-1 product"
+            # int8 tensor peak = measured bf16 peak x the nominal int8:bf16 ratio (2).  The kernel is bracketed by its
+            # own event pair inside a sub-millisecond step with idle gaps (L2 flush) around it, so it runs at burst
+            # clocks: the burst figure is the denominator (the sustained one would read above 1).
+            bound, peak = "tensor", 2.0 * peaks["bf16_tflops"]
+            peak_note = (f"2 x {peaks['source']} burst bf16 ({peaks['bf16_tflops']} TF/s; sustained "
+                         f"{peaks['bf16_tflops_sustained']}); one int8 MAC = one +-1 product")
             kernel = "tcgen05 kind::i8 xnor product 10000x4096x4096, threshold epilogue (gemm_i8_kernel)"
             dtype = "int8"
         else:
@@ -484,7 +491,7 @@ def main():
                                    "8-bit inputs as 8 bit-planes (K 784 padded to 800+), thresholds in [-64,64], seed 1",
                        "global_batch": BATCH * world, "parallelism": f"dp{world} (independent batch shards, no collective)",
                        "algo": {0: "auto", 1: "popc", 2: "tc_i8", 3: "b1_mma"}[resolved],
-                       "l2": "flushed between steps (256 MiB device fill, untimed)",
+                       "l2": "flushed between steps (256 MiB device fill, then a 256 MiB read so no dirty lines remain; untimed)",
                        "weights": "packed once at load (not in the step)"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * DIMS[0],
                     "d2h_bytes_per_step": BATCH * DIMS[-1] * 4, "ms_per_step": e2e_ms / args.steps,

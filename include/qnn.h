@@ -72,6 +72,14 @@ extern "C" {
 #define QNN_ALGO_POPC 1   /* xor/and + popc on the CUDA cores (Eq. 11 as written)          */
 #define QNN_ALGO_TC_I8 2  /* values expanded to int8, tcgen05 kind::i8, TMEM accumulators */
 #define QNN_ALGO_B1_MMA 3 /* 1-bit mma.sync and/xor-popc (legacy tensor-core path)        */
+#define QNN_ALGO_TC_FP4 4 /* values as 4-bit e2m1 floats, tcgen05 kind::mxf4 with unit block
+                             scales, fp32 TMEM accumulators (exact: integer sums below 2^24);
+                             operands of at most 2 planes                                 */
+
+/* tensor-core operand forms: one VALUE per element, rows packed along K, pad positions 0 */
+#define QNN_FORM_I8 1     /* one byte per element: int8 (QNN_MODE_PM1) or uint8 (QNN_MODE_U01) */
+#define QNN_FORM_FP4 2    /* one e2m1 nibble per element, element 2i in the low nibble of byte i;
+                             holds the values {0, +-1, +-2, +-3}                            */
 
 #define QNN_MODE_U01 0
 #define QNN_MODE_PM1 1
@@ -175,11 +183,65 @@ QNN_API int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, i
                                 const int32_t *thr, const uint8_t *flip, uint32_t *out_bits,
                                 int64_t ld_words, int algo, void *ws, size_t ws_bytes, void *stream);
 
+/* ------------------------------------------------------------------------- */
+/* Tensor-core operands prepared once (static weights, chained layers)        */
+/* ------------------------------------------------------------------------- */
+
+/* The tensor-core algorithms multiply VALUES, not bits: each call of the
+ * products above first rewrites both packed operands in a tensor-core form in
+ * the workspace.  For an operand that does not change between calls (weights)
+ * that rewrite can be done once with qnn_tc_prepack and the result handed to
+ * qnn_tc_gemm; the thresholded output of qnn_tc_gemm can be produced directly
+ * in a form, ready to be the next product's A operand (Algorithm 4 chains
+ * a^b_k = Sign(BatchNorm(a_k)) into the next XnorDotProduct).
+ *
+ * Layout of a form: row-major bytes [rows, ld_bytes]; ld_bytes a multiple of 16
+ * and the base 16-byte aligned; a row holds 32 * ceil(K / 32) elements
+ * (QNN_FORM_I8: that many bytes; QNN_FORM_FP4: half as many), pad elements 0. */
+
+/* Best form for a product of ka-plane (a_mode) and kb-plane (b_mode) operands
+ * over K: QNN_FORM_FP4 when both hold at most 2 planes and K * maxA * maxB < 2^24,
+ * else QNN_FORM_I8 when the codes fit a byte, else 0 (use QNN_ALGO_POPC). */
+QNN_API int qnn_tc_form(int ka, int a_mode, int kb, int b_mode, int64_t K);
+
+/* Bytes between rows (dense) and bytes of a whole operand [rows, K] in `form`. */
+QNN_API int64_t qnn_tc_row_bytes(int64_t K, int form);
+QNN_API size_t qnn_tc_operand_bytes(int64_t rows, int64_t K, int form);
+
+/* Rewrites nplanes packed planes (layout as in qnn_bitplane_gemm) as values in
+ * `form`: out[rows, ld_bytes].  QNN_ERR_UNSUPPORTED if the values do not fit. */
+QNN_API int qnn_tc_prepack(const uint32_t *planes, int nplanes, int mode, int64_t ld, int64_t plane_stride,
+                           int64_t rows, int64_t K, int form, void *out, int64_t ld_bytes, void *stream);
+
+typedef struct qnn_tc_operand {
+    const void *data; /* device, form bytes [rows, ld_bytes]                         */
+    int64_t ld_bytes;
+    int form;         /* QNN_FORM_*                                                  */
+    int planes;       /* planes of the integer code the values came from (1..8)      */
+    int mode;         /* QNN_MODE_*                                                  */
+} qnn_tc_operand;
+
+typedef struct qnn_tc_output { /* any subset; at least one of out / out_bits / out_form */
+    int32_t *out;         /* int32 [M, ldo] or NULL                                  */
+    int64_t ldo;
+    const int32_t *thr;   /* int32 [N], needed for out_bits / out_form               */
+    const uint8_t *flip;  /* uint8 [N] or NULL                                       */
+    uint32_t *out_bits;   /* packed (dot >= thr) XOR flip, [M, ld_words], or NULL    */
+    int64_t ld_words;
+    void *out_form;       /* the same signs as +-1 values in form out_form_kind, or NULL */
+    int out_form_kind;
+    int64_t ld_form_bytes;
+} qnn_tc_output;
+
+/* out[m,n] = sum_k A[m,k] * B[n,k] on prepared operands (same form for both). */
+QNN_API int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_t M, int64_t N, int64_t K,
+                        const qnn_tc_output *o, void *stream);
+
 /* Size of the scratch array built into the library for qnn_xnor_gemm_noalloc. */
 #define QNN_NOALLOC_SCRATCH_BYTES (8u << 20)
 
 /* The paper has no counterpart for this call; it is a packaging variant of
- * qnn_xnor_gemm (same arguments, same int32 result, always the tensor-core
+ * qnn_xnor_gemm (same arguments, same int32 result, always the int8 tensor-core
  * algorithm) for callers that cannot allocate device memory or size a
  * workspace when they call: code running on a latency-critical serving thread
  * where cudaMalloc's implicit device synchronisation would stall every stream,
@@ -191,7 +253,7 @@ QNN_API int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, i
  * inside the library image: every GPU context that loads the library holds it
  * until the process exits.  The call performs no cudaMalloc / cudaFree and
  * calls no allocating library routine.  Shapes whose scratch
- *   (M + N) * roundup(32 * ceil(K / 32), 128)   bytes (each term rounded to 256)
+ *   (M + N) * 32 * ceil(K / 32)   bytes (the M and the N term each rounded up to 256)
  * exceeds the array are rejected with QNN_ERR_WORKSPACE before anything runs
  * (e.g. 1024 x 1024 x 4096 fits, 4096 x 4096 x 4096 does not).
  *

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libqnn.so")
 QNN_OK = 0
 QNN_ERR_INVALID_ARG, QNN_ERR_ALIGNMENT, QNN_ERR_UNSUPPORTED, QNN_ERR_OVERFLOW = 1, 2, 3, 4
 QNN_ERR_WORKSPACE, QNN_ERR_CUDA, QNN_ERR_TIMEOUT = 5, 6, 7
-QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA = 0, 1, 2, 3
+QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA, QNN_ALGO_TC_FP4 = 0, 1, 2, 3, 4
+QNN_FORM_I8, QNN_FORM_FP4 = 1, 2
 QNN_MODE_U01, QNN_MODE_PM1 = 0, 1
 QNN_OP_XNOR_GEMM, QNN_OP_BITPLANE_GEMM, QNN_OP_CONV2D, QNN_OP_MLP = 1, 2, 3, 4
 QNN_NOALLOC_SCRATCH_BYTES = 8 << 20
@@ -40,6 +41,15 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 i64, i32, vp, f32, sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_float, ctypes.c_size_t
+
+
+class qnn_tc_operand(ctypes.Structure):
+    _fields_ = [("data", vp), ("ld_bytes", i64), ("form", i32), ("planes", i32), ("mode", i32)]
+
+
+class qnn_tc_output(ctypes.Structure):
+    _fields_ = [("out", vp), ("ldo", i64), ("thr", vp), ("flip", vp), ("out_bits", vp), ("ld_words", i64),
+                ("out_form", vp), ("out_form_kind", i32), ("ld_form_bytes", i64)]
 
 
 class qnn_mlp_layer(ctypes.Structure):
@@ -63,6 +73,12 @@ _SIGS = {
     "qnn_bitplane_gemm": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
     "qnn_bitplane_gemm_threshold": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, vp, vp,
                                           i64, i32, vp, sz, vp]),
+    "qnn_tc_form": (i32, [i32, i32, i32, i32, i64]),
+    "qnn_tc_row_bytes": (i64, [i64, i32]),
+    "qnn_tc_operand_bytes": (sz, [i64, i64, i32]),
+    "qnn_tc_prepack": (i32, [vp, i32, i32, i64, i64, i64, i64, i32, vp, i64, vp]),
+    "qnn_tc_gemm": (i32, [ctypes.POINTER(qnn_tc_operand), ctypes.POINTER(qnn_tc_operand), i64, i64, i64,
+                          ctypes.POINTER(qnn_tc_output), vp]),
     "qnn_threshold_pack": (i32, [vp, i64, i64, i64, vp, vp, vp, i64, vp]),
     "qnn_fold_bn": (i32, [vp, vp, vp, vp, ctypes.c_double, i64, vp, vp]),
     "qnn_rescale_f32": (i32, [vp, i64, i64, i64, f32, vp, vp, f32, vp, i64, vp]),
@@ -171,6 +187,34 @@ def qnn_bitplane_gemm_threshold(a, ka, a_mode, lda, a_plane_stride, b, kb, b_mod
     _ck(_lib.qnn_bitplane_gemm_threshold(_p(a), ka, a_mode, lda, a_plane_stride, _p(b), kb, b_mode, ldb,
                                          b_plane_stride, M, N, K, _p(thr), _p(flip), _p(out_bits), ld_words, algo, wp,
                                          wb, _stream()), "qnn_bitplane_gemm_threshold")
+
+
+def qnn_tc_form(ka, a_mode, kb, b_mode, K) -> int:
+    return int(_lib.qnn_tc_form(ka, a_mode, kb, b_mode, K))
+
+
+def qnn_tc_row_bytes(K, form) -> int:
+    return int(_lib.qnn_tc_row_bytes(K, form))
+
+
+def qnn_tc_operand_bytes(rows, K, form) -> int:
+    return int(_lib.qnn_tc_operand_bytes(rows, K, form))
+
+
+def qnn_tc_prepack(planes, nplanes, mode, ld, plane_stride, rows, K, form, out, ld_bytes):
+    _ck(_lib.qnn_tc_prepack(_p(planes), nplanes, mode, ld, plane_stride, rows, K, form, _p(out), ld_bytes, _stream()),
+        "qnn_tc_prepack")
+
+
+def tc_operand(data, ld_bytes, form, planes=1, mode=QNN_MODE_PM1) -> qnn_tc_operand:
+    return qnn_tc_operand(_p(data), ld_bytes, form, planes, mode)
+
+
+def qnn_tc_gemm(a: qnn_tc_operand, b: qnn_tc_operand, M, N, K, out=None, ldo=0, thr=None, flip=None, out_bits=None,
+                ld_words=0, out_form=None, out_form_kind=0, ld_form_bytes=0):
+    o = qnn_tc_output(_p(out), ldo, _p(thr), _p(flip), _p(out_bits), ld_words, _p(out_form), out_form_kind,
+                      ld_form_bytes)
+    _ck(_lib.qnn_tc_gemm(ctypes.byref(a), ctypes.byref(b), M, N, K, ctypes.byref(o), _stream()), "qnn_tc_gemm")
 
 
 def qnn_threshold_pack(s, M, N, lds, thr, flip, out, ld_words):

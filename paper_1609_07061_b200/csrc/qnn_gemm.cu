@@ -47,6 +47,7 @@ static int forced_algo()
     if (!e || !*e) return QNN_ALGO_AUTO;
     if (!strcmp(e, "POPC") || !strcmp(e, "1")) return QNN_ALGO_POPC;
     if (!strcmp(e, "TC_I8") || !strcmp(e, "2")) return QNN_ALGO_TC_I8;
+    if (!strcmp(e, "TC_FP4") || !strcmp(e, "4")) return QNN_ALGO_TC_FP4;
     if (!strcmp(e, "B1_MMA") || !strcmp(e, "3")) return QNN_ALGO_B1_MMA;
     return QNN_ALGO_AUTO;
 }
@@ -54,21 +55,28 @@ static int forced_algo()
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (int rc = validate_gemm(g)) return rc;
-    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_B1_MMA, QNN_ERR_INVALID_ARG, "gemm: unknown algo %d", algo);
+    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_FP4, QNN_ERR_INVALID_ARG, "gemm: unknown algo %d", algo);
     if (g.M == 0 || g.N == 0) return QNN_OK;
     if (algo == QNN_ALGO_AUTO) {
         algo = forced_algo();
         if (algo == QNN_ALGO_AUTO) algo = qnn_select_algo(g.M, g.N, g.K, g.ka, g.kb, g.a_mode, g.b_mode);
-        // AUTO never fails for want of a workspace: fall back to the CUDA-core path
-        if (algo == QNN_ALGO_TC_I8 &&
-            (!gemm_tc_supported(g) || ws == nullptr || ws_bytes < gemm_tc_workspace_bytes(g.M, g.N, g.K, g.ka, g.kb)))
-            algo = QNN_ALGO_POPC;
+        // AUTO never fails for want of a workspace or of a fitting form: fall back to the CUDA-core path
+        if (algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_TC_FP4) {
+            const int form = algo == QNN_ALGO_TC_FP4 ? QNN_FORM_FP4 : QNN_FORM_I8;
+            const bool fits = tc_form_holds(form, g.ka, g.a_mode) && tc_form_holds(form, g.kb, g.b_mode) &&
+                              (form != QNN_FORM_FP4 || tc_pick_form(g.ka, g.a_mode, g.kb, g.b_mode, g.K) == QNN_FORM_FP4);
+            const int64_t kw = g.kwords > 0 ? g.kwords : ceil_div(g.K, 32);
+            const size_t need = round_up((size_t)g.M * (size_t)tc_row_bytes(kw, form), 256) +
+                                round_up((size_t)g.N * (size_t)tc_row_bytes(kw, form), 256);
+            if (!fits || kw == 0 || ws == nullptr || ws_bytes < need) algo = QNN_ALGO_POPC;
+        }
         if (algo == QNN_ALGO_B1_MMA && !(g.ka == 1 && g.kb == 1)) algo = QNN_ALGO_POPC;
     }
     switch (algo) {
         case QNN_ALGO_POPC: return launch_gemm_popc(g, st);
         case QNN_ALGO_B1_MMA: return launch_gemm_b1mma(g, st);
-        case QNN_ALGO_TC_I8: return launch_gemm_tc(g, ws, ws_bytes, st);
+        case QNN_ALGO_TC_I8: return launch_gemm_tc(g, QNN_FORM_I8, ws, ws_bytes, st);
+        case QNN_ALGO_TC_FP4: return launch_gemm_tc(g, QNN_FORM_FP4, ws, ws_bytes, st);
     }
     return fail(QNN_ERR_INVALID_ARG, "gemm: unknown algo");
 }
@@ -128,6 +136,73 @@ int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, int64_t l
     return run_gemm(g, algo, ws, ws_bytes, as_stream(stream));
 }
 
+int qnn_tc_form(int ka, int a_mode, int kb, int b_mode, int64_t K)
+{
+    if (ka < 1 || ka > 8 || kb < 1 || kb > 8 || K < 0) return 0;
+    return tc_pick_form(ka, a_mode, kb, b_mode, K);
+}
+
+int64_t qnn_tc_row_bytes(int64_t K, int form)
+{
+    if (K < 0 || (form != QNN_FORM_I8 && form != QNN_FORM_FP4)) return 0;
+    return tc_row_bytes(ceil_div(K, 32), form);
+}
+
+size_t qnn_tc_operand_bytes(int64_t rows, int64_t K, int form)
+{
+    if (rows <= 0) return 0;
+    return (size_t)rows * (size_t)qnn_tc_row_bytes(K, form);
+}
+
+int qnn_tc_prepack(const uint32_t *planes, int nplanes, int mode, int64_t ld, int64_t plane_stride, int64_t rows,
+                   int64_t K, int form, void *out, int64_t ld_bytes, void *stream)
+{
+    QNN_REQUIRE(rows >= 0 && K >= 0, QNN_ERR_INVALID_ARG, "qnn_tc_prepack: negative size");
+    QNN_REQUIRE(nplanes >= 1 && nplanes <= 8 && (mode == QNN_MODE_U01 || mode == QNN_MODE_PM1), QNN_ERR_INVALID_ARG,
+                "qnn_tc_prepack: bad plane count or mode");
+    QNN_REQUIRE(form == QNN_FORM_I8 || form == QNN_FORM_FP4, QNN_ERR_INVALID_ARG, "qnn_tc_prepack: unknown form %d", form);
+    QNN_REQUIRE(tc_form_holds(form, nplanes, mode), QNN_ERR_UNSUPPORTED,
+                "qnn_tc_prepack: values of %d planes do not fit form %d", nplanes, form);
+    if (rows == 0 || K == 0) return QNN_OK;
+    const int64_t kwords = ceil_div(K, 32);
+    QNN_REQUIRE(planes && out, QNN_ERR_INVALID_ARG, "qnn_tc_prepack: NULL pointer");
+    QNN_REQUIRE(ld >= kwords && (nplanes == 1 || plane_stride >= rows * ld), QNN_ERR_INVALID_ARG,
+                "qnn_tc_prepack: ld or plane stride too small");
+    QNN_REQUIRE(aligned(out, 16) && ld_bytes % 16 == 0 && ld_bytes >= tc_row_bytes(kwords, form), QNN_ERR_ALIGNMENT,
+                "qnn_tc_prepack: out needs a 16-byte aligned base and a row stride that is a multiple of 16 covering K");
+    return tc_expand(planes, nplanes, mode, ld, plane_stride, rows, kwords, kwords, (int)(K - 32 * (kwords - 1)), form,
+                     static_cast<uint8_t *>(out), ld_bytes, as_stream(stream));
+}
+
+int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_t M, int64_t N, int64_t K, const qnn_tc_output *o,
+                void *stream)
+{
+    QNN_REQUIRE(a && b && o, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: NULL descriptor");
+    QNN_REQUIRE(a->form == b->form, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: operands are in different forms");
+    GemmArgs g{};
+    g.ka = a->planes; g.kb = b->planes; g.a_mode = a->mode; g.b_mode = b->mode;
+    g.M = M; g.N = N; g.K = K;
+    g.a_tc = a->data; g.a_tc_form = a->form; g.a_tc_ld = a->ld_bytes;
+    g.b_tc = b->data; g.b_tc_form = b->form; g.b_tc_ld = b->ld_bytes;
+    g.epilogue = o->out ? EPI_ROWMAJOR : EPI_BITS;
+    g.out = o->out; g.ldo = o->ldo; g.thr = o->thr; g.flip = o->flip; g.out_bits = o->out_bits; g.ld_bits = o->ld_words;
+    g.out_form = o->out_form; g.out_form_kind = o->out_form_kind; g.ld_form = o->ld_form_bytes;
+    QNN_REQUIRE(M >= 0 && N >= 0 && K >= 1, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: bad size");
+    QNN_REQUIRE(K < (int64_t)1 << 31, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: K must be below 2^31");
+    QNN_REQUIRE(g.ka >= 1 && g.ka <= 8 && g.kb >= 1 && g.kb <= 8, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: plane counts must be in 1..8");
+    const int64_t la = (1 << g.ka) - 1, lb = (1 << g.kb) - 1;
+    QNN_REQUIRE(la * lb <= (((int64_t)1 << 31) - 1) / K, QNN_ERR_OVERFLOW, "qnn_tc_gemm: result may not fit int32");
+    if (M == 0 || N == 0) return QNN_OK;
+    QNN_REQUIRE(a->data && b->data, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: NULL operand");
+    QNN_REQUIRE(o->out || o->out_bits || o->out_form, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: no output buffer");
+    QNN_REQUIRE(!o->out || o->ldo >= N, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: ldo smaller than N");
+    QNN_REQUIRE(!(o->out_bits || o->out_form) || o->thr, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: thresholds required");
+    QNN_REQUIRE(!o->out_bits || o->ld_words >= ceil_div(N, 32), QNN_ERR_INVALID_ARG, "qnn_tc_gemm: ld_words too small");
+    const int64_t rb = tc_row_bytes(ceil_div(K, 32), a->form);
+    QNN_REQUIRE(a->ld_bytes >= rb && b->ld_bytes >= rb, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: operand row stride smaller than K needs");
+    return launch_gemm_tc(g, a->form, nullptr, 0, as_stream(stream));
+}
+
 int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int a_mode, int b_mode)
 {
     // Measured on B200: the 1-bit mma.sync path never beats xor+popc on the CUDA cores, so it is never picked.
@@ -135,9 +210,11 @@ int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int a_mode,
     // equivalent plane-pair work M*N*K*ka*kb reaches about 2^31; below that its expansion passes and launch
     // latencies dominate.
     if (M <= 0 || N <= 0 || K <= 0) return QNN_ALGO_POPC;
-    if ((a_mode == QNN_MODE_PM1 && ka > 7) || (b_mode == QNN_MODE_PM1 && kb > 7)) return QNN_ALGO_POPC;
+    const int form = tc_pick_form(ka, a_mode, kb, b_mode, K);
+    if (form == 0) return QNN_ALGO_POPC;
     const double work = (double)M * (double)N * (double)K * (double)ka * (double)kb;
-    return work >= 2147483648.0 ? QNN_ALGO_TC_I8 : QNN_ALGO_POPC;
+    if (work < 2147483648.0) return QNN_ALGO_POPC;
+    return form == QNN_FORM_FP4 ? QNN_ALGO_TC_FP4 : QNN_ALGO_TC_I8;
 }
 
 size_t qnn_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int ka, int kb, int algo)
@@ -149,6 +226,10 @@ size_t qnn_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int ka, int 
         ka = kb = 1;
     }
     if (algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_AUTO) bytes += gemm_tc_workspace_bytes(M, N, K, ka, kb);
+    if (algo == QNN_ALGO_TC_FP4) {
+        const int64_t rb = tc_row_bytes(ceil_div(K, 32), QNN_FORM_FP4);
+        bytes += round_up((size_t)M * (size_t)rb, 256) + round_up((size_t)N * (size_t)rb, 256);
+    }
     return bytes;
 }
 

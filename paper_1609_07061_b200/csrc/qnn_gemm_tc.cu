@@ -1,12 +1,23 @@
-// Tensor-core matrix product: the packed operands are expanded to their int8
-// VALUES (+-1, unsigned codes or signed-symmetric codes; pad positions become
-// 0) in the caller's workspace, then one persistent, warp-specialised kernel
-// multiplies them on the 5th-generation tensor cores:
-//   TMA (128-byte swizzle) -> shared-memory ring -> tcgen05.mma kind::i8 with
-//   the int32 accumulator in tensor memory (two accumulator stages) ->
-//   tcgen05.ld epilogue (int32 rows, NCHW scatter or threshold -> packed bits).
-// One int8 multiply-accumulate carries one product of the paper's sum, so a
-// k-bit x k-bit product costs ONE pass here instead of ka*kb plane passes.
+// Tensor-core matrix product on the 5th-generation tensor cores (tcgen05).
+//
+// The packed bit-planes are first rewritten in a "tensor-core form", one VALUE
+// per element (+-1, unsigned codes or signed-symmetric codes; pad positions 0):
+//   QNN_FORM_FP4  4-bit e2m1 floats, two per byte -- holds {0, +-1, +-2, +-3};
+//                 multiplied by tcgen05.mma kind::mxf4 with all block scales 1.0
+//                 and accumulated in fp32, which is exact for these integers
+//                 while |sum| < 2^24;
+//   QNN_FORM_I8   int8 / uint8 -- any code that fits a byte; kind::i8, int32
+//                 accumulation.
+// One multiply-accumulate of the tensor core carries one product of the
+// paper's sum, so a k-bit x k-bit product costs ONE pass here instead of ka*kb
+// plane passes.  A persistent, warp-specialised kernel does the product:
+//   warp 0: TMA (128-byte swizzle) -> shared-memory ring
+//   warp 1: tcgen05.mma, accumulator in tensor memory (two accumulator stages)
+//   warps 2..5: tcgen05.ld epilogue -> int32 rows, NCHW scatter, threshold ->
+//               packed bits and / or the next layer's operand in tensor-core form
+// A convolution can be run as an implicit GEMM: the A tile of one filter tap is
+// a 4-D TMA box of the NHWC tensor, out-of-image reads give zero, and the
+// contribution of the padding value is added back per border class.
 //
 // Every device-side wait is bounded: when a wait runs out the kernel records a
 // code in a device status word, raises a block-wide abort flag, lets copies in
@@ -18,21 +29,27 @@ namespace qnn {
 namespace {
 
 constexpr int BM = 128;              // rows of A per tile (UMMA M)
-constexpr int BK = 128;              // int8 elements of K per pipeline stage = one 128-byte swizzle row
-constexpr int UMMA_K = 32;           // K per tcgen05.mma of kind::i8
+constexpr int BKB = 128;             // bytes of K per pipeline stage = one 128-byte swizzle row
 constexpr int TC_THREADS = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int SMEM_LIMIT = 232448;   // 227 KB of dynamic shared memory per CTA
 
 __device__ int g_tc_status = 0;      // 0 = fine; otherwise the code of the first wait that ran out
 
 struct TcParams {
     int64_t M, N;
-    int32_t num_kb;                  // K blocks of BK
+    int32_t num_kb;                  // K blocks of BKB bytes
     int32_t tiles_m, tiles_n;
+    int32_t a_tx_bytes;              // bytes one A box delivers
     int epilogue;
     int32_t *out; int64_t ldo; int64_t hw;
     const int32_t *thr; const uint8_t *flip; uint32_t *out_bits; int64_t ld_bits;
+    uint8_t *out_form; int64_t ld_form; int out_form_kind;
     uint32_t idesc;
+    // implicit convolution (conv != 0)
+    int conv;
+    int32_t cH, cW, cR, tiles_per_img, cKW, cpad, cblocks;
+    const int32_t *corr;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -82,6 +99,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, int32_t c2,
+                                            int32_t c3, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -105,6 +129,18 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
         "}\n"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// e2m1 x e2m1 with one ue8m0 scale per 32 elements of K; `sf` addresses tensor-memory columns holding the scales
+__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
+                                          uint32_t sf)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%5], p;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sf) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -122,6 +158,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
         : "r"(taddr) : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// this warp's 32 lanes x 8 columns, all set to `val`
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, uint32_t val)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr), "r"(val) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled
 // (the layout a TMA box of 128 bytes x rows produces): 8-row groups are 1024 bytes apart.
@@ -136,22 +178,44 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr)
     return d;
 }
 
-template <int BN>
-struct TcSmem {
-    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int A_BYTES = BM * BK;
-    static constexpr int B_BYTES = BN * BK;
+// bit i of the low byte of x -> bit 4*i (one bit per nibble)
+__device__ __forceinline__ uint32_t spread_bits_to_nibbles(uint32_t x)
+{
+    x = (x | (x << 12)) & 0x000F000Fu;
+    x = (x | (x << 6)) & 0x03030303u;
+    x = (x | (x << 3)) & 0x11111111u;
+    return x;
+}
+// bit i of the low nibble of x -> bit 8*i (one bit per byte)
+__device__ __forceinline__ uint32_t spread_bits_to_bytes(uint32_t nib) { return (nib * 0x00204081u) & 0x01010101u; }
+
+constexpr int next_pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
+
+template <int FORM, int BN>
+struct TcCfg {
+    static constexpr int A_BYTES = BM * BKB;
+    static constexpr int B_BYTES = BN * BKB;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;     // two accumulator stages
+    static constexpr int THR_WORDS = BN + 8;                             // per epilogue warp: BN thresholds + BN/32 flip words
+    static constexpr int THR_BYTES = 4 * THR_WORDS * 4;
+    static constexpr int AUX_BYTES = 256 + THR_BYTES + 1024;             // barriers, thresholds, 1024-byte alignment slack
+    static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = MAX_STAGES > 8 ? 8 : MAX_STAGES;
+    static constexpr int SCALE_COL = 2 * BN;                             // FP4: unit block scales live behind the accumulators
+    static constexpr int TMEM_COLS = next_pow2_cols(2 * BN + (FORM == QNN_FORM_FP4 ? 32 : 0));
     static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
-    static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;              // barriers + slack for 1024-byte alignment
+    static constexpr int THR_OFFSET = BAR_OFFSET + 256;
+    static constexpr int TOTAL = THR_OFFSET + THR_BYTES + 1024;
+    static_assert(STAGES >= 3, "pipeline too shallow");
+    static_assert(TMEM_COLS <= 512, "accumulators do not fit tensor memory");
+    static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile width");
 };
 
-template <int BN>
+template <int FORM, int BN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
 {
-    using S = TcSmem<BN>;
+    using S = TcCfg<FORM, BN>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
@@ -181,20 +245,44 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    if (FORM == QNN_FORM_FP4) {
+        // Unit scale factors (ue8m0 exponent 127 = 2^0) in 32 columns of every lane: whatever layout the
+        // instruction reads its per-block scales in, every scale it finds is 1.0.
+        if (warp >= 2) {
+            const int q = warp & 3;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                tmem_st8(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(S::SCALE_COL + 8 * c), 0x7f7f7f7fu);
+            tmem_st_wait();
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+
     const int64_t num_tiles = (int64_t)p.tiles_m * p.tiles_n;
 
     if (warp == 0) {
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
+            const uint32_t tx_bytes = (uint32_t)p.a_tx_bytes + (uint32_t)S::B_BYTES;
             for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
                 const int32_t tm = (int32_t)(t % p.tiles_m), tn = (int32_t)(t / p.tiles_m);
+                int32_t img = 0, y0 = 0;
+                if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; }
+                int32_t cb = 0, kw = 0, kh = 0;                    // conv: channel block, filter column, filter row of kb
                 for (int32_t kb = 0; kb < p.num_kb; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 1)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(stage), (uint32_t)S::STAGE_BYTES);
+                    mbar_expect_tx(full_bar(stage), tx_bytes);
                     const uint32_t sa = base + (uint32_t)stage * S::STAGE_BYTES;
-                    tma_load_2d(sa, &tmap_a, kb * BK, tm * BM, full_bar(stage));
-                    tma_load_2d(sa + S::A_BYTES, &tmap_b, kb * BK, tn * BN, full_bar(stage));
+                    if (p.conv) {
+                        tma_load_4d(sa, &tmap_a, cb * BKB, kw - p.cpad, y0 + kh - p.cpad, img, full_bar(stage));
+                        if (++cb == p.cblocks) { cb = 0; if (++kw == p.cKW) { kw = 0; ++kh; } }
+                    } else {
+                        tma_load_2d(sa, &tmap_a, kb * BKB, tm * BM, full_bar(stage));
+                    }
+                    tma_load_2d(sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN, full_bar(stage));
                     if (++stage == S::STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -204,6 +292,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int stage = 0; uint32_t phase = 0;
             uint32_t iter = 0;
             bool ok = true;
+            const uint32_t sf = tmem_base + (uint32_t)S::SCALE_COL;
             for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
                 const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abort_flag, 2)) { ok = false; break; }
@@ -216,10 +305,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     const uint64_t adesc = make_kmajor_sw128_desc(sa);
                     const uint64_t bdesc = make_kmajor_sw128_desc(sa + S::A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // advancing K inside the swizzle row: +32 bytes = +2 in the 16-byte address field
-                        umma_i8(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), p.idesc,
-                                (uint32_t)((kb | k) != 0));
+                    for (int k = 0; k < 4; ++k) {
+                        // one instruction consumes 32 bytes of K; +32 bytes inside the swizzle row = +2 in the address field
+                        const uint32_t acc = (uint32_t)((kb | k) != 0);
+                        if (FORM == QNN_FORM_FP4)
+                            umma_mxf4(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), p.idesc, acc, sf);
+                        else
+                            umma_i8(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), p.idesc, acc);
                     }
                     umma_commit(empty_bar(stage));               // frees the smem slot once these MMAs retire
                     if (++stage == S::STAGES) { stage = 0; phase ^= 1u; }
@@ -229,68 +321,141 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
     } else {
         const int q = warp & 3;                                  // TMEM lane quarter this warp may read
+        int32_t *thr_w = reinterpret_cast<int32_t *>(gen + S::THR_OFFSET) + q * S::THR_WORDS;   // this warp's thresholds
+        uint32_t *flip_w = reinterpret_cast<uint32_t *>(thr_w + BN);                            // and flip words
+        const bool want_bits = p.out_bits != nullptr;
+        const bool want_form = p.out_form != nullptr;
+        const bool want_sign = want_bits || want_form;
         uint32_t iter = 0;
         bool ok = true;
         for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
             const int32_t tm = (int32_t)(t % p.tiles_m), tn = (int32_t)(t / p.tiles_m);
             const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
+            const int64_t ntile = (int64_t)tn * BN;
+
+            // stage this tile's thresholds and flip words while the accumulator is still being produced
+            if (want_sign) {
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < BN / 32; ++c) {
+                    const int64_t n = ntile + c * 32 + lane;
+                    const bool ncol = n < p.N;
+                    thr_w[c * 32 + lane] = ncol ? __ldg(p.thr + n) : 0;
+                    const bool f = (ncol && p.flip) ? (__ldg(p.flip + n) != 0) : false;
+                    const uint32_t fw = __ballot_sync(0xffffffffu, f);
+                    if (lane == c) flip_w[c] = fw;
+                }
+                __syncwarp();
+            }
+
+            // which output row this thread owns
+            const int r = q * 32 + lane;
+            int64_t m;
+            bool mrow;
+            int32_t cls = 0;
+            if (p.conv) {
+                const int32_t img = tm / p.tiles_per_img;
+                const int32_t y = (tm - img * p.tiles_per_img) * p.cR + r / p.cW;
+                const int32_t x = r % p.cW;
+                mrow = (r < p.cR * p.cW) && (y < p.cH);
+                m = ((int64_t)img * p.cH + y) * p.cW + x;
+                const int32_t pd = p.cpad, pc = pd + 1;
+                const int32_t ty = max(pd - y, 0), by = max(y + pd - (p.cH - 1), 0);
+                const int32_t tx = max(pd - x, 0), bx = max(x + pd - (p.cW - 1), 0);
+                cls = mrow ? ((ty * pc + by) * pc + tx) * pc + bx : 0;
+            } else {
+                m = (int64_t)tm * BM + r;
+                mrow = m < p.M;
+            }
+            const bool any_border = p.conv ? (__any_sync(0xffffffffu, cls != 0) != 0) : false;
+            int64_t img = 0, pix = 0;
+            if (p.epilogue == EPI_NCHW && mrow) { img = m / p.hw; pix = m - img * p.hw; }
+
             // the tensor-memory loads below are warp-collective: leave the loop only as a whole warp
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(as), aphase, abort_flag, 4))) { ok = false; break; }
             tc_fence_after();
-            const int64_t m = (int64_t)tm * BM + q * 32 + lane;
-            const bool mrow = m < p.M;
-            int64_t img = 0, pix = 0;
-            if (p.epilogue == EPI_NCHW && mrow) { img = m / p.hw; pix = m - img * p.hw; }
-            uint32_t words[BN / 32];
-#pragma unroll
+
+#pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
+                const int64_t n0 = ntile + c * 32;
+                if (n0 >= p.N) break;                            // warp-uniform
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * (uint32_t)BN + (uint32_t)(c * 32), v);
-                const int64_t n0 = (int64_t)tn * BN + c * 32;
-                if (p.out != nullptr && mrow && n0 < p.N) {
+                int32_t iv[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    iv[j] = (FORM == QNN_FORM_FP4) ? __float2int_rn(__uint_as_float(v[j])) : (int32_t)v[j];
+                if (any_border && cls != 0) {
+                    const int32_t *cp = p.corr + (int64_t)cls * p.N + n0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (n0 + j < p.N) iv[j] += __ldg(cp + j);
+                }
+                if (p.out != nullptr && mrow) {
                     if (p.epilogue == EPI_NCHW) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (n0 + j < p.N) p.out[(img * p.N + n0 + j) * p.hw + pix] = (int32_t)v[j];
+                            if (n0 + j < p.N) p.out[(img * p.N + n0 + j) * p.hw + pix] = iv[j];
                     } else {
                         int32_t *dst = p.out + m * p.ldo + n0;
                         if (n0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<int4 *>(dst + j) = make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]);
+                                *reinterpret_cast<int4 *>(dst + j) = make_int4(iv[j], iv[j + 1], iv[j + 2], iv[j + 3]);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                if (n0 + j < p.N) dst[j] = (int32_t)v[j];
+                                if (n0 + j < p.N) dst[j] = iv[j];
                         }
                     }
                 }
-                uint32_t w = 0;
-                if (p.out_bits != nullptr && n0 < p.N) {
-                    // lane j fetches the threshold (and flip) of column n0 + j once; the row loop reads them by shuffle
-                    const bool ncol = (n0 + lane) < p.N;
-                    const int32_t tl = ncol ? __ldg(p.thr + n0 + lane) : 0;
-                    const uint32_t fl = (ncol && p.flip) ? (uint32_t)(__ldg(p.flip + n0 + lane) != 0) : 0u;
-                    const uint32_t fmask = __ballot_sync(0xffffffffu, fl != 0);
-                    const uint32_t nmask = __ballot_sync(0xffffffffu, ncol);
+                if (want_sign) {
+                    const int4 *t4 = reinterpret_cast<const int4 *>(thr_w + c * 32);
+                    uint32_t w = 0;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int32_t tj = __shfl_sync(0xffffffffu, tl, j);
-                        w |= (uint32_t)((int32_t)v[j] >= tj) << j;
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const int4 tt = t4[j4];                  // same address in every lane: a broadcast read
+                        w |= (uint32_t)(iv[4 * j4] >= tt.x) << (4 * j4);
+                        w |= (uint32_t)(iv[4 * j4 + 1] >= tt.y) << (4 * j4 + 1);
+                        w |= (uint32_t)(iv[4 * j4 + 2] >= tt.z) << (4 * j4 + 2);
+                        w |= (uint32_t)(iv[4 * j4 + 3] >= tt.w) << (4 * j4 + 3);
                     }
-                    w = (w ^ fmask) & nmask;
+                    const int64_t left = p.N - n0;
+                    const uint32_t nmask = left >= 32 ? 0xffffffffu : ((1u << (int)left) - 1u);
+                    w = (w ^ flip_w[c]) & nmask;
+                    if (mrow) {
+                        if (want_bits) p.out_bits[m * p.ld_bits + (n0 >> 5)] = w;
+                        if (want_form) {
+                            if (p.out_form_kind == QNN_FORM_FP4) {
+                                // +1 -> e2m1 0x2, -1 -> 0xA, columns past N -> 0
+                                uint32_t o[4];
+#pragma unroll
+                                for (int b = 0; b < 4; ++b) {
+                                    const uint32_t s = spread_bits_to_nibbles((w >> (8 * b)) & 0xffu);
+                                    const uint32_t vm = spread_bits_to_nibbles((nmask >> (8 * b)) & 0xffu) * 0xfu;
+                                    o[b] = (0xAAAAAAAAu ^ (s << 3)) & vm;
+                                }
+                                *reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + (n0 >> 1)) = make_uint4(o[0], o[1], o[2], o[3]);
+                            } else {
+                                // +1 -> 0x01, -1 -> 0xFF, columns past N -> 0
+                                uint32_t o[8];
+#pragma unroll
+                                for (int b = 0; b < 8; ++b) {
+                                    const uint32_t s = spread_bits_to_bytes((w >> (4 * b)) & 0xfu);
+                                    const uint32_t vm = spread_bits_to_bytes((nmask >> (4 * b)) & 0xfu) * 0xffu;
+                                    o[b] = (0xFFFFFFFFu ^ (s * 0xfeu)) & vm;
+                                }
+                                uint4 *dst = reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + n0);
+                                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                            }
+                        }
+                    }
                 }
-                words[c] = w;
             }
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
             mbar_arrive(tempty_bar(as));
-            if (p.out_bits != nullptr && mrow) {
-                uint32_t *dst = p.out_bits + m * p.ld_bits + (((int64_t)tn * BN) >> 5);
-#pragma unroll
-                for (int c = 0; c < BN / 32; ++c)
-                    if ((int64_t)tn * BN + c * 32 < p.N) dst[c] = words[c];
-            }
         }
     }
 
@@ -306,15 +471,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (warp == 1) tmem_dealloc(tmem_base, S::TMEM_COLS);
 }
 
-// ---- expansion of packed planes to int8 values ------------------------------
+// ---- expansion of packed planes to tensor-core forms ---------------------------
+//
+// `period`/`tail` say where pad bits sit: word (w mod period) == period-1 has only `tail` valid
+// bits; every pad position expands to the value 0.
 
-// One thread produces 16 consecutive bytes of a row.  `period`/`tail` describe where pad bits sit:
-// word (w mod period) == period-1 has only `tail` valid bits; every pad position expands to 0.
+// int8 form: one thread produces 16 consecutive bytes (half a source word) of a row.
 __global__ void __launch_bounds__(256) expand_i8_kernel(const uint32_t *__restrict__ planes, int nplanes, int pm1,
                                                         int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
-                                                        int64_t period, int tail, int64_t kp, uint8_t *__restrict__ out)
+                                                        int64_t period, int tail, uint8_t *__restrict__ out, int64_t out_ld)
 {
-    const int64_t chunks = kp >> 4;
+    const int64_t chunks = kwords * 2;
     const int64_t total = rows * chunks;
     const uint32_t lcode = (1u << nplanes) - 1u;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -322,33 +489,68 @@ __global__ void __launch_bounds__(256) expand_i8_kernel(const uint32_t *__restri
         const int64_t ch = e - r * chunks;
         const int64_t widx = ch >> 1;
         const int half = (int)(ch & 1);
-        uint32_t o[4] = {0u, 0u, 0u, 0u};
-        if (widx < kwords) {
-            const int valid = ((widx % period) == period - 1) ? tail : 32;
-            const uint32_t vword = (valid >= 32) ? 0xffffffffu : ((1u << valid) - 1u);
-            const uint32_t vm = (vword >> (16 * half)) & 0xffffu;
-            uint32_t acc[4] = {0u, 0u, 0u, 0u};
-            for (int i = 0; i < nplanes; ++i) {
-                const uint32_t w = __ldg(planes + i * plane_stride + r * ld + widx);
-                const uint32_t h = (w >> (16 * half)) & 0xffffu;
+        const int valid = ((widx % period) == period - 1) ? tail : 32;
+        const uint32_t vword = (valid >= 32) ? 0xffffffffu : ((1u << valid) - 1u);
+        const uint32_t vm = (vword >> (16 * half)) & 0xffffu;
+        uint32_t acc[4] = {0u, 0u, 0u, 0u};
+        for (int i = 0; i < nplanes; ++i) {
+            const uint32_t w = __ldg(planes + i * plane_stride + r * ld + widx);
+            const uint32_t h = (w >> (16 * half)) & 0xffffu;
 #pragma unroll
-                for (int nb = 0; nb < 4; ++nb) {
-                    const uint32_t nib = (h >> (4 * nb)) & 0xfu;
-                    acc[nb] += ((nib * 0x00204081u) & 0x01010101u) << i;       // bit j of the nibble -> byte j
-                }
-            }
-#pragma unroll
-            for (int nb = 0; nb < 4; ++nb) {
-                uint32_t v = acc[nb];
-                if (pm1) v = __vsub4(v << 1, lcode * 0x01010101u);              // 2q - (2^k - 1) per byte
-                const uint32_t mnib = (vm >> (4 * nb)) & 0xfu;
-                const uint32_t mask = ((mnib * 0x00204081u) & 0x01010101u) * 0xffu;
-                o[nb] = v & mask;
-            }
+            for (int nb = 0; nb < 4; ++nb) acc[nb] += spread_bits_to_bytes((h >> (4 * nb)) & 0xfu) << i;
         }
-        *reinterpret_cast<uint4 *>(out + r * kp + ch * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        uint32_t o[4];
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+            uint32_t v = acc[nb];
+            if (pm1) v = __vsub4(v << 1, lcode * 0x01010101u);                  // 2q - (2^k - 1) per byte
+            o[nb] = v & (spread_bits_to_bytes((vm >> (4 * nb)) & 0xfu) * 0xffu);
+        }
+        *reinterpret_cast<uint4 *>(out + r * out_ld + ch * 16) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
+
+// e2m1 code of an integer value in {0, +-1, +-2, +-3}: sign bit 3; magnitudes 1 -> 0b010, 2 -> 0b100, 3 -> 0b101.
+// fp4 form: one thread turns one source word (per plane) into 32 nibbles = 16 bytes.
+__global__ void __launch_bounds__(256) expand_fp4_kernel(const uint32_t *__restrict__ planes, int nplanes, int pm1,
+                                                         int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
+                                                         int64_t period, int tail, uint8_t *__restrict__ out, int64_t out_ld)
+{
+    const int64_t total = rows * kwords;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = e / kwords;
+        const int64_t w = e - r * kwords;
+        const int valid = ((w % period) == period - 1) ? tail : 32;
+        const uint32_t vword = (valid >= 32) ? 0xffffffffu : ((1u << valid) - 1u);
+        const uint32_t p0 = __ldg(planes + r * ld + w);
+        const uint32_t p1 = nplanes > 1 ? __ldg(planes + plane_stride + r * ld + w) : 0u;
+        uint32_t o[4];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const uint32_t s0 = spread_bits_to_nibbles((p0 >> (8 * b)) & 0xffu);
+            const uint32_t s1 = spread_bits_to_nibbles((p1 >> (8 * b)) & 0xffu);
+            const uint32_t vm = spread_bits_to_nibbles((vword >> (8 * b)) & 0xffu) * 0xfu;
+            uint32_t code;
+            if (pm1) {
+                if (nplanes == 1) {
+                    code = 0xAAAAAAAAu ^ (s0 << 3);                            // bit 1 -> +1 (0x2), bit 0 -> -1 (0xA)
+                } else {
+                    // value 2*q - 3 with q = s0 + 2*s1: q 0 -> -3, 1 -> -1, 2 -> +1, 3 -> +3
+                    const uint32_t neg = (s1 ^ 0x11111111u) << 3;               // sign: negative while plane 1 is clear
+                    const uint32_t three = ~(s0 ^ s1) & 0x11111111u;            // |value| = 3 when both planes agree
+                    code = neg | (three * 0x5u) | ((three ^ 0x11111111u) << 1);  // 3 -> 0b101, 1 -> 0b010
+                }
+            } else {
+                // unsigned code q = s0 + 2*s1: 0 -> 0, 1 -> 0b010, 2 -> 0b100, 3 -> 0b101
+                code = (s1 << 2) | ((s0 & ~s1) << 1) | (s0 & s1);
+            }
+            o[b] = code & vm;
+        }
+        *reinterpret_cast<uint4 *>(out + r * out_ld + w * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// ---- tensor maps -------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -367,26 +569,43 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-int make_map(CUtensorMap *map, const uint8_t *base, int64_t rows, int64_t kp, int box_rows)
+// 2-D byte matrix [rows, row_bytes] with rows ld_bytes apart; box = 128 bytes x box_rows; reads past either extent give 0
+int make_map_2d(CUtensorMap *map, const void *base, int64_t rows, int64_t row_bytes, int64_t ld_bytes, int box_rows)
 {
     EncodeTiledFn fn = encode_fn();
     QNN_REQUIRE(fn != nullptr, QNN_ERR_CUDA, "tc gemm: cuTensorMapEncodeTiled is not available from this driver");
-    cuuint64_t dims[2] = {(cuuint64_t)kp, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)kp};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)BKB, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t *>(base), dims, strides, box, estr,
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     QNN_REQUIRE(r == CUDA_SUCCESS, QNN_ERR_CUDA, "tc gemm: cuTensorMapEncodeTiled failed with code %d", (int)r);
     return QNN_OK;
 }
 
-template <int BN>
+// 4-D NHWC byte tensor [B, H, W, cbytes]; box = 128 bytes x W x box_h x 1
+int make_map_nhwc(CUtensorMap *map, const void *base, int B, int H, int W, int64_t cbytes, int box_h)
+{
+    EncodeTiledFn fn = encode_fn();
+    QNN_REQUIRE(fn != nullptr, QNN_ERR_CUDA, "tc conv: cuTensorMapEncodeTiled is not available from this driver");
+    cuuint64_t dims[4] = {(cuuint64_t)cbytes, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t strides[3] = {(cuuint64_t)cbytes, (cuuint64_t)cbytes * W, (cuuint64_t)cbytes * W * H};
+    cuuint32_t box[4] = {(cuuint32_t)BKB, (cuuint32_t)W, (cuuint32_t)box_h, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    QNN_REQUIRE(r == CUDA_SUCCESS, QNN_ERR_CUDA, "tc conv: cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return QNN_OK;
+}
+
+template <int FORM, int BN>
 int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cudaStream_t st)
 {
-    using S = TcSmem<BN>;
-    auto kern = gemm_i8_kernel<BN>;
+    using S = TcCfg<FORM, BN>;
+    auto kern = gemm_tc_kernel<FORM, BN>;
     QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
     p.tiles_n = (int32_t)ceil_div(p.N, BN);
     p.idesc |= (uint32_t)(BN >> 3) << 17;
@@ -398,39 +617,103 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cuda
     return check_launch("tc gemm");
 }
 
-inline int64_t kp_of(int64_t kwords) { return (int64_t)round_up((size_t)kwords * 32, BK); }
+// Tile width: fewest waves of the persistent grid, weighted by the width (a wave of wider tiles takes longer).
+int pick_bn(int form, int64_t tiles_m, int64_t N)
+{
+    static const int fp4_bn[] = {224, 192, 128, 64, 32};
+    static const int i8_bn[] = {256, 128, 64, 32};
+    const int *cand = form == QNN_FORM_FP4 ? fp4_bn : i8_bn;
+    const int ncand = form == QNN_FORM_FP4 ? 5 : 4;
+    int best = cand[0];
+    double best_cost = 1e300;
+    for (int i = 0; i < ncand; ++i) {
+        const int bn = cand[i];
+        const int64_t tiles = tiles_m * ceil_div(N, bn);
+        const int64_t waves = ceil_div(tiles, sm_count());
+        const double cost = (double)waves * (bn + 24);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+int grid_for_items(int64_t items)
+{
+    const int64_t need = ceil_div(items, 256);
+    const int64_t cap = (int64_t)sm_count() * 16;
+    return (int)(need < cap ? need : cap);
+}
 
 }  // namespace
 
+bool tc_form_holds(int form, int planes, int mode)
+{
+    if (form == QNN_FORM_FP4) return planes <= 2;                       // {0..3} or {-3,-1,1,3}
+    if (form == QNN_FORM_I8) return mode == QNN_MODE_PM1 ? planes <= 7 : planes <= 8;   // +-127 / 0..255
+    return false;
+}
+
+int tc_pick_form(int ka, int a_mode, int kb, int b_mode, int64_t K)
+{
+    const int64_t la = (1 << ka) - 1, lb = (1 << kb) - 1;
+    // fp32 accumulation of integer products stays exact while every partial sum is below 2^24
+    if (tc_form_holds(QNN_FORM_FP4, ka, a_mode) && tc_form_holds(QNN_FORM_FP4, kb, b_mode) && K * la * lb < ((int64_t)1 << 24))
+        return QNN_FORM_FP4;
+    if (tc_form_holds(QNN_FORM_I8, ka, a_mode) && tc_form_holds(QNN_FORM_I8, kb, b_mode)) return QNN_FORM_I8;
+    return 0;
+}
+
+int64_t tc_row_bytes(int64_t kwords, int form) { return form == QNN_FORM_FP4 ? kwords * 16 : kwords * 32; }
+
+int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
+              int64_t pad_period, int pad_tail, int form, uint8_t *dst, int64_t dst_ld, cudaStream_t st)
+{
+    if (rows == 0 || kwords == 0) return QNN_OK;
+    QNN_REQUIRE(tc_form_holds(form, planes, mode), QNN_ERR_UNSUPPORTED, "tc expand: %d planes do not fit form %d", planes, form);
+    if (form == QNN_FORM_FP4) {
+        expand_fp4_kernel<<<grid_for_items(rows * kwords), 256, 0, st>>>(src, planes, mode == QNN_MODE_PM1, ld, plane_stride,
+                                                                        rows, kwords, pad_period, pad_tail, dst, dst_ld);
+    } else {
+        expand_i8_kernel<<<grid_for_items(rows * kwords * 2), 256, 0, st>>>(src, planes, mode == QNN_MODE_PM1, ld, plane_stride,
+                                                                           rows, kwords, pad_period, pad_tail, dst, dst_ld);
+    }
+    return check_launch("tc expand");
+}
+
 bool gemm_tc_supported(const GemmArgs &g)
 {
-    // signed-symmetric codes of 8 planes reach +-255 and do not fit int8
-    if (g.a_mode == QNN_MODE_PM1 && g.ka > 7) return false;
-    if (g.b_mode == QNN_MODE_PM1 && g.kb > 7) return false;
+    if (tc_pick_form(g.ka, g.a_mode, g.kb, g.b_mode, g.K) == 0) return false;
     if (g.M > (int64_t)1 << 30 || g.N > (int64_t)1 << 30) return false;
     return true;
 }
 
 size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K, int, int)
 {
-    const int64_t kp = kp_of(ceil_div(K, 32));
-    return round_up((size_t)M * (size_t)kp, 256) + round_up((size_t)N * (size_t)kp, 256);
+    const int64_t rb = tc_row_bytes(ceil_div(K, 32), QNN_FORM_I8);
+    return round_up((size_t)M * (size_t)rb, 256) + round_up((size_t)N * (size_t)rb, 256);
 }
 
-int launch_gemm_tc(const GemmArgs &g, void *ws, size_t ws_bytes, cudaStream_t st)
+int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    QNN_REQUIRE(gemm_tc_supported(g), QNN_ERR_UNSUPPORTED,
-                "tc gemm: signed-symmetric operands of 8 planes do not fit int8; use QNN_ALGO_POPC");
     const int64_t kwords = g.kwords > 0 ? g.kwords : ceil_div(g.K, 32);
     QNN_REQUIRE(kwords > 0, QNN_ERR_UNSUPPORTED, "tc gemm: K = 0 is handled by QNN_ALGO_POPC");
-    const int64_t kp = kp_of(kwords);
-    const size_t a_bytes = round_up((size_t)g.M * (size_t)kp, 256);
-    const size_t need = a_bytes + round_up((size_t)g.N * (size_t)kp, 256);
-    QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= need, QNN_ERR_WORKSPACE,
-                "tc gemm: workspace of at least %zu bytes (256-byte aligned) required", need);
-    QNN_REQUIRE(kp / BK < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: K too large");
-    uint8_t *a8 = static_cast<uint8_t *>(ws);
-    uint8_t *b8 = a8 + a_bytes;
+    const int best = tc_pick_form(g.ka, g.a_mode, g.kb, g.b_mode, g.K);
+    if (form == 0) {
+        form = best;
+        if (g.a_tc) form = g.a_tc_form;                    // operands that already exist decide
+        else if (g.b_tc) form = g.b_tc_form;
+    }
+    QNN_REQUIRE(form == QNN_FORM_I8 || form == QNN_FORM_FP4, QNN_ERR_UNSUPPORTED,
+                "tc gemm: operand values do not fit a tensor-core form; use QNN_ALGO_POPC");
+    QNN_REQUIRE(tc_form_holds(form, g.ka, g.a_mode) && tc_form_holds(form, g.kb, g.b_mode) &&
+                    (form != QNN_FORM_FP4 || best == QNN_FORM_FP4),
+                QNN_ERR_UNSUPPORTED, "tc gemm: operand values (%d and %d planes, K = %lld) do not fit form %d", g.ka, g.kb,
+                (long long)g.K, form);
+    QNN_REQUIRE((!g.a_tc || g.a_tc_form == form) && (!g.b_tc || g.b_tc_form == form), QNN_ERR_INVALID_ARG,
+                "tc gemm: a prepared operand is in another form than the product uses");
+    QNN_REQUIRE(g.M <= (int64_t)1 << 30 && g.N <= (int64_t)1 << 30, QNN_ERR_UNSUPPORTED, "tc gemm: M or N too large");
+
+    const int64_t row_bytes = tc_row_bytes(kwords, form);
+    QNN_REQUIRE(ceil_div(row_bytes, BKB) < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: K too large");
 
     // where the pad bits are: a plain matrix pads only its last word; conv rows pad the last word of every tap
     int64_t period = kwords;
@@ -438,38 +721,97 @@ int launch_gemm_tc(const GemmArgs &g, void *ws, size_t ws_bytes, cudaStream_t st
     if (g.pad_period > 0) { period = g.pad_period; tail = g.pad_tail; }
     QNN_REQUIRE(tail >= 1 && tail <= 32, QNN_ERR_INVALID_ARG, "tc gemm: inconsistent K / kwords");
 
-    auto expand = [&](const uint32_t *src, int planes, int mode, int64_t ld, int64_t stride, int64_t rows, uint8_t *dst) {
-        const int64_t total = rows * (kp >> 4);
-        const int64_t need_blocks = ceil_div(total, 256);
-        const int64_t cap = (int64_t)sm_count() * 16;
-        const int blocks = (int)(need_blocks < cap ? need_blocks : cap);
-        expand_i8_kernel<<<blocks, 256, 0, st>>>(src, planes, mode == QNN_MODE_PM1, ld, stride, rows, kwords, period, tail,
-                                                 kp, dst);
-        return check_launch("tc gemm expand");
-    };
-    if (int rc = expand(g.a, g.ka, g.a_mode, g.lda, g.a_plane_stride, g.M, a8)) return rc;
-    if (int rc = expand(g.b, g.kb, g.b_mode, g.ldb, g.b_plane_stride, g.N, b8)) return rc;
+    // operands: use prepared ones, expand the others into the workspace
+    const uint8_t *a8 = static_cast<const uint8_t *>(g.a_tc);
+    const uint8_t *b8 = static_cast<const uint8_t *>(g.b_tc);
+    int64_t a_ld = g.a_tc_ld, b_ld = g.b_tc_ld;
+    int64_t a_row_bytes = row_bytes;
+    size_t need = 0;
+    const size_t a_bytes = g.a_tc ? 0 : round_up((size_t)g.M * (size_t)row_bytes, 256);
+    const size_t b_bytes = g.b_tc ? 0 : round_up((size_t)g.N * (size_t)row_bytes, 256);
+    need = a_bytes + b_bytes;
+    if (need > 0)
+        QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= need, QNN_ERR_WORKSPACE,
+                    "tc gemm: workspace of at least %zu bytes (256-byte aligned) required", need);
+    if (g.a_tc) {
+        QNN_REQUIRE(aligned(g.a_tc, 16) && a_ld % 16 == 0 && a_ld > 0, QNN_ERR_ALIGNMENT,
+                    "tc gemm: prepared A operand needs a 16-byte aligned base and row stride");
+        if (!g.conv && a_ld < row_bytes) a_row_bytes = a_ld;           // e.g. raw uint8 codes: K bytes per row, rest reads 0
+    } else {
+        QNN_REQUIRE(!g.conv, QNN_ERR_INVALID_ARG, "tc conv: the NHWC operand must be prepared");
+        uint8_t *dst = static_cast<uint8_t *>(ws);
+        if (int rc = tc_expand(g.a, g.ka, g.a_mode, g.lda, g.a_plane_stride, g.M, kwords, period, tail, form, dst, row_bytes, st))
+            return rc;
+        a8 = dst; a_ld = row_bytes;
+    }
+    if (g.b_tc) {
+        QNN_REQUIRE(aligned(g.b_tc, 16) && b_ld % 16 == 0 && b_ld >= row_bytes, QNN_ERR_ALIGNMENT,
+                    "tc gemm: prepared B operand needs a 16-byte aligned base and row stride");
+    } else {
+        uint8_t *dst = static_cast<uint8_t *>(ws) + a_bytes;
+        if (int rc = tc_expand(g.b, g.kb, g.b_mode, g.ldb, g.b_plane_stride, g.N, kwords, period, tail, form, dst, row_bytes, st))
+            return rc;
+        b8 = dst; b_ld = row_bytes;
+    }
 
     TcParams p{};
-    p.M = g.M; p.N = g.N; p.num_kb = (int32_t)(kp / BK);
+    p.M = g.M; p.N = g.N; p.num_kb = (int32_t)ceil_div(row_bytes, BKB);
     p.tiles_m = (int32_t)ceil_div(g.M, BM);
+    p.a_tx_bytes = BM * BKB;
     p.epilogue = g.epilogue; p.out = g.out; p.ldo = g.ldo; p.hw = g.hw > 0 ? g.hw : 1;
     p.thr = g.thr; p.flip = g.flip; p.out_bits = g.out_bits; p.ld_bits = g.ld_bits;
-    // instruction descriptor: int32 accumulator, A/B int8 signed (PM1) or unsigned (U01), both K-major, M = 128
-    p.idesc = (2u << 4) | ((g.a_mode == QNN_MODE_PM1 ? 1u : 0u) << 7) | ((g.b_mode == QNN_MODE_PM1 ? 1u : 0u) << 10) |
-              ((uint32_t)(BM >> 4) << 24);
+    p.out_form = static_cast<uint8_t *>(g.out_form); p.ld_form = g.ld_form; p.out_form_kind = g.out_form_kind;
+    if (g.out_form) {
+        QNN_REQUIRE(g.thr != nullptr, QNN_ERR_INVALID_ARG, "tc gemm: thresholds required for a form output");
+        QNN_REQUIRE(g.out_form_kind == QNN_FORM_I8 || g.out_form_kind == QNN_FORM_FP4, QNN_ERR_INVALID_ARG, "tc gemm: bad output form");
+        QNN_REQUIRE(aligned(g.out_form, 16) && g.ld_form % 16 == 0 &&
+                        g.ld_form >= tc_row_bytes(ceil_div(g.N, 32), g.out_form_kind),
+                    QNN_ERR_ALIGNMENT, "tc gemm: form output needs a 16-byte aligned base and a row stride covering N");
+    }
+    if (form == QNN_FORM_FP4) {
+        // block-scaled instruction descriptor: A and B e2m1 (format 1), both K-major, ue8m0 scales, M = 128
+        p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((uint32_t)(BM >> 4) << 24);
+    } else {
+        // int32 accumulator, A/B int8 signed (PM1) or unsigned (U01), both K-major, M = 128
+        p.idesc = (2u << 4) | ((g.a_mode == QNN_MODE_PM1 ? 1u : 0u) << 7) | ((g.b_mode == QNN_MODE_PM1 ? 1u : 0u) << 10) |
+                  ((uint32_t)(BM >> 4) << 24);
+    }
 
-    // widest tile that still gives every SM work
-    const int64_t tm = p.tiles_m;
-    int bn = 256;
-    if (tm * ceil_div(g.N, 256) < sm_count()) bn = 128;
-    if (bn == 128 && tm * ceil_div(g.N, 128) < sm_count()) bn = 64;
     CUtensorMap ma, mb;
-    if (int rc = make_map(&ma, a8, g.M, kp, BM)) return rc;
-    if (int rc = make_map(&mb, b8, g.N, kp, bn)) return rc;
-    if (bn == 256) return launch_tc_cfg<256>(ma, mb, p, st);
-    if (bn == 128) return launch_tc_cfg<128>(ma, mb, p, st);
-    return launch_tc_cfg<64>(ma, mb, p, st);
+    if (g.conv) {
+        const ConvImplicit &c = *g.conv;
+        QNN_REQUIRE(c.W >= 1 && c.W <= BM && c.KH == 2 * c.pad + 1 && c.KW == 2 * c.pad + 1 && c.pad <= 3,
+                    QNN_ERR_UNSUPPORTED, "tc conv: implicit path needs a stride-1 'same' filter and W <= 128");
+        const int R = BM / c.W < c.H ? BM / c.W : c.H;                  // image rows per tile
+        QNN_REQUIRE(R >= 1 && R <= 256, QNN_ERR_UNSUPPORTED, "tc conv: bad tile height");
+        p.conv = 1; p.cH = c.H; p.cW = c.W; p.cR = R; p.tiles_per_img = (int32_t)ceil_div(c.H, R);
+        p.cKW = c.KW; p.cpad = c.pad; p.cblocks = c.cblocks; p.corr = c.corr;
+        p.tiles_m = c.B * p.tiles_per_img;
+        p.a_tx_bytes = R * c.W * BKB;
+        QNN_REQUIRE(p.num_kb == c.KH * c.KW * c.cblocks, QNN_ERR_INVALID_ARG, "tc conv: K blocks do not match the filter");
+        QNN_REQUIRE(g.M == (int64_t)c.B * c.H * c.W, QNN_ERR_INVALID_ARG, "tc conv: M does not match the image geometry");
+        if (int rc = make_map_nhwc(&ma, a8, c.B, c.H, c.W, (int64_t)c.cblocks * BKB, R)) return rc;
+    } else {
+        if (int rc = make_map_2d(&ma, a8, g.M, a_row_bytes, a_ld, BM)) return rc;
+    }
+    const int bn = pick_bn(form, p.tiles_m, g.N);
+    if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn)) return rc;
+
+    if (form == QNN_FORM_FP4) {
+        switch (bn) {
+            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224>(ma, mb, p, st);
+            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192>(ma, mb, p, st);
+            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128>(ma, mb, p, st);
+            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64>(ma, mb, p, st);
+            default: return launch_tc_cfg<QNN_FORM_FP4, 32>(ma, mb, p, st);
+        }
+    }
+    switch (bn) {
+        case 256: return launch_tc_cfg<QNN_FORM_I8, 256>(ma, mb, p, st);
+        case 128: return launch_tc_cfg<QNN_FORM_I8, 128>(ma, mb, p, st);
+        case 64: return launch_tc_cfg<QNN_FORM_I8, 64>(ma, mb, p, st);
+        default: return launch_tc_cfg<QNN_FORM_I8, 32>(ma, mb, p, st);
+    }
 }
 
 }  // namespace qnn

@@ -42,6 +42,15 @@ void profile_after(cudaStream_t st);
 
 enum Epilogue { EPI_ROWMAJOR = 0, EPI_NCHW = 1, EPI_BITS = 2 };
 
+// Implicit-GEMM view of a stride-1 "same" convolution for the tensor-core path: the A operand is the
+// NHWC activation tensor in tensor-core form, read tap by tap through a 4-D tensor map whose
+// out-of-image reads return zero; `corr` adds back what the padding value contributes.
+struct ConvImplicit {
+    int32_t B, H, W, KH, KW, pad;
+    int32_t cblocks;            // 128-byte channel blocks per pixel
+    const int32_t *corr;        // [(pad+1)^4][N] border corrections, class 0 (interior) is all zero
+};
+
 struct GemmArgs {
     const uint32_t *a;      // ka planes [M, lda]
     const uint32_t *b;      // kb planes [N, ldb]
@@ -59,14 +68,33 @@ struct GemmArgs {
     const uint8_t *flip;
     uint32_t *out_bits;     // EPI_BITS: [M, ld_bits]
     int64_t ld_bits;
+    // ---- tensor-core extras (all optional) ----
+    const void *a_tc;       // A already in tensor-core form (QNN_FORM_*), rows a_tc_ld bytes apart
+    int a_tc_form;
+    int64_t a_tc_ld;
+    const void *b_tc;       // B likewise
+    int b_tc_form;
+    int64_t b_tc_ld;
+    void *out_form;         // thresholded signs written as the next product's A operand in form out_form_kind
+    int out_form_kind;
+    int64_t ld_form;        // bytes between rows of out_form
+    const ConvImplicit *conv;   // non-null: A is an NHWC tensor read as an implicit im2col
 };
 
 int validate_gemm(const GemmArgs &g);
 int launch_gemm_popc(const GemmArgs &g, cudaStream_t st);
 int launch_gemm_b1mma(const GemmArgs &g, cudaStream_t st);
-int launch_gemm_tc(const GemmArgs &g, void *ws, size_t ws_bytes, cudaStream_t st);
+// form: QNN_FORM_I8, QNN_FORM_FP4, or 0 = the best form the operands allow
+int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaStream_t st);
+// upper bound over the forms (the int8 form is the larger one)
 size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K, int ka, int kb);
 bool gemm_tc_supported(const GemmArgs &g);
+// best tensor-core form for the operand value sets (0 = none)
+int tc_pick_form(int ka, int a_mode, int kb, int b_mode, int64_t K);
+bool tc_form_holds(int form, int planes, int mode);
+int64_t tc_row_bytes(int64_t kwords, int form);
+int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
+              int64_t pad_period, int pad_tail, int form, uint8_t *dst, int64_t dst_ld, cudaStream_t st);
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st);
 
 }  // namespace qnn

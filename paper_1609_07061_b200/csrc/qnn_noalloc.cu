@@ -57,5 +57,5 @@ extern "C" int qnn_xnor_gemm_noalloc(const uint32_t *a, int64_t lda, const uint3
     if (int rc = scratch_for_current_device(&scratch)) return rc;
     // Every byte the product kernel reads from the scratch is rewritten by this call's expansion
     // passes first (pad positions included), so nothing has to be cleared between calls.
-    return launch_gemm_tc(g, scratch, (size_t)QNN_NOALLOC_SCRATCH_BYTES, as_stream(stream));
+    return launch_gemm_tc(g, QNN_FORM_I8, scratch, (size_t)QNN_NOALLOC_SCRATCH_BYTES, as_stream(stream));
 }

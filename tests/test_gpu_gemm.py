@@ -17,7 +17,7 @@ def q():
 
 
 def _algos(q):
-    return [q.QNN_ALGO_POPC, q.QNN_ALGO_B1_MMA, q.QNN_ALGO_TC_I8, q.QNN_ALGO_AUTO]
+    return [q.QNN_ALGO_POPC, q.QNN_ALGO_B1_MMA, q.QNN_ALGO_TC_I8, q.QNN_ALGO_AUTO, q.QNN_ALGO_TC_FP4]
 
 
 def _ws(q, op, M, N, K, ka=1, kb=1, algo=0):
@@ -54,7 +54,7 @@ SHAPES = [(1, 1, 1), (2, 3, 31), (5, 7, 32), (3, 2, 33), (31, 33, 63), (32, 32, 
           (257, 513, 784), (1, 1000, 2304), (300, 1, 96)]
 
 
-@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3])
+@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("M,N,K", SHAPES)
 def test_xnor_gemm_shapes(q, M, N, K, algo_idx):
     algo = _algos(q)[algo_idx]
@@ -65,7 +65,7 @@ def test_xnor_gemm_shapes(q, M, N, K, algo_idx):
     np.testing.assert_array_equal(got, oracle.xnor_gemm(X, W))
 
 
-@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3])
+@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3, 4])
 def test_xnor_gemm_extremes(q, algo_idx):
     """All-agree, all-disagree and alternating rows: closed forms K, -K, 0."""
     algo = _algos(q)[algo_idx]
@@ -77,7 +77,7 @@ def test_xnor_gemm_extremes(q, algo_idx):
     np.testing.assert_array_equal(got, oracle.xnor_gemm(X, W))
 
 
-@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3])
+@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3, 4])
 def test_fc_single_layer_config(q, algo_idx):
     """Config 1: X[100,4096] ~ N(0,1), W[4096,4096] ~ U(-1,1), seed 0, through the GPU packers and the product."""
     algo = _algos(q)[algo_idx]
@@ -108,7 +108,7 @@ def test_fc_single_layer_config(q, algo_idx):
         assert torch.equal(out2, out.t)
 
 
-@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3])
+@pytest.mark.parametrize("algo_idx", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("M,N,K", [(5, 7, 33), (64, 64, 128), (100, 130, 1000), (257, 96, 784), (33, 4096, 96)])
 @pytest.mark.parametrize("with_flip", [False, True])
 def test_xnor_gemm_threshold(q, M, N, K, with_flip, algo_idx):
@@ -148,7 +148,7 @@ def _values(codes, bits, mode):
     return codes.astype(np.int32) if mode == 0 else (2 * codes.astype(np.int32) - ((1 << bits) - 1))
 
 
-@pytest.mark.parametrize("algo_idx", [0, 2, 3])
+@pytest.mark.parametrize("algo_idx", [0, 2, 3, 4])
 @pytest.mark.parametrize("ka,a_mode,kb,b_mode", [(8, 0, 1, 1), (2, 0, 1, 1), (4, 1, 4, 1), (1, 1, 1, 1), (3, 0, 2, 0),
                                                  (2, 1, 3, 0), (1, 0, 1, 0), (8, 0, 8, 0), (7, 1, 7, 1), (8, 1, 2, 1)])
 @pytest.mark.parametrize("M,N,K", [(3, 5, 31), (65, 33, 100), (130, 257, 800)])
@@ -175,7 +175,7 @@ def test_bitplane_gemm_modes(q, ka, a_mode, kb, b_mode, M, N, K, algo_idx):
     out.check()
 
 
-@pytest.mark.parametrize("algo_idx", [0, 2, 3])
+@pytest.mark.parametrize("algo_idx", [0, 2, 3, 4])
 def test_bitplane_gemm_threshold(q, algo_idx):
     algo = _algos(q)[algo_idx]
     rng = np.random.default_rng(99)

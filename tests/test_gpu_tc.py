@@ -1,0 +1,198 @@
+"""GPU parity: tensor-core operand forms (prepack), the product on prepared operands, chained form outputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from util import Guarded, as_i32_words, dev, pack_bits_ref, unpack_words, words_np, words_per_row
+
+pytestmark = pytest.mark.gpu
+
+E2M1 = {0: 0x0, 1: 0x2, 2: 0x4, 3: 0x5, -1: 0xA, -2: 0xC, -3: 0xD}
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_1609_07061_b200.binding as b
+    return b
+
+
+def _planes_ref(codes, bits, ld):
+    return np.stack([pack_bits_ref(((codes >> i) & 1).astype(np.uint8), ld) for i in range(bits)])
+
+
+def _values(codes, bits, mode):
+    return codes.astype(np.int32) if mode == 0 else (2 * codes.astype(np.int32) - ((1 << bits) - 1))
+
+
+def form_ref(values, K, form, q):
+    """Test-side encoding of integer values [rows, K] in a tensor-core form (independent of the library)."""
+    rows = values.shape[0]
+    kp = words_per_row(K) * 32
+    v = np.zeros((rows, kp), np.int32)
+    v[:, :K] = values
+    if form == q.QNN_FORM_I8:
+        return (v & 0xff).astype(np.uint8)
+    nib = np.vectorize(E2M1.__getitem__)(v).astype(np.uint8)
+    return (nib[:, 0::2] | (nib[:, 1::2] << 4)).astype(np.uint8)
+
+
+@pytest.mark.parametrize("planes,mode,form_name", [(1, 1, "FP4"), (1, 0, "FP4"), (2, 0, "FP4"), (2, 1, "FP4"),
+                                                   (1, 1, "I8"), (8, 0, "I8"), (4, 1, "I8"), (7, 1, "I8"), (3, 0, "I8")])
+@pytest.mark.parametrize("rows,K", [(1, 1), (5, 31), (7, 33), (130, 784), (33, 1000)])
+def test_prepack_matches_reference_encoding(q, planes, mode, form_name, rows, K):
+    form = getattr(q, "QNN_FORM_" + form_name)
+    rng = np.random.default_rng(rows * 31 + K + planes * 7 + mode)
+    codes = rng.integers(0, 1 << planes, (rows, K)).astype(np.int32)
+    ld = words_per_row(K) + 2
+    pl = _planes_ref(codes, planes, ld)
+    rb = q.qnn_tc_row_bytes(K, form)
+    assert rb == words_per_row(K) * (32 if form == q.QNN_FORM_I8 else 16)
+    ldb = rb + 16
+    out = Guarded((rows, ldb), torch.uint8, fill=0x5C)
+    q.qnn_tc_prepack(as_i32_words(pl).cuda(), planes, mode, ld, rows * ld, rows, K, form, out.t, ldb)
+    torch.cuda.synchronize()
+    got = out.t.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :rb], form_ref(_values(codes, planes, mode), K, form, q))
+    assert (got[:, rb:] == 0x5C).all()
+    out.check()
+
+
+def test_prepack_rejects_values_that_do_not_fit(q):
+    out = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    pl = torch.zeros(8, 1, 1, dtype=torch.int32, device="cuda")
+    for planes, mode, form in [(3, 0, q.QNN_FORM_FP4), (3, 1, q.QNN_FORM_FP4), (8, 1, q.QNN_FORM_I8)]:
+        with pytest.raises(q.QnnError) as ei:
+            q.qnn_tc_prepack(pl, planes, mode, 1, 1, 1, 32, form, out, 32)
+        assert ei.value.status == q.QNN_ERR_UNSUPPORTED
+    assert q.qnn_tc_form(1, 1, 1, 1, 4096) == q.QNN_FORM_FP4
+    assert q.qnn_tc_form(2, 0, 1, 1, 9216) == q.QNN_FORM_FP4
+    assert q.qnn_tc_form(1, 1, 1, 1, 1 << 24) == q.QNN_FORM_I8       # fp32 sums would no longer be exact
+    assert q.qnn_tc_form(4, 1, 4, 1, 2048) == q.QNN_FORM_I8
+    assert q.qnn_tc_form(8, 1, 1, 1, 64) == 0
+
+
+@pytest.mark.parametrize("form_name", ["FP4", "I8"])
+@pytest.mark.parametrize("out_form_name", ["FP4", "I8"])
+@pytest.mark.parametrize("M,N,K", [(5, 7, 33), (130, 257, 800), (300, 96, 4096), (129, 1000, 96)])
+def test_tc_gemm_all_outputs(q, form_name, out_form_name, M, N, K):
+    """int32, packed bits and form output of one call, prepared operands, ragged shapes."""
+    form = getattr(q, "QNN_FORM_" + form_name)
+    oform = getattr(q, "QNN_FORM_" + out_form_name)
+    rng = np.random.default_rng(M + 3 * N + 5 * K)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+    s = oracle.xnor_gemm(X, W)
+    T = rng.integers(-20, 21, N).astype(np.int32)
+    T[::4] = s[0, ::4]
+    flip = rng.integers(0, 2, N).astype(np.uint8)
+    ld = words_per_row(K)
+    a = as_i32_words(pack_bits_ref((X >= 0).astype(np.uint8), ld)).cuda()
+    b = as_i32_words(pack_bits_ref((W >= 0).astype(np.uint8).T, ld)).cuda()
+    rb = q.qnn_tc_row_bytes(K, form)
+    af = torch.empty(M, rb, dtype=torch.uint8, device="cuda")
+    bf = torch.empty(N, rb + 32, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(a, 1, 1, ld, 0, M, K, form, af, rb)
+    q.qnn_tc_prepack(b, 1, 1, ld, 0, N, K, form, bf, rb + 32)
+    out = Guarded((M, N + 1), torch.int32, fill=-7)
+    ldw = words_per_row(N) + 1
+    bits = Guarded((M, ldw), torch.int32, fill=0x77777777)
+    orb = q.qnn_tc_row_bytes(N, oform)
+    of = Guarded((M, orb + 16), torch.uint8, fill=0x5C)
+    q.qnn_tc_gemm(q.tc_operand(af, rb, form), q.tc_operand(bf, rb + 32, form), M, N, K, out.t, N + 1, dev(T), dev(flip),
+                  bits.t, ldw, of.t, oform, orb + 16)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    np.testing.assert_array_equal(out.t.cpu().numpy()[:, :N], s)
+    assert (out.t.cpu().numpy()[:, N:] == -7).all()
+    want_bits = oracle.threshold(s, T, flip)
+    np.testing.assert_array_equal(unpack_words(words_np(bits.t), N), want_bits)
+    assert (words_np(bits.t)[:, words_per_row(N):] == 0x77777777).all()
+    got_f = of.t.cpu().numpy()
+    np.testing.assert_array_equal(got_f[:, :orb], form_ref(2 * want_bits.astype(np.int32) - 1, N, oform, q))
+    assert (got_f[:, orb:] == 0x5C).all()
+    for g in (out, bits, of):
+        g.check()
+
+
+@pytest.mark.parametrize("form_name", ["FP4", "I8"])
+def test_tc_gemm_chain_two_layers(q, form_name):
+    """Hidden layer -> form output -> next product, without ever materialising packed bits."""
+    form = getattr(q, "QNN_FORM_" + form_name)
+    rng = np.random.default_rng(17)
+    M, K, H, N = 200, 300, 500, 70
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W1 = rng.uniform(-1, 1, (K, H)).astype(np.float32)
+    W2 = rng.uniform(-1, 1, (H, N)).astype(np.float32)
+    T = rng.integers(-10, 11, H).astype(np.int32)
+    s1 = oracle.xnor_gemm(X, W1)
+    h = 2.0 * oracle.threshold(s1, T, None).astype(np.float32) - 1.0
+    want = oracle.xnor_gemm(h, W2)
+
+    def prep(bits01, rows, KK):
+        ld = words_per_row(KK)
+        w = as_i32_words(pack_bits_ref(bits01, ld)).cuda()
+        rb = q.qnn_tc_row_bytes(KK, form)
+        o = torch.empty(rows, rb, dtype=torch.uint8, device="cuda")
+        q.qnn_tc_prepack(w, 1, 1, ld, 0, rows, KK, form, o, rb)
+        return o, rb
+
+    af, rba = prep((X >= 0).astype(np.uint8), M, K)
+    w1f, _ = prep((W1 >= 0).astype(np.uint8).T, H, K)
+    w2f, rbh = prep((W2 >= 0).astype(np.uint8).T, N, H)
+    hf = torch.empty(M, rbh, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_gemm(q.tc_operand(af, rba, form), q.tc_operand(w1f, rba, form), M, H, K, thr=dev(T), out_form=hf,
+                  out_form_kind=form, ld_form_bytes=rbh)
+    out = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    q.qnn_tc_gemm(q.tc_operand(hf, rbh, form), q.tc_operand(w2f, rbh, form), M, N, H, out, N)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("K", [65536, 1 << 20])
+def test_fp4_accumulation_exact_at_large_sums(q, K):
+    """Closed forms at sums far beyond fp16/bf16 range: all-agree rows give +K, all-disagree -K, half-and-half 0."""
+    form = q.QNN_FORM_FP4
+    M, N = 4, 40
+    ld = K // 32
+    a = np.zeros((M, ld), np.uint32)
+    a[0, :] = 0xffffffff                                  # all +1
+    a[1, :] = 0                                           # all -1
+    a[2, : ld // 2] = 0xffffffff                          # first half +1
+    a[3, :] = 0x55555555
+    b = np.full((N, ld), 0xffffffff, np.uint32)           # all +1
+    b[1, :] = 0
+    b[2, :] = 0xaaaaaaaa
+    rb = q.qnn_tc_row_bytes(K, form)
+    af = torch.empty(M, rb, dtype=torch.uint8, device="cuda")
+    bf = torch.empty(N, rb, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(as_i32_words(a).cuda(), 1, 1, ld, 0, M, K, form, af, rb)
+    q.qnn_tc_prepack(as_i32_words(b).cuda(), 1, 1, ld, 0, N, K, form, bf, rb)
+    out = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    q.qnn_tc_gemm(q.tc_operand(af, rb, form), q.tc_operand(bf, rb, form), M, N, K, out, N)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy()
+    assert got[0, 0] == K and got[1, 0] == -K and got[2, 0] == 0 and got[3, 0] == 0
+    assert got[0, 1] == -K and got[1, 1] == K
+    assert got[3, 2] == -K and got[0, 2] == 0
+    assert (got[0, 3:] == K).all()
+
+
+def test_tc_gemm_argument_errors(q):
+    t = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    o = torch.zeros(16, dtype=torch.int32, device="cuda")
+    a = q.tc_operand(t, 16, q.QNN_FORM_FP4)
+    b8 = q.tc_operand(t, 32, q.QNN_FORM_I8)
+    with pytest.raises(q.QnnError) as ei:
+        q.qnn_tc_gemm(a, b8, 2, 2, 32, o, 2)
+    assert ei.value.status == q.QNN_ERR_INVALID_ARG
+    with pytest.raises(q.QnnError) as ei:
+        q.qnn_tc_gemm(a, a, 2, 2, 32)                      # no output
+    assert ei.value.status == q.QNN_ERR_INVALID_ARG
+    with pytest.raises(q.QnnError) as ei:
+        q.qnn_tc_gemm(a, a, 2, 2, 64, o, 2)                # rows of 16 bytes cannot hold K = 64
+    assert ei.value.status == q.QNN_ERR_INVALID_ARG
+    with pytest.raises(q.QnnError) as ei:
+        q.qnn_tc_gemm(q.tc_operand(t, 16, q.QNN_FORM_FP4, planes=3), a, 2, 2, 32, o, 2)
+    assert ei.value.status == q.QNN_ERR_UNSUPPORTED
