@@ -158,6 +158,8 @@ class MlpBench:
             self.packed.append(out); self.ldws.append(ld)
         self.thr = [t.cuda() for t in wl.Ts]
         self.layers = q.make_mlp_layers(self.packed, self.ldws, DIMS[:-1], DIMS[1:], self.thr, [None] * len(self.thr))
+        # weights rewritten once in the tensor-core form of their layer (model load, outside the step)
+        self.w_tc = q.prepack_mlp_weights(self.layers, self.packed, IN_BITS) if algo in (q.QNN_ALGO_AUTO,) else []
         self.ws = torch.empty(q.qnn_mlp_workspace_bytes(M, IN_BITS, self.layers, algo, 1), dtype=torch.uint8,
                               device="cuda")
         self.scores = torch.empty(M, DIMS[-1], dtype=torch.int32, device="cuda")
@@ -166,6 +168,7 @@ class MlpBench:
         self.kw0 = self.ldws[0]
         self.planes = torch.zeros(IN_BITS, M, self.kw0, dtype=torch.int32, device="cuda")
         self.act = [torch.zeros(M, 128, dtype=torch.int32, device="cuda") for _ in range(2)]
+        self.actf = [torch.zeros(M, 4096 // 2, dtype=torch.uint8, device="cuda") for _ in range(2)]
         gw = max(q.qnn_workspace_bytes(q.QNN_OP_BITPLANE_GEMM, M, DIMS[1], DIMS[0], IN_BITS, 1, algo),
                  q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, 4096, 4096, 1, 1, algo), 256)
         self.gws = torch.empty(gw, dtype=torch.uint8, device="cuda")
@@ -180,13 +183,39 @@ class MlpBench:
 
     def step_calls(self, ev=None):
         """The Algorithm-4 pass as individual C-ABI calls; `ev` (optional) brackets the dominant product."""
+        if self.algo == self.q.QNN_ALGO_AUTO:
+            return self.step_calls_tc(ev)
+        return self.step_calls_bits(ev)
+
+    def step_calls_tc(self, ev=None):
+        """Tensor-core chain: the uint8 input is the int8-form operand of layer 1 (Eq. 8 recomposed), hidden
+        activations travel as e2m1 values written by the previous product's threshold epilogue, the last
+        hidden layer emits packed bits for the 10-unit xor/popc head."""
+        q, M = self.q, self.M
+        I8, FP4 = q.QNN_FORM_I8, q.QNN_FORM_FP4
+        L = self.layers
+        rb = 4096 // 2
+        q.qnn_tc_gemm(q.tc_operand(self.x, DIMS[0], I8, IN_BITS, q.QNN_MODE_U01),
+                      q.tc_operand(self.w_tc[0], L[0].w_tc_ld, I8), M, DIMS[1], DIMS[0],
+                      thr=self.thr[0], out_form=self.actf[0], out_form_kind=FP4, ld_form_bytes=rb)
+        if ev is not None:
+            q.qnn_set_kernel_events(ev[0], ev[1])        # recorded by the library right around the product kernel
+        q.qnn_tc_gemm(q.tc_operand(self.actf[0], rb, FP4), q.tc_operand(self.w_tc[1], L[1].w_tc_ld, FP4), M, DIMS[2],
+                      DIMS[1], thr=self.thr[1], out_form=self.actf[1], out_form_kind=FP4, ld_form_bytes=rb)
+        q.qnn_tc_gemm(q.tc_operand(self.actf[1], rb, FP4), q.tc_operand(self.w_tc[2], L[2].w_tc_ld, FP4), M, DIMS[3],
+                      DIMS[2], thr=self.thr[2], out_bits=self.act[0], ld_words=128)
+        q.qnn_xnor_gemm(self.act[0], 128, self.packed[3], self.ldws[3], M, DIMS[4], DIMS[3], self.scores, DIMS[4],
+                        q.QNN_ALGO_POPC, None)
+
+    def step_calls_bits(self, ev=None):
+        """The pass on packed bits with a forced algorithm (plane split, per-call operand rewriting)."""
         q, M = self.q, self.M
         q.qnn_pack_planes_u8(self.x, M, DIMS[0], DIMS[0], IN_BITS, self.planes, self.kw0, M * self.kw0)
         q.qnn_bitplane_gemm_threshold(self.planes, IN_BITS, q.QNN_MODE_U01, self.kw0, M * self.kw0, self.packed[0], 1,
                                       q.QNN_MODE_PM1, self.ldws[0], 0, M, DIMS[1], DIMS[0], self.thr[0], None,
                                       self.act[0], 128, self.algo, self.gws)
         if ev is not None:
-            q.qnn_set_kernel_events(ev[0], ev[1])        # recorded by the library right around the product kernel
+            q.qnn_set_kernel_events(ev[0], ev[1])
         q.qnn_xnor_gemm_threshold(self.act[0], 128, self.packed[1], self.ldws[1], M, DIMS[2], DIMS[1], self.thr[1],
                                   None, self.act[1], 128, self.algo, self.gws)
         q.qnn_xnor_gemm_threshold(self.act[1], 128, self.packed[2], self.ldws[2], M, DIMS[3], DIMS[2], self.thr[2],
@@ -384,7 +413,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--algo", default="auto", choices=["auto", "popc", "tc_i8", "b1_mma"])
+    ap.add_argument("--algo", default="auto", choices=["auto", "popc", "tc_i8", "b1_mma", "tc_fp4"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-config extra records")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -398,7 +427,8 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     from paper_1609_07061_b200 import binding as q
     rank, world, local = _dist_setup(args.gpus)
-    algo = {"auto": q.QNN_ALGO_AUTO, "popc": q.QNN_ALGO_POPC, "tc_i8": q.QNN_ALGO_TC_I8, "b1_mma": q.QNN_ALGO_B1_MMA}[args.algo]
+    algo = {"auto": q.QNN_ALGO_AUTO, "popc": q.QNN_ALGO_POPC, "tc_i8": q.QNN_ALGO_TC_I8, "b1_mma": q.QNN_ALGO_B1_MMA,
+            "tc_fp4": q.QNN_ALGO_TC_FP4}[args.algo]
     peaks = _peaks()
     bench = MlpBench(q, rank, algo)
     per_layer = _ops(BATCH)
@@ -467,14 +497,19 @@ def main():
         resolved = q.qnn_select_algo(BATCH, 4096, 4096, 1, 1, 1, 1) if algo == q.QNN_ALGO_AUTO else algo
         dom_ops = per_layer[1]
         achieved = dom_ops / (dom_ms / 1e3) / 1e12
-        if resolved == q.QNN_ALGO_TC_I8:
-            # int8 tensor peak = measured bf16 peak x the nominal int8:bf16 ratio (2).  The kernel is bracketed by its
-            # own event pair inside a sub-millisecond step with idle gaps (L2 flush) around it, so it runs at burst
-            # clocks: the burst figure is the denominator (the sustained one would read above 1).
+        if resolved == q.QNN_ALGO_TC_FP4:
+            # e2m1 tensor peak = measured bf16 peak x the nominal fp4:bf16 ratio (4).  The kernel is bracketed by its own
+            # event pair inside a sub-millisecond step with idle gaps (L2 flush) around it, so it runs at burst clocks.
+            bound, peak = "tensor", 4.0 * peaks["bf16_tflops"]
+            peak_note = (f"4 x {peaks['source']} burst bf16 ({peaks['bf16_tflops']} TF/s; sustained "
+                         f"{peaks['bf16_tflops_sustained']}); one e2m1 MAC = one +-1 product")
+            kernel = "tcgen05 kind::mxf4 xnor product 10000x4096x4096, threshold epilogue (gemm_tc_kernel<FP4>)"
+            dtype = "fp4 (e2m1 values, unit scales, fp32 accumulate: exact integers)"
+        elif resolved == q.QNN_ALGO_TC_I8:
             bound, peak = "tensor", 2.0 * peaks["bf16_tflops"]
             peak_note = (f"2 x {peaks['source']} burst bf16 ({peaks['bf16_tflops']} TF/s; sustained "
                          f"{peaks['bf16_tflops_sustained']}); one int8 MAC = one +-1 product")
-            kernel = "tcgen05 kind::i8 xnor product 10000x4096x4096, threshold epilogue (gemm_i8_kernel)"
+            kernel = "tcgen05 kind::i8 xnor product 10000x4096x4096, threshold epilogue (gemm_tc_kernel<I8>)"
             dtype = "int8"
         else:
             # xor+popc+add on the CUDA cores: the popc unit issues 16 lanes/clk/SM -> 148 SM x 16 x 64 binary ops/clk
@@ -490,9 +525,9 @@ def main():
             "config": {"workload": "MNIST-shaped binarised MLP 784-4096-4096-4096-10 (Algorithm 4), batch 10000 per GPU, "
                                    "8-bit inputs as 8 bit-planes (K 784 padded to 800+), thresholds in [-64,64], seed 1",
                        "global_batch": BATCH * world, "parallelism": f"dp{world} (independent batch shards, no collective)",
-                       "algo": {0: "auto", 1: "popc", 2: "tc_i8", 3: "b1_mma"}[resolved],
+                       "algo": {0: "auto", 1: "popc", 2: "tc_i8", 3: "b1_mma", 4: "tc_fp4"}[resolved],
                        "l2": "flushed between steps (256 MiB device fill, then a 256 MiB read so no dirty lines remain; untimed)",
-                       "weights": "packed once at load (not in the step)"},
+                       "weights": "packed and rewritten in tensor-core form once at load (not in the step)"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * DIMS[0],
                     "d2h_bytes_per_step": BATCH * DIMS[-1] * 4, "ms_per_step": e2e_ms / args.steps,
                     "matches_device_arm": same},

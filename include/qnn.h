@@ -55,7 +55,7 @@
 extern "C" {
 #endif
 
-#define QNN_VERSION 100
+#define QNN_VERSION 200
 
 /* status codes */
 #define QNN_OK 0
@@ -233,7 +233,10 @@ typedef struct qnn_tc_output { /* any subset; at least one of out / out_bits / o
     int64_t ld_form_bytes;
 } qnn_tc_output;
 
-/* out[m,n] = sum_k A[m,k] * B[n,k] on prepared operands (same form for both). */
+/* out[m,n] = sum_k A[m,k] * B[n,k] on prepared operands (same form for both).
+ * The A operand of a QNN_FORM_I8 product may also be a plain uint8 / int8 matrix
+ * of codes (planes = their bit-width) with ld_bytes >= K: Eq. 8's 8-bit input
+ * needs no plane split on this path. */
 QNN_API int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_t M, int64_t N, int64_t K,
                         const qnn_tc_output *o, void *stream);
 
@@ -325,7 +328,18 @@ typedef struct qnn_mlp_layer {
     int64_t N;           /* units of this layer                               */
     const int32_t *thr;  /* int32 [N]; ignored for the last layer             */
     const uint8_t *flip; /* uint8 [N] or NULL; ignored for the last layer     */
+    /* Optional: the same weights already in a tensor-core form (qnn_tc_prepack
+     * with 1 plane, QNN_MODE_PM1), so that the runner does not rewrite them on
+     * every pass.  Used when w_tc != NULL and w_tc_form is the form the layer
+     * runs in (qnn_mlp_layer_form); ignored otherwise. */
+    const void *w_tc;
+    int64_t w_tc_ld;     /* bytes between rows of w_tc                        */
+    int w_tc_form;       /* QNN_FORM_*                                        */
 } qnn_mlp_layer;
+
+/* Form in which layer `l` multiplies when it runs on the tensor cores
+ * (layer 0: in_bits-bit unsigned codes x +-1 weights; others +-1 x +-1). */
+QNN_API int qnn_mlp_layer_form(const qnn_mlp_layer *layers, int L, int l, int in_bits);
 
 /* Algorithm 4 "Running a BNN with L layers" on device buffers:
  * layer 1 is the bit-plane product of the in_bits-bit input (Eq. 8), hidden

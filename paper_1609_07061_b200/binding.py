@@ -53,7 +53,8 @@ class qnn_tc_output(ctypes.Structure):
 
 
 class qnn_mlp_layer(ctypes.Structure):
-    _fields_ = [("w", vp), ("ldw", i64), ("K", i64), ("N", i64), ("thr", vp), ("flip", vp)]
+    _fields_ = [("w", vp), ("ldw", i64), ("K", i64), ("N", i64), ("thr", vp), ("flip", vp),
+                ("w_tc", vp), ("w_tc_ld", i64), ("w_tc_form", i32)]
 
 
 _SIGS = {
@@ -85,6 +86,7 @@ _SIGS = {
     "qnn_binary_conv2d": (i32, [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, vp, sz, vp]),
     "qnn_mlp_forward": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
     "qnn_mlp_forward_host": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
+    "qnn_mlp_layer_form": (i32, [ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
     "qnn_mlp_workspace_bytes": (sz, [i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
     "qnn_workspace_bytes": (sz, [i32, i64, i64, i64, i32, i32, i32]),
     "qnn_select_algo": (i32, [i64, i64, i64, i32, i32, i32, i32]),
@@ -254,6 +256,27 @@ def make_mlp_layers(ws: Sequence[torch.Tensor], ldws: Sequence[int], Ks: Sequenc
         arr[l].thr = _p(thrs[l]) if l < len(thrs) else None
         arr[l].flip = _p(flips[l]) if l < len(flips) else None
     return arr
+
+
+def qnn_mlp_layer_form(layers, l, in_bits) -> int:
+    return int(_lib.qnn_mlp_layer_form(layers, len(layers), l, in_bits))
+
+
+def prepack_mlp_weights(layers, ws: Sequence[torch.Tensor], in_bits: int) -> List[torch.Tensor]:
+    """Rewrites every layer's packed weights once in the tensor-core form the layer runs in (qnn_tc_prepack) and
+    stores the pointers in the layer structs.  Returns the buffers: the caller keeps them alive."""
+    keep = []
+    for l in range(len(layers)):
+        form = qnn_mlp_layer_form(layers, l, in_bits)
+        if form == 0:
+            continue
+        K, N = int(layers[l].K), int(layers[l].N)
+        rb = qnn_tc_row_bytes(K, form)
+        buf = torch.empty(N, rb, dtype=torch.uint8, device="cuda")
+        qnn_tc_prepack(ws[l], 1, QNN_MODE_PM1, int(layers[l].ldw), 0, N, K, form, buf, rb)
+        layers[l].w_tc, layers[l].w_tc_ld, layers[l].w_tc_form = buf.data_ptr(), rb, form
+        keep.append(buf)
+    return keep
 
 
 def qnn_mlp_workspace_bytes(M, in_bits, layers, algo=QNN_ALGO_AUTO, host_io=0) -> int:

@@ -20,13 +20,21 @@ int validate_gemm(const GemmArgs &g)
                 (long long)la, (long long)lb);
     if (g.M == 0 || g.N == 0) return QNN_OK;
     const int64_t kw = g.kwords > 0 ? g.kwords : ceil_div(g.K, 32);
-    QNN_REQUIRE(g.out != nullptr || g.out_bits != nullptr, QNN_ERR_INVALID_ARG, "gemm: no output buffer");
+    QNN_REQUIRE(g.out != nullptr || g.out_bits != nullptr || g.out_form != nullptr, QNN_ERR_INVALID_ARG,
+                "gemm: no output buffer");
     if (g.K > 0) {
-        QNN_REQUIRE(g.a && g.b, QNN_ERR_INVALID_ARG, "gemm: NULL operand");
-        QNN_REQUIRE(g.lda >= kw && g.ldb >= kw, QNN_ERR_INVALID_ARG, "gemm: lda/ldb smaller than ceil(K/32)");
-        QNN_REQUIRE(g.ka == 1 || g.a_plane_stride >= g.M * g.lda, QNN_ERR_INVALID_ARG, "gemm: a_plane_stride too small");
-        QNN_REQUIRE(g.kb == 1 || g.b_plane_stride >= g.N * g.ldb, QNN_ERR_INVALID_ARG, "gemm: b_plane_stride too small");
-        QNN_REQUIRE(aligned(g.a, 4) && aligned(g.b, 4), QNN_ERR_ALIGNMENT, "gemm: operands must be 4-byte aligned");
+        // an operand is given as packed planes, or already in a tensor-core form
+        QNN_REQUIRE((g.a || g.a_tc) && (g.b || g.b_tc), QNN_ERR_INVALID_ARG, "gemm: NULL operand");
+        if (!g.a_tc) {
+            QNN_REQUIRE(g.lda >= kw, QNN_ERR_INVALID_ARG, "gemm: lda smaller than ceil(K/32)");
+            QNN_REQUIRE(g.ka == 1 || g.a_plane_stride >= g.M * g.lda, QNN_ERR_INVALID_ARG, "gemm: a_plane_stride too small");
+            QNN_REQUIRE(aligned(g.a, 4), QNN_ERR_ALIGNMENT, "gemm: operands must be 4-byte aligned");
+        }
+        if (!g.b_tc) {
+            QNN_REQUIRE(g.ldb >= kw, QNN_ERR_INVALID_ARG, "gemm: ldb smaller than ceil(K/32)");
+            QNN_REQUIRE(g.kb == 1 || g.b_plane_stride >= g.N * g.ldb, QNN_ERR_INVALID_ARG, "gemm: b_plane_stride too small");
+            QNN_REQUIRE(aligned(g.b, 4), QNN_ERR_ALIGNMENT, "gemm: operands must be 4-byte aligned");
+        }
     }
     if (g.out) {
         QNN_REQUIRE(aligned(g.out, 4), QNN_ERR_ALIGNMENT, "gemm: out must be 4-byte aligned");
@@ -72,6 +80,8 @@ int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_
         }
         if (algo == QNN_ALGO_B1_MMA && !(g.ka == 1 && g.kb == 1)) algo = QNN_ALGO_POPC;
     }
+    if (algo == QNN_ALGO_POPC || algo == QNN_ALGO_B1_MMA)
+        QNN_REQUIRE(g.a && g.b && !g.out_form, QNN_ERR_INVALID_ARG, "gemm: the CUDA-core paths take packed planes and write no form output");
     switch (algo) {
         case QNN_ALGO_POPC: return launch_gemm_popc(g, st);
         case QNN_ALGO_B1_MMA: return launch_gemm_b1mma(g, st);
@@ -199,7 +209,9 @@ int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_t M, int
     QNN_REQUIRE(!(o->out_bits || o->out_form) || o->thr, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: thresholds required");
     QNN_REQUIRE(!o->out_bits || o->ld_words >= ceil_div(N, 32), QNN_ERR_INVALID_ARG, "qnn_tc_gemm: ld_words too small");
     const int64_t rb = tc_row_bytes(ceil_div(K, 32), a->form);
-    QNN_REQUIRE(a->ld_bytes >= rb && b->ld_bytes >= rb, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: operand row stride smaller than K needs");
+    // A in the int8 form may be a plain byte matrix whose rows are only K bytes apart: the rest of the last word reads 0
+    const int64_t a_min = a->form == QNN_FORM_I8 ? K : rb;
+    QNN_REQUIRE(a->ld_bytes >= a_min && b->ld_bytes >= rb, QNN_ERR_INVALID_ARG, "qnn_tc_gemm: operand row stride smaller than K needs");
     return launch_gemm_tc(g, a->form, nullptr, 0, as_stream(stream));
 }
 

@@ -214,6 +214,80 @@ __global__ void __launch_bounds__(THREADS) gemm_popc_kernel(const PopcParams P)
     }
 }
 
+// Few output units (a classifier head: N <= 16), 1-bit x 1-bit: the work is one pass over the packed
+// activations, so the kernel is a streaming one.  B's rows sit in shared memory; a warp owns a row
+// of A, each lane xor/popc-ing every 32nd 128-bit chunk against all N rows, then the N partial
+// counts are summed across the warp.
+constexpr int SKINNY_N = 16;
+__global__ void __launch_bounds__(256) gemm_popc_skinny_kernel(const uint32_t *__restrict__ a, int64_t lda,
+                                                               const uint32_t *__restrict__ b, int64_t ldb, int64_t M,
+                                                               int N, int64_t kwords, int32_t K, int32_t *__restrict__ out,
+                                                               int64_t ldo)
+{
+    extern __shared__ __align__(16) uint32_t bs[];               // [N][kw4], kw4 = kwords rounded up to 4, zero padded
+    const int64_t kw4 = (kwords + 3) & ~(int64_t)3;
+    for (int64_t e = threadIdx.x; e < (int64_t)N * kw4; e += blockDim.x) {
+        const int64_t n = e / kw4, k = e - n * kw4;
+        bs[e] = k < kwords ? __ldg(b + n * ldb + k) : 0u;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const bool vec = ((lda & 3) == 0) && ((reinterpret_cast<uintptr_t>(a) & 15) == 0);
+    for (int64_t m = warp0; m < M; m += nwarps) {
+        int32_t acc[SKINNY_N];
+#pragma unroll
+        for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0;
+        const uint32_t *arow = a + m * lda;
+        for (int64_t k = (int64_t)lane * 4; k < kwords; k += 128) {
+            uint4 av;
+            if (vec && k + 4 <= kwords) {
+                av = __ldcs(reinterpret_cast<const uint4 *>(arow + k));
+            } else {
+                av.x = arow[k];
+                av.y = k + 1 < kwords ? arow[k + 1] : 0u;
+                av.z = k + 2 < kwords ? arow[k + 2] : 0u;
+                av.w = k + 3 < kwords ? arow[k + 3] : 0u;
+            }
+#pragma unroll
+            for (int n = 0; n < SKINNY_N; ++n) {
+                if (n < N) {
+                    const uint4 bv = *reinterpret_cast<const uint4 *>(bs + n * kw4 + k);
+                    acc[n] += __popc(av.x ^ bv.x) + __popc(av.y ^ bv.y) + __popc(av.z ^ bv.z) + __popc(av.w ^ bv.w);
+                }
+            }
+        }
+        int32_t mine = 0;
+#pragma unroll
+        for (int n = 0; n < SKINNY_N; ++n) {
+            if (n < N) {
+                int32_t v = acc[n];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == n) mine = v;
+            }
+        }
+        if (lane < N) out[m * ldo + lane] = K - 2 * mine;
+    }
+}
+
+int launch_skinny(const PopcParams &P, cudaStream_t st)
+{
+    const GemmArgs &g = P.g;
+    const int64_t kw4 = (P.kwords + 3) & ~(int64_t)3;
+    const size_t smem = sizeof(uint32_t) * (size_t)g.N * (size_t)kw4;
+    auto kern = gemm_popc_skinny_kernel;
+    if (smem > 48 * 1024) QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int64_t need = ceil_div(g.M, 8);
+    const int64_t cap = (int64_t)sm_count() * 8;
+    const int blocks = (int)(need < cap ? need : cap);
+    profile_before(st);
+    kern<<<blocks, 256, smem, st>>>(g.a, g.lda, g.b, g.ldb, g.M, (int)g.N, P.kwords, P.kll, g.out, g.ldo);
+    profile_after(st);
+    return check_launch("popc gemm (few units)");
+}
+
 template <int BM, int BN, int TM, int TN, int MODE, bool SINGLE>
 int launch_cfg(const PopcParams &P, cudaStream_t st)
 {
@@ -259,7 +333,13 @@ int launch_gemm_popc(const GemmArgs &g, cudaStream_t st)
     P.kll = (int32_t)(g.K * P.la * P.lb);
     const bool a_pm = g.a_mode == QNN_MODE_PM1, b_pm = g.b_mode == QNN_MODE_PM1;
     if (a_pm && b_pm) {
-        if (g.ka == 1 && g.kb == 1) return launch_mode<M_XOR, true>(P, st);
+        if (g.ka == 1 && g.kb == 1) {
+            const bool skinny = g.N <= SKINNY_N && g.M >= 64 && g.epilogue == EPI_ROWMAJOR && g.out != nullptr &&
+                                g.out_bits == nullptr && g.kwords == 0 &&
+                                sizeof(uint32_t) * (size_t)g.N * (size_t)(P.kwords + 3) <= 160 * 1024;
+            if (skinny) return launch_skinny(P, st);
+            return launch_mode<M_XOR, true>(P, st);
+        }
         return launch_mode<M_XOR, false>(P, st);
     }
     if (!a_pm && b_pm) return launch_mode<M_AND_SA, false>(P, st);

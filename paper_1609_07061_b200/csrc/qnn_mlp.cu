@@ -1,21 +1,62 @@
 // Algorithm 4 ("Running a BNN with L layers") as a chain of library calls on
 // one stream: bit-plane first layer, thresholded XNOR hidden layers with packed
 // activations ping-ponging between two workspace buffers, int32 scores last.
+#include <cstdlib>
+#include <cstring>
 #include "qnn_internal.cuh"
 
 namespace qnn {
 namespace {
 
+struct LayerChoice {
+    int algo;               // resolved algorithm of this layer (never AUTO)
+    int form;               // tensor-core form when algo is a tensor-core one, else 0
+};
+
 struct MlpPlan {
     int64_t kw0;            // words per row of one input plane
     size_t off_x, off_scores, off_planes, off_act0, off_act1, off_gemm;
-    size_t gemm_bytes, total;
+    size_t gemm_bytes, act_bytes, total;
 };
+
+inline bool is_tc(int algo) { return algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_TC_FP4; }
+
+int resolve_env_algo()
+{
+    const char *e = getenv("QNN_FORCE_ALGO");
+    if (!e || !*e) return QNN_ALGO_AUTO;
+    if (!strcmp(e, "POPC") || !strcmp(e, "1")) return QNN_ALGO_POPC;
+    if (!strcmp(e, "TC_I8") || !strcmp(e, "2")) return QNN_ALGO_TC_I8;
+    if (!strcmp(e, "B1_MMA") || !strcmp(e, "3")) return QNN_ALGO_B1_MMA;
+    if (!strcmp(e, "TC_FP4") || !strcmp(e, "4")) return QNN_ALGO_TC_FP4;
+    return QNN_ALGO_AUTO;
+}
+
+// Algorithm and form of layer l.  A forced algorithm that cannot run a layer's operands (the 1-bit
+// paths on the 8-plane first layer, a form that does not hold the values) falls back to the one
+// AUTO would take, so that a network always runs.
+LayerChoice choose_layer(int64_t M, int in_bits, const qnn_mlp_layer *layers, int l, int algo)
+{
+    const qnn_mlp_layer &ly = layers[l];
+    const int ka = l == 0 ? in_bits : 1;
+    const int a_mode = l == 0 ? QNN_MODE_U01 : QNN_MODE_PM1;
+    const int best_form = tc_pick_form(ka, a_mode, 1, QNN_MODE_PM1, ly.K);
+    if (algo == QNN_ALGO_AUTO) algo = resolve_env_algo();
+    LayerChoice c{algo, 0};
+    if (algo == QNN_ALGO_AUTO) c.algo = qnn_select_algo(M, ly.N, ly.K, ka, 1, a_mode, QNN_MODE_PM1);
+    if (c.algo == QNN_ALGO_B1_MMA && ka != 1) c.algo = QNN_ALGO_POPC;
+    if (c.algo == QNN_ALGO_TC_FP4 && best_form != QNN_FORM_FP4) c.algo = best_form ? QNN_ALGO_TC_I8 : QNN_ALGO_POPC;
+    if (c.algo == QNN_ALGO_TC_I8 && !(tc_form_holds(QNN_FORM_I8, ka, a_mode))) c.algo = QNN_ALGO_POPC;
+    if (c.algo == QNN_ALGO_TC_FP4) c.form = QNN_FORM_FP4;
+    if (c.algo == QNN_ALGO_TC_I8) c.form = QNN_FORM_I8;
+    return c;
+}
 
 int plan_mlp(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int algo, int host_io, MlpPlan *p)
 {
     QNN_REQUIRE(layers != nullptr && L >= 1, QNN_ERR_INVALID_ARG, "mlp: need at least one layer");
     QNN_REQUIRE(M >= 0 && in_bits >= 1 && in_bits <= 8, QNN_ERR_INVALID_ARG, "mlp: bad batch or input bit-width");
+    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_FP4, QNN_ERR_INVALID_ARG, "mlp: unknown algo %d", algo);
     for (int l = 0; l < L; ++l) {
         QNN_REQUIRE(layers[l].K >= 1 && layers[l].N >= 1 && layers[l].w != nullptr, QNN_ERR_INVALID_ARG,
                     "mlp: layer %d has a bad shape or NULL weights", l);
@@ -29,17 +70,21 @@ int plan_mlp(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int alg
     p->off_x = host_io ? take((size_t)M * (size_t)layers[0].K) : 0;
     p->off_scores = host_io ? take(sizeof(int32_t) * (size_t)M * (size_t)layers[L - 1].N) : 0;
     p->off_planes = take(sizeof(uint32_t) * (size_t)in_bits * (size_t)M * (size_t)p->kw0);
-    int64_t maxw = 4;
+    // an activation buffer holds one hidden layer's output either as packed bits or in a tensor-core form
+    int64_t max_row = 16;
     for (int l = 0; l < L - 1; ++l) {
         const int64_t wds = (int64_t)round_up((size_t)ceil_div(layers[l].N, 32), 4);
-        if (wds > maxw) maxw = wds;
+        const int64_t row = wds * 32;                      // the int8 form is the widest: one byte per element
+        if (row > max_row) max_row = row;
     }
-    p->off_act0 = take(sizeof(uint32_t) * (size_t)M * (size_t)maxw);
-    p->off_act1 = take(sizeof(uint32_t) * (size_t)M * (size_t)maxw);
+    p->act_bytes = (size_t)M * (size_t)max_row;
+    // each buffer holds a layer's packed bits (first quarter at most) and its tensor-core form side by side
+    p->off_act0 = take(p->act_bytes + (p->act_bytes >> 2));
+    p->off_act1 = take(p->act_bytes + (p->act_bytes >> 2));
     size_t gb = 0;
     for (int l = 0; l < L; ++l) {
         const size_t b = qnn_workspace_bytes(l == 0 ? QNN_OP_BITPLANE_GEMM : QNN_OP_XNOR_GEMM, M, layers[l].N,
-                                             layers[l].K, l == 0 ? in_bits : 1, 1, algo);
+                                             layers[l].K, l == 0 ? in_bits : 1, 1, QNN_ALGO_AUTO);
         if (b > gb) gb = b;
     }
     p->gemm_bytes = gb;
@@ -53,30 +98,64 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
 {
     if (M == 0) return QNN_OK;
     uint32_t *planes = reinterpret_cast<uint32_t *>(ws + p.off_planes);
-    uint32_t *act[2] = {reinterpret_cast<uint32_t *>(ws + p.off_act0), reinterpret_cast<uint32_t *>(ws + p.off_act1)};
+    char *act[2] = {ws + p.off_act0, ws + p.off_act1};
     void *gws = ws + p.off_gemm;
     const int64_t plane_stride = M * p.kw0;
-    if (int rc = qnn_pack_planes_u8(x_dev, M, layers[0].K, layers[0].K, in_bits, planes, p.kw0, plane_stride, nullptr, st))
-        return rc;
-    const uint32_t *cur = planes;
-    int64_t cur_ld = p.kw0;
+
+    LayerChoice choice[64];
+    QNN_REQUIRE(L <= 64, QNN_ERR_UNSUPPORTED, "mlp: at most 64 layers");
+    for (int l = 0; l < L; ++l) choice[l] = choose_layer(M, in_bits, layers, l, algo);
+
+    // what the previous layer left behind for this one
+    const uint32_t *cur_bits = nullptr; int64_t cur_ld = 0;
+    const void *cur_form = nullptr; int cur_form_kind = 0; int64_t cur_form_ld = 0;
+
     for (int l = 0; l < L; ++l) {
         const qnn_mlp_layer &ly = layers[l];
+        const LayerChoice &c = choice[l];
         const bool last = (l == L - 1);
         GemmArgs g{};
-        g.a = cur; g.lda = cur_ld; g.b = ly.w; g.ldb = ly.ldw;
-        g.ka = (l == 0) ? in_bits : 1; g.kb = 1;
-        g.a_mode = (l == 0) ? QNN_MODE_U01 : QNN_MODE_PM1; g.b_mode = QNN_MODE_PM1;
-        g.a_plane_stride = (l == 0) ? plane_stride : 0;
+        g.b = ly.w; g.ldb = ly.ldw; g.kb = 1; g.b_mode = QNN_MODE_PM1;
+        g.ka = (l == 0) ? in_bits : 1;
+        g.a_mode = (l == 0) ? QNN_MODE_U01 : QNN_MODE_PM1;
         g.M = M; g.N = ly.N; g.K = ly.K;
+        if (l == 0) {
+            // 8-bit inputs ARE the int8-form operand (Eq. 8 recomposed): no plane split, no expansion
+            const bool direct = c.form == QNN_FORM_I8 && in_bits == 8 && (ly.K % 16 == 0) && aligned(x_dev, 16);
+            if (direct) {
+                g.a_tc = x_dev; g.a_tc_form = QNN_FORM_I8; g.a_tc_ld = ly.K;
+            } else {
+                if (int rc = qnn_pack_planes_u8(x_dev, M, ly.K, ly.K, in_bits, planes, p.kw0, plane_stride, nullptr, st))
+                    return rc;
+                g.a = planes; g.lda = p.kw0; g.a_plane_stride = plane_stride;
+            }
+        } else if (cur_form != nullptr && cur_form_kind == c.form) {
+            g.a_tc = cur_form; g.a_tc_form = cur_form_kind; g.a_tc_ld = cur_form_ld;
+        } else {
+            g.a = cur_bits; g.lda = cur_ld;
+        }
+        if (is_tc(c.algo) && ly.w_tc != nullptr && ly.w_tc_form == c.form) {
+            g.b_tc = ly.w_tc; g.b_tc_form = ly.w_tc_form; g.b_tc_ld = ly.w_tc_ld;
+        }
         if (last) {
             g.epilogue = EPI_ROWMAJOR; g.out = scores_dev; g.ldo = ly.N;
         } else {
-            g.epilogue = EPI_BITS; g.thr = ly.thr; g.flip = ly.flip; g.out_bits = act[l & 1];
-            g.ld_bits = (int64_t)round_up((size_t)ceil_div(ly.N, 32), 4);
+            // hand the next layer what it consumes: its tensor-core form when this layer can write it, else packed bits
+            const LayerChoice &nx = choice[l + 1];
+            char *buf = act[l & 1];
+            const int64_t wds = (int64_t)round_up((size_t)ceil_div(ly.N, 32), 4);
+            g.epilogue = EPI_BITS; g.thr = ly.thr; g.flip = ly.flip;
+            const bool give_form = is_tc(c.algo) && is_tc(nx.algo);
+            cur_bits = nullptr; cur_form = nullptr;
+            if (give_form) {
+                g.out_form = buf + (p.act_bytes >> 2); g.out_form_kind = nx.form; g.ld_form = tc_row_bytes(wds, nx.form);
+                cur_form = g.out_form; cur_form_kind = nx.form; cur_form_ld = g.ld_form;
+            } else {
+                g.out_bits = reinterpret_cast<uint32_t *>(buf); g.ld_bits = wds;
+                cur_bits = g.out_bits; cur_ld = wds;
+            }
         }
-        if (int rc = run_gemm(g, algo, gws, p.gemm_bytes, st)) return rc;
-        if (!last) { cur = act[l & 1]; cur_ld = g.ld_bits; }
+        if (int rc = run_gemm(g, c.algo, gws, p.gemm_bytes, st)) return rc;
     }
     return QNN_OK;
 }
@@ -87,6 +166,12 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
 using namespace qnn;
 
 extern "C" {
+
+int qnn_mlp_layer_form(const qnn_mlp_layer *layers, int L, int l, int in_bits)
+{
+    if (layers == nullptr || l < 0 || l >= L || in_bits < 1 || in_bits > 8) return 0;
+    return tc_pick_form(l == 0 ? in_bits : 1, l == 0 ? QNN_MODE_U01 : QNN_MODE_PM1, 1, QNN_MODE_PM1, layers[l].K);
+}
 
 size_t qnn_mlp_workspace_bytes(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int algo, int host_io)
 {

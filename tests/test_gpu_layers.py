@@ -9,7 +9,7 @@ from util import Guarded, as_i32_words, dev, pack_bits_ref, unpack_words, words_
 
 pytestmark = pytest.mark.gpu
 
-ALGOS = [1, 2, 0]          # POPC, TC_I8, AUTO
+ALGOS = [1, 2, 4, 0]       # POPC, TC_I8, TC_FP4, AUTO
 
 
 @pytest.fixture(scope="module")
@@ -90,7 +90,7 @@ def test_cifar_conv_config_sampled(q, algo):
     assert np.all(np.abs(got) <= 2304) and np.all(got % 2 == 0)
 
 
-def _mlp_gpu(q, wl, M, algo, host=False, in_bits=8):
+def _mlp_gpu(q, wl, M, algo, host=False, in_bits=8, prepack=False):
     dims = wl.dims
     packed, ldws = [], []
     for W in wl.Ws:
@@ -101,6 +101,7 @@ def _mlp_gpu(q, wl, M, algo, host=False, in_bits=8):
         packed.append(out); ldws.append(ld)
     thr = [t.cuda() for t in wl.Ts]
     layers = q.make_mlp_layers(packed, ldws, dims[:-1], dims[1:], thr, [None] * len(thr))
+    keep = q.prepack_mlp_weights(layers, packed, in_bits) if prepack else None   # noqa: F841 (keeps the buffers alive)
     n = q.qnn_mlp_workspace_bytes(M, in_bits, layers, algo, 1 if host else 0)
     ws = torch.empty(n, dtype=torch.uint8, device="cuda")
     try:
@@ -127,6 +128,32 @@ def test_mlp_forward_small(q, M, dims, algo):
                               [t.numpy() for t in wl.Ts])
     np.testing.assert_array_equal(_mlp_gpu(q, wl, M, algo), want)
     np.testing.assert_array_equal(_mlp_gpu(q, wl, M, algo, host=True), want)
+
+
+@pytest.mark.parametrize("algo", [2, 4, 0])
+@pytest.mark.parametrize("M,dims,in_bits", [(37, (50, 40, 24, 10), 8), (300, (784, 512, 256, 10), 8), (130, (100, 300, 10), 8),
+                                            (129, (96, 160, 33), 4), (2100, (784, 1024, 1024, 10), 8)])
+def test_mlp_forward_prepacked_weights(q, M, dims, in_bits, algo):
+    """Weights rewritten once in their layer's tensor-core form (w_tc) give the same scores as per-call rewriting,
+    also when a layer is large enough for the automatic choice to take the tensor-core chain."""
+    wl = workloads.mnist_mlp(M=M, dims=dims, seed=1)
+    x = wl.X.numpy().astype(np.int32) & ((1 << in_bits) - 1)
+    want = oracle.mlp_forward(x, [oracle.sign(w.numpy()) for w in wl.Ws], [t.numpy() for t in wl.Ts])
+    np.testing.assert_array_equal(_mlp_gpu(q, wl, M, algo, in_bits=in_bits, prepack=True), want)
+    np.testing.assert_array_equal(_mlp_gpu(q, wl, M, algo, host=True, in_bits=in_bits, prepack=True), want)
+
+
+@pytest.mark.parametrize("prepack", [False, True])
+def test_mnist_mlp_config_auto_chain(q, prepack):
+    """Config 2 at full size on the automatic choice: uint8 input fed straight to the int8 product, hidden
+    activations chained in e2m1 form, packed bits only in front of the 10-unit head."""
+    wl = workloads.mnist_mlp()
+    got = _mlp_gpu(q, wl, 10000, 0, prepack=prepack)
+    rows = np.array([0, 1, 63, 64, 127, 128, 129, 255, 256, 1000, 4095, 4096, 5000, 7777, 9983, 9984, 9985, 9998, 9999])
+    want = oracle.mlp_forward(wl.X.numpy()[rows].astype(np.int32), [oracle.sign(w.numpy()) for w in wl.Ws],
+                              [t.numpy() for t in wl.Ts])
+    np.testing.assert_array_equal(got[rows], want)
+    assert q.qnn_device_status() == 0
 
 
 @pytest.mark.parametrize("algo", ALGOS)
