@@ -70,6 +70,38 @@ __global__ void __launch_bounds__(256) rescale_kernel(const int32_t *__restrict_
     }
 }
 
+// Border corrections of the implicit-GEMM convolution.  The tensor-core kernel reads out-of-image
+// taps as 0; the padding value (+1 or -1) times the weights of those taps is added back here.
+// A pixel's class says how many filter rows fall off the top / bottom and how many filter columns
+// fall off the left / right: cls = ((ty*(pad+1) + by)*(pad+1) + tx)*(pad+1) + bx.
+// corr[cls, co] = (+-1) * sum over out-of-image taps of sum_c w[co, c, tap].
+__global__ void __launch_bounds__(256) conv_border_corr_kernel(const uint32_t *__restrict__ w, int Cout, int C, int KH, int KW,
+                                                               int pad, int pad_bit, int32_t *__restrict__ corr, int classes)
+{
+    const int Cw = (C + 31) >> 5;
+    const int pc = pad + 1;
+    const int total = classes * Cout;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
+        const int co = e % Cout;
+        int cls = e / Cout;
+        const int bx = cls % pc; cls /= pc;
+        const int tx = cls % pc; cls /= pc;
+        const int by = cls % pc; cls /= pc;
+        const int ty = cls;
+        int32_t sum = 0;
+        for (int kh = 0; kh < KH; ++kh)
+            for (int kw = 0; kw < KW; ++kw) {
+                const bool oob = kh < ty || kh >= KH - by || kw < tx || kw >= KW - bx;
+                if (!oob) continue;
+                const uint32_t *wp = w + ((int64_t)co * KH * KW + kh * KW + kw) * Cw;
+                int32_t ones = 0;
+                for (int cw = 0; cw < Cw; ++cw) ones += __popc(__ldg(wp + cw));
+                sum += 2 * ones - C;
+            }
+        corr[e] = pad_bit ? sum : -sum;
+    }
+}
+
 inline int grid_for(int64_t total)
 {
     const int64_t need = ceil_div(total, 256);
@@ -122,18 +154,65 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
     const int64_t Cw = ceil_div(C, 32);
     const int64_t M = (int64_t)B * Ho * Wo;
     const int64_t kwords = (int64_t)KH * KW * Cw;
-    const size_t col_bytes = round_up(sizeof(uint32_t) * (size_t)M * (size_t)kwords, 256);
-    QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= col_bytes, QNN_ERR_WORKSPACE,
-                "qnn_binary_conv2d: workspace of at least %zu bytes (256-byte aligned) required", col_bytes);
     cudaStream_t st = as_stream(stream);
-    uint32_t *col = static_cast<uint32_t *>(ws);
+    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_FP4, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: unknown algo %d", algo);
 
     GemmArgs g{};
-    g.a = col; g.lda = kwords; g.b = w; g.ldb = kwords; g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;
+    g.b = w; g.ldb = kwords; g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;
     g.M = M; g.N = Cout; g.K = (int64_t)KH * KW * C; g.kwords = kwords;
     g.pad_period = Cw; g.pad_tail = (int)(C - 32 * (Cw - 1));
     g.epilogue = EPI_NCHW; g.out = out_nchw; g.hw = (int64_t)Ho * Wo;
     g.thr = thr; g.flip = flip; g.out_bits = out_bits; g.ld_bits = ceil_div(Cout, 32);
+
+    // ---- implicit GEMM on the tensor cores: no im2col matrix ------------------------------------
+    // Needs a stride-1 "same" filter, an image row that fits a 128-pixel tile and whole 128-byte
+    // channel blocks per pixel (256 channels as e2m1 values, 128 as int8).
+    int form = 0;
+    if (stride == 1 && KH == 2 * pad + 1 && KW == 2 * pad + 1 && pad <= 3 && W <= 128 && (int64_t)KH * KW * C < (1 << 24)) {
+        if (C % 256 == 0 && algo != QNN_ALGO_TC_I8) form = QNN_FORM_FP4;
+        else if (C % 128 == 0 && algo != QNN_ALGO_TC_FP4) form = QNN_FORM_I8;
+    }
+    if (algo == QNN_ALGO_AUTO) {
+        const int pick = qnn_select_algo(M, Cout, g.K, 1, 1, QNN_MODE_PM1, QNN_MODE_PM1);
+        if (pick != QNN_ALGO_TC_FP4 && pick != QNN_ALGO_TC_I8) form = 0;
+    } else if (algo == QNN_ALGO_POPC || algo == QNN_ALGO_B1_MMA) {
+        form = 0;
+    }
+    if (form != 0) {
+        const int64_t cbytes = tc_row_bytes(Cw, form);
+        const int classes = (pad + 1) * (pad + 1) * (pad + 1) * (pad + 1);
+        const size_t x_bytes = round_up((size_t)M * (size_t)cbytes, 256);
+        const size_t w_bytes = round_up((size_t)Cout * (size_t)tc_row_bytes(kwords, form), 256);
+        const size_t c_bytes = round_up(sizeof(int32_t) * (size_t)classes * (size_t)Cout, 256);
+        if (ws != nullptr && aligned(ws, 256) && ws_bytes >= x_bytes + w_bytes + c_bytes) {
+            uint8_t *xf = static_cast<uint8_t *>(ws);
+            uint8_t *wf = xf + x_bytes;
+            int32_t *corr = reinterpret_cast<int32_t *>(wf + w_bytes);
+            g.a_tc = xf; g.a_tc_form = form; g.a_tc_ld = cbytes;
+            g.b_tc = wf; g.b_tc_form = form; g.b_tc_ld = tc_row_bytes(kwords, form);
+            if (int rc = validate_gemm(g)) return rc;
+            if (int rc = tc_expand(x, 1, QNN_MODE_PM1, Cw, 0, M, Cw, Cw, 32, form, xf, cbytes, st)) return rc;
+            if (int rc = tc_expand(w, 1, QNN_MODE_PM1, kwords, 0, Cout, kwords, kwords, 32, form, wf, tc_row_bytes(kwords, form), st))
+                return rc;
+            conv_border_corr_kernel<<<grid_for((int64_t)classes * Cout), 256, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, classes);
+            if (int rc = check_launch("qnn_binary_conv2d border table")) return rc;
+            ConvImplicit ci{};
+            ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;
+            ci.cblocks = (int32_t)(cbytes / 128);
+            ci.corr = corr;
+            g.conv = &ci;
+            return launch_gemm_tc(g, form, nullptr, 0, st);
+        }
+        QNN_REQUIRE(algo == QNN_ALGO_AUTO, QNN_ERR_WORKSPACE,
+                    "qnn_binary_conv2d: workspace of at least %zu bytes (256-byte aligned) required", x_bytes + w_bytes + c_bytes);
+    }
+
+    // ---- packed im2col + matrix product ------------------------------------------------------------
+    const size_t col_bytes = round_up(sizeof(uint32_t) * (size_t)M * (size_t)kwords, 256);
+    QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= col_bytes, QNN_ERR_WORKSPACE,
+                "qnn_binary_conv2d: workspace of at least %zu bytes (256-byte aligned) required", col_bytes);
+    uint32_t *col = static_cast<uint32_t *>(ws);
+    g.a = col; g.lda = kwords;
     if (int rc = validate_gemm(g)) return rc;
 
     const int64_t total = M * kwords;

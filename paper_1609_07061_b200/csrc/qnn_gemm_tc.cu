@@ -790,6 +790,7 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
         p.a_tx_bytes = R * c.W * BKB;
         QNN_REQUIRE(p.num_kb == c.KH * c.KW * c.cblocks, QNN_ERR_INVALID_ARG, "tc conv: K blocks do not match the filter");
         QNN_REQUIRE(g.M == (int64_t)c.B * c.H * c.W, QNN_ERR_INVALID_ARG, "tc conv: M does not match the image geometry");
+        QNN_REQUIRE(a_ld == (int64_t)c.cblocks * BKB, QNN_ERR_INVALID_ARG, "tc conv: pixels must be whole 128-byte channel blocks apart");
         if (int rc = make_map_nhwc(&ma, a8, c.B, c.H, c.W, (int64_t)c.cblocks * BKB, R)) return rc;
     } else {
         if (int rc = make_map_2d(&ma, a8, g.M, a_row_bytes, a_ld, BM)) return rc;

@@ -54,7 +54,11 @@ def _conv_gpu(q, X, Wt, T, flip, stride, pad, pad_bit, algo, want_int=True, want
 @pytest.mark.parametrize("B,C,H,W,Co,KH,KW,stride,pad,pad_bit", [
     (2, 3, 5, 6, 4, 3, 3, 1, 1, 1), (1, 33, 4, 4, 5, 3, 3, 1, 1, 1), (2, 64, 8, 8, 70, 3, 3, 1, 1, 1),
     (2, 40, 7, 5, 33, 1, 1, 1, 0, 1), (1, 32, 9, 9, 16, 3, 3, 2, 1, 1), (1, 16, 6, 6, 8, 5, 3, 1, 2, 0),
-    (3, 256, 16, 16, 256, 3, 3, 1, 1, 1)])
+    (3, 256, 16, 16, 256, 3, 3, 1, 1, 1),
+    # geometries of the implicit tensor-core path: ragged tiles, W not dividing 128, -1 padding, 5x5, 7x7, one row per tile
+    (2, 128, 13, 12, 70, 3, 3, 1, 1, 0), (1, 256, 7, 20, 33, 5, 5, 1, 2, 1), (2, 128, 5, 128, 16, 3, 3, 1, 1, 1),
+    (1, 256, 40, 3, 8, 3, 3, 1, 1, 1), (2, 512, 9, 9, 40, 1, 1, 1, 0, 1), (1, 128, 6, 5, 9, 7, 7, 1, 3, 0),
+    (5, 256, 3, 2, 300, 3, 3, 1, 1, 1)])
 def test_conv2d(q, B, C, H, W, Co, KH, KW, stride, pad, pad_bit, algo):
     rng = np.random.default_rng(B + C + H + Co)
     X = rng.standard_normal((B, C, H, W)).astype(np.float32)
