@@ -46,6 +46,9 @@ struct TcParams {
     const int32_t *thr; const uint8_t *flip; uint32_t *out_bits; int64_t ld_bits;
     uint8_t *out_form; int64_t ld_form; int out_form_kind;
     uint32_t idesc;
+    // asynchronous (TMA) stores through the per-warp staging buffers: 0 = plain stores from registers
+    int tma_out;                     // 1: int32 row-major [M, N]; 2: int32 NCHW [img, n, pix]
+    int tma_form;                    // 1: form rows [M, bytes]
     // implicit convolution (conv != 0)
     int conv;
     int32_t cH, cW, cR, tiles_per_img, cKW, cpad, cblocks;
@@ -85,7 +88,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it > 128) __nanosleep(64);
+        if (it > 4096) __nanosleep(64);
         if ((it & 63) == 63 && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -106,6 +109,24 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
 }
+
+// bulk tensor stores (shared -> global); rows / columns past the tensor's extents are clipped by the hardware
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, int32_t y, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int32_t x, int32_t y, int32_t z, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until the shared-memory side of all but the N most recent store groups has been read
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -198,22 +219,27 @@ struct TcCfg {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int THR_WORDS = BN + 8;                             // per epilogue warp: BN thresholds + BN/32 flip words
     static constexpr int THR_BYTES = 4 * THR_WORDS * 4;
+    static constexpr int STG_WARP_BYTES = 8192;                          // epilogue staging per warp (two 4 KB int32 tiles, or one form tile)
+    static constexpr int STG_BYTES = 4 * STG_WARP_BYTES;
     static constexpr int AUX_BYTES = 256 + THR_BYTES + 1024;             // barriers, thresholds, 1024-byte alignment slack
-    static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES) / STAGE_BYTES;
-    static constexpr int STAGES = MAX_STAGES > 8 ? 8 : MAX_STAGES;
+    static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES - STG_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = MAX_STAGES > 6 ? 6 : MAX_STAGES;
     static constexpr int SCALE_COL = 2 * BN;                             // FP4: unit block scales live behind the accumulators
     static constexpr int TMEM_COLS = next_pow2_cols(2 * BN + (FORM == QNN_FORM_FP4 ? 32 : 0));
-    static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+    static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;              // 1024-byte aligned like the stages
+    static constexpr int BAR_OFFSET = STG_OFFSET + STG_BYTES;
     static constexpr int THR_OFFSET = BAR_OFFSET + 256;
     static constexpr int TOTAL = THR_OFFSET + THR_BYTES + 1024;
     static_assert(STAGES >= 3, "pipeline too shallow");
     static_assert(TMEM_COLS <= 512, "accumulators do not fit tensor memory");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile width");
+    static_assert(32 * BN <= STG_WARP_BYTES, "a warp's form tile (32 rows of at most BN bytes) must fit its staging buffer");
 };
 
 template <int FORM, int BN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const TcParams p)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_form, const TcParams p)
 {
     using S = TcCfg<FORM, BN>;
     extern __shared__ uint8_t smem_raw[];
@@ -323,10 +349,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int q = warp & 3;                                  // TMEM lane quarter this warp may read
         int32_t *thr_w = reinterpret_cast<int32_t *>(gen + S::THR_OFFSET) + q * S::THR_WORDS;   // this warp's thresholds
         uint32_t *flip_w = reinterpret_cast<uint32_t *>(thr_w + BN);                            // and flip words
+        uint8_t *stg = gen + S::STG_OFFSET + q * S::STG_WARP_BYTES;                             // this warp's staging buffer
+        const uint32_t stg_u32 = base + (uint32_t)(S::STG_OFFSET + q * S::STG_WARP_BYTES);
         const bool want_bits = p.out_bits != nullptr;
         const bool want_form = p.out_form != nullptr;
         const bool want_sign = want_bits || want_form;
+        const bool form_fp4 = p.out_form_kind == QNN_FORM_FP4;
+        const int form_row_bytes = form_fp4 ? BN / 2 : BN;       // bytes of a row of this tile in the output form
         uint32_t iter = 0;
+        uint32_t nstore = 0;                                     // int32 tiles handed to the bulk-store engine so far
         bool ok = true;
         for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
             const int32_t tm = (int32_t)(t % p.tiles_m), tn = (int32_t)(t / p.tiles_m);
@@ -340,7 +371,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 for (int c = 0; c < BN / 32; ++c) {
                     const int64_t n = ntile + c * 32 + lane;
                     const bool ncol = n < p.N;
-                    thr_w[c * 32 + lane] = ncol ? __ldg(p.thr + n) : 0;
+                    int32_t tv = ncol ? __ldg(p.thr + n) : 0;
+                    if (FORM == QNN_FORM_FP4) {
+                        // accumulators are exact integers below 2^24 held as floats: compare there.  A threshold
+                        // beyond +-2^24 decides the same way as +-2^24, which a float holds exactly.
+                        tv = tv > (1 << 24) ? (1 << 24) : (tv < -(1 << 24) ? -(1 << 24) : tv);
+                        tv = __float_as_int((float)tv);
+                    }
+                    thr_w[c * 32 + lane] = tv;
                     const bool f = (ncol && p.flip) ? (__ldg(p.flip + n) != 0) : false;
                     const uint32_t fw = __ballot_sync(0xffffffffu, f);
                     if (lane == c) flip_w[c] = fw;
@@ -350,26 +388,36 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
             // which output row this thread owns
             const int r = q * 32 + lane;
-            int64_t m;
+            int64_t m, m_warp0;                                  // this thread's row, and the row of the warp's lane 0
             bool mrow;
-            int32_t cls = 0;
+            int32_t cls = 0, c_img = 0, c_pix0 = 0;
             if (p.conv) {
-                const int32_t img = tm / p.tiles_per_img;
-                const int32_t y = (tm - img * p.tiles_per_img) * p.cR + r / p.cW;
+                c_img = tm / p.tiles_per_img;
+                const int32_t y0 = (tm - c_img * p.tiles_per_img) * p.cR;
+                const int32_t y = y0 + r / p.cW;
                 const int32_t x = r % p.cW;
                 mrow = (r < p.cR * p.cW) && (y < p.cH);
-                m = ((int64_t)img * p.cH + y) * p.cW + x;
+                m = ((int64_t)c_img * p.cH + y) * p.cW + x;
+                c_pix0 = y0 * p.cW + q * 32;
+                m_warp0 = (int64_t)c_img * p.cH * p.cW + c_pix0;
                 const int32_t pd = p.cpad, pc = pd + 1;
                 const int32_t ty = max(pd - y, 0), by = max(y + pd - (p.cH - 1), 0);
                 const int32_t tx = max(pd - x, 0), bx = max(x + pd - (p.cW - 1), 0);
                 cls = mrow ? ((ty * pc + by) * pc + tx) * pc + bx : 0;
             } else {
                 m = (int64_t)tm * BM + r;
+                m_warp0 = (int64_t)tm * BM + q * 32;
                 mrow = m < p.M;
             }
             const bool any_border = p.conv ? (__any_sync(0xffffffffu, cls != 0) != 0) : false;
             int64_t img = 0, pix = 0;
             if (p.epilogue == EPI_NCHW && mrow) { img = m / p.hw; pix = m - img * p.hw; }
+
+            // the form tile of the previous output tile must have left the staging buffer
+            if (p.tma_form) {
+                if (lane == 0) bulk_wait_read<0>();
+                __syncwarp();
+            }
 
             // the tensor-memory loads below are warp-collective: leave the loop only as a whole warp
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(as), aphase, abort_flag, 4))) { ok = false; break; }
@@ -381,71 +429,123 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (n0 >= p.N) break;                            // warp-uniform
                 uint32_t v[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * (uint32_t)BN + (uint32_t)(c * 32), v);
-                int32_t iv[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    iv[j] = (FORM == QNN_FORM_FP4) ? __float2int_rn(__uint_as_float(v[j])) : (int32_t)v[j];
+                // FP4: the fp32 accumulators are exact integers; the border corrections are added in float too
                 if (any_border && cls != 0) {
                     const int32_t *cp = p.corr + (int64_t)cls * p.N + n0;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (n0 + j < p.N) iv[j] += __ldg(cp + j);
+                    for (int j = 0; j < 32; ++j) {
+                        if (n0 + j < p.N) {
+                            const int32_t cv = __ldg(cp + j);
+                            if (FORM == QNN_FORM_FP4) v[j] = __float_as_uint(__uint_as_float(v[j]) + (float)cv);
+                            else v[j] += (uint32_t)cv;
+                        }
+                    }
                 }
-                if (p.out != nullptr && mrow) {
-                    if (p.epilogue == EPI_NCHW) {
+                int32_t iv[32];
+                if (FORM != QNN_FORM_FP4 || p.out != nullptr) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (n0 + j < p.N) p.out[(img * p.N + n0 + j) * p.hw + pix] = iv[j];
-                    } else {
-                        int32_t *dst = p.out + m * p.ldo + n0;
-                        if (n0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+                    for (int j = 0; j < 32; ++j)
+                        iv[j] = (FORM == QNN_FORM_FP4) ? __float2int_rn(__uint_as_float(v[j])) : (int32_t)v[j];
+                }
+                if (p.out != nullptr) {
+                    if (p.tma_out) {
+                        // registers -> staging tile -> one asynchronous bulk store per 32 x 32 block
+                        uint8_t *buf = stg + (nstore & 1u) * 4096u;
+                        if (lane == 0) bulk_wait_read<1>();      // the store issued two blocks ago has read this buffer
+                        __syncwarp();
+                        if (p.tma_out == 1) {
+                            // [row][32 columns], 16-byte chunks swizzled by the row (the tensor map's 128-byte swizzle)
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<int4 *>(dst + j) = make_int4(iv[j], iv[j + 1], iv[j + 2], iv[j + 3]);
+                            for (int ch = 0; ch < 8; ++ch)
+                                *reinterpret_cast<int4 *>(buf + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
+                                    make_int4(iv[4 * ch], iv[4 * ch + 1], iv[4 * ch + 2], iv[4 * ch + 3]);
                         } else {
+                            // [channel][32 pixels]: a row of 32 lanes is one 128-byte line
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) *reinterpret_cast<int32_t *>(buf + j * 128 + lane * 4) = iv[j];
+                        }
+                        fence_async_shared();
+                        __syncwarp();
+                        if (lane == 0) {
+                            const uint32_t src = stg_u32 + (nstore & 1u) * 4096u;
+                            if (p.tma_out == 1) tma_store_2d(&tmap_out, (int32_t)n0, (int32_t)m_warp0, src);
+                            else tma_store_3d(&tmap_out, c_pix0, (int32_t)n0, c_img, src);
+                            bulk_commit();
+                        }
+                        ++nstore;
+                    } else if (mrow) {
+                        if (p.epilogue == EPI_NCHW) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
-                                if (n0 + j < p.N) dst[j] = iv[j];
+                                if (n0 + j < p.N) p.out[(img * p.N + n0 + j) * p.hw + pix] = iv[j];
+                        } else {
+                            int32_t *dst = p.out + m * p.ldo + n0;
+                            if (n0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4)
+                                    *reinterpret_cast<int4 *>(dst + j) = make_int4(iv[j], iv[j + 1], iv[j + 2], iv[j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (n0 + j < p.N) dst[j] = iv[j];
+                            }
                         }
                     }
                 }
                 if (want_sign) {
                     const int4 *t4 = reinterpret_cast<const int4 *>(thr_w + c * 32);
                     uint32_t w = 0;
+                    if (FORM == QNN_FORM_FP4) {
+                        // bit j = (acc_j >= thr_j) = NOT sign(acc_j - thr_j): one subtraction and one funnel shift per
+                        // column, last column first so that column 0 lands in bit 0
 #pragma unroll
-                    for (int j4 = 0; j4 < 8; ++j4) {
-                        const int4 tt = t4[j4];                  // same address in every lane: a broadcast read
-                        w |= (uint32_t)(iv[4 * j4] >= tt.x) << (4 * j4);
-                        w |= (uint32_t)(iv[4 * j4 + 1] >= tt.y) << (4 * j4 + 1);
-                        w |= (uint32_t)(iv[4 * j4 + 2] >= tt.z) << (4 * j4 + 2);
-                        w |= (uint32_t)(iv[4 * j4 + 3] >= tt.w) << (4 * j4 + 3);
+                        for (int j4 = 7; j4 >= 0; --j4) {
+                            const int4 tt = t4[j4];              // same address in every lane: a broadcast read
+                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4 + 3]) - __int_as_float(tt.w)), w, 1);
+                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4 + 2]) - __int_as_float(tt.z)), w, 1);
+                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4 + 1]) - __int_as_float(tt.y)), w, 1);
+                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4]) - __int_as_float(tt.x)), w, 1);
+                        }
+                        w = ~w;
+                    } else {
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            const int4 tt = t4[j4];
+                            w |= (uint32_t)(iv[4 * j4] >= tt.x) << (4 * j4);
+                            w |= (uint32_t)(iv[4 * j4 + 1] >= tt.y) << (4 * j4 + 1);
+                            w |= (uint32_t)(iv[4 * j4 + 2] >= tt.z) << (4 * j4 + 2);
+                            w |= (uint32_t)(iv[4 * j4 + 3] >= tt.w) << (4 * j4 + 3);
+                        }
                     }
                     const int64_t left = p.N - n0;
                     const uint32_t nmask = left >= 32 ? 0xffffffffu : ((1u << (int)left) - 1u);
                     w = (w ^ flip_w[c]) & nmask;
-                    if (mrow) {
-                        if (want_bits) p.out_bits[m * p.ld_bits + (n0 >> 5)] = w;
-                        if (want_form) {
-                            if (p.out_form_kind == QNN_FORM_FP4) {
-                                // +1 -> e2m1 0x2, -1 -> 0xA, columns past N -> 0
-                                uint32_t o[4];
+                    if (want_bits && mrow) p.out_bits[m * p.ld_bits + (n0 >> 5)] = w;
+                    if (want_form) {
+                        if (form_fp4) {
+                            // +1 -> e2m1 0x2, -1 -> 0xA, columns past N -> 0
+                            uint32_t o[4];
 #pragma unroll
-                                for (int b = 0; b < 4; ++b) {
-                                    const uint32_t s = spread_bits_to_nibbles((w >> (8 * b)) & 0xffu);
-                                    const uint32_t vm = spread_bits_to_nibbles((nmask >> (8 * b)) & 0xffu) * 0xfu;
-                                    o[b] = (0xAAAAAAAAu ^ (s << 3)) & vm;
-                                }
-                                *reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + (n0 >> 1)) = make_uint4(o[0], o[1], o[2], o[3]);
-                            } else {
-                                // +1 -> 0x01, -1 -> 0xFF, columns past N -> 0
-                                uint32_t o[8];
+                            for (int b = 0; b < 4; ++b) o[b] = 0xAAAAAAAAu ^ (spread_bits_to_nibbles((w >> (8 * b)) & 0xffu) << 3);
+                            if (left < 32) {                     // warp-uniform: only the last chunk of a ragged N
 #pragma unroll
-                                for (int b = 0; b < 8; ++b) {
-                                    const uint32_t s = spread_bits_to_bytes((w >> (4 * b)) & 0xfu);
-                                    const uint32_t vm = spread_bits_to_bytes((nmask >> (4 * b)) & 0xfu) * 0xffu;
-                                    o[b] = (0xFFFFFFFFu ^ (s * 0xfeu)) & vm;
-                                }
-                                uint4 *dst = reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + n0);
+                                for (int b = 0; b < 4; ++b) o[b] &= spread_bits_to_nibbles((nmask >> (8 * b)) & 0xffu) * 0xfu;
+                            }
+                            const uint4 o4 = make_uint4(o[0], o[1], o[2], o[3]);
+                            if (p.tma_form) *reinterpret_cast<uint4 *>(stg + lane * form_row_bytes + c * 16) = o4;
+                            else if (mrow) *reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + (n0 >> 1)) = o4;
+                        } else {
+                            // +1 -> 0x01, -1 -> 0xFF, columns past N -> 0
+                            uint32_t o[8];
+#pragma unroll
+                            for (int b = 0; b < 8; ++b) {
+                                const uint32_t sb = spread_bits_to_bytes((w >> (4 * b)) & 0xfu);
+                                const uint32_t vm = spread_bits_to_bytes((nmask >> (4 * b)) & 0xfu) * 0xffu;
+                                o[b] = (0xFFFFFFFFu ^ (sb * 0xfeu)) & vm;
+                            }
+                            uint4 *dst = p.tma_form ? reinterpret_cast<uint4 *>(stg + lane * form_row_bytes + c * 32)
+                                                    : reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + n0);
+                            if (p.tma_form || mrow) {
                                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
                             }
@@ -456,7 +556,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
             mbar_arrive(tempty_bar(as));
+            if (p.tma_form) {
+                // this warp's 32 rows of the tile, in the output form, leave as one bulk store; columns of the
+                // tile past the operand's row length are clipped (a tile with no column there stores nothing)
+                fence_async_shared();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&tmap_form, (int32_t)(form_fp4 ? (ntile >> 1) : ntile), (int32_t)m_warp0, stg_u32);
+                    bulk_commit();
+                }
+            }
         }
+        // stores still reading shared memory must finish before the block's shared memory goes away
+        if (lane == 0) bulk_wait_all();
+        __syncwarp();
     }
 
     // ---- teardown ------------------------------------------------------------
@@ -601,18 +714,64 @@ int make_map_nhwc(CUtensorMap *map, const void *base, int B, int H, int W, int64
     return QNN_OK;
 }
 
+// destination maps of the epilogue's bulk stores
+int make_map_out(CUtensorMap *map, CUtensorMapDataType type, int rank, void *base, const cuuint64_t *dims,
+                 const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swz)
+{
+    EncodeTiledFn fn = encode_fn();
+    QNN_REQUIRE(fn != nullptr, QNN_ERR_CUDA, "tc gemm: cuTensorMapEncodeTiled is not available from this driver");
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, type, (cuuint32_t)rank, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    QNN_REQUIRE(r == CUDA_SUCCESS, QNN_ERR_CUDA, "tc gemm: cuTensorMapEncodeTiled (output) failed with code %d", (int)r);
+    return QNN_OK;
+}
+
 template <int FORM, int BN>
-int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cudaStream_t st)
+int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, const GemmArgs &g, cudaStream_t st)
 {
     using S = TcCfg<FORM, BN>;
     auto kern = gemm_tc_kernel<FORM, BN>;
+    // Outputs leave through bulk stores where their layout allows it (16-byte aligned rows); otherwise the
+    // epilogue stores from registers.
+    CUtensorMap mo = ma, mf = ma;
+    p.tma_out = 0; p.tma_form = 0;
+    const bool conv_full_tiles = p.conv && p.cR * p.cW == BM;
+    if (p.out != nullptr && aligned(p.out, 16)) {
+        // (the bulk store clips the innermost extent in 16-byte units, so N must be a whole number of them)
+        if (!p.conv && p.epilogue == EPI_ROWMAJOR && p.ldo % 4 == 0 && p.N % 4 == 0) {
+            cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
+            cuuint64_t strides[1] = {(cuuint64_t)p.ldo * 4};
+            cuuint32_t box[2] = {32, 32};
+            if (int rc = make_map_out(&mo, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, p.out, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+                return rc;
+            p.tma_out = 1;
+        } else if (conv_full_tiles && p.epilogue == EPI_NCHW && p.hw % 4 == 0 && p.hw == (int64_t)p.cH * p.cW) {
+            cuuint64_t dims[3] = {(cuuint64_t)p.hw, (cuuint64_t)p.N, (cuuint64_t)(p.M / p.hw)};
+            cuuint64_t strides[2] = {(cuuint64_t)p.hw * 4, (cuuint64_t)p.hw * 4 * (cuuint64_t)p.N};
+            cuuint32_t box[3] = {32, 32, 1};
+            if (int rc = make_map_out(&mo, CU_TENSOR_MAP_DATA_TYPE_INT32, 3, p.out, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+                return rc;
+            p.tma_out = 2;
+        }
+    }
+    if (p.out_form != nullptr && p.tma_out == 0 && (!p.conv || (conv_full_tiles && p.cH % p.cR == 0))) {
+        const int64_t row = tc_row_bytes(ceil_div(p.N, 32), p.out_form_kind);
+        cuuint64_t dims[2] = {(cuuint64_t)row, (cuuint64_t)p.M};
+        cuuint64_t strides[1] = {(cuuint64_t)p.ld_form};
+        cuuint32_t box[2] = {(cuuint32_t)(p.out_form_kind == QNN_FORM_FP4 ? BN / 2 : BN), 32};
+        if (int rc = make_map_out(&mf, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, p.out_form, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
+            return rc;
+        p.tma_form = 1;
+    }
     QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
     p.tiles_n = (int32_t)ceil_div(p.N, BN);
     p.idesc |= (uint32_t)(BN >> 3) << 17;
     const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     profile_before(st);
-    kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, p);
+    (void)g;
+    kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, mf, p);
     profile_after(st);
     return check_launch("tc gemm");
 }
@@ -621,9 +780,9 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cuda
 int pick_bn(int form, int64_t tiles_m, int64_t N)
 {
     static const int fp4_bn[] = {224, 192, 128, 64, 32};
-    static const int i8_bn[] = {256, 128, 64, 32};
-    const int *cand = form == QNN_FORM_FP4 ? fp4_bn : i8_bn;
-    const int ncand = form == QNN_FORM_FP4 ? 5 : 4;
+    (void)form;
+    const int *cand = fp4_bn;
+    const int ncand = 5;
     int best = cand[0];
     double best_cost = 1e300;
     for (int i = 0; i < ncand; ++i) {
@@ -800,18 +959,19 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
 
     if (form == QNN_FORM_FP4) {
         switch (bn) {
-            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224>(ma, mb, p, st);
-            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192>(ma, mb, p, st);
-            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128>(ma, mb, p, st);
-            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64>(ma, mb, p, st);
-            default: return launch_tc_cfg<QNN_FORM_FP4, 32>(ma, mb, p, st);
+            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224>(ma, mb, p, g, st);
+            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192>(ma, mb, p, g, st);
+            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128>(ma, mb, p, g, st);
+            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64>(ma, mb, p, g, st);
+            default: return launch_tc_cfg<QNN_FORM_FP4, 32>(ma, mb, p, g, st);
         }
     }
     switch (bn) {
-        case 256: return launch_tc_cfg<QNN_FORM_I8, 256>(ma, mb, p, st);
-        case 128: return launch_tc_cfg<QNN_FORM_I8, 128>(ma, mb, p, st);
-        case 64: return launch_tc_cfg<QNN_FORM_I8, 64>(ma, mb, p, st);
-        default: return launch_tc_cfg<QNN_FORM_I8, 32>(ma, mb, p, st);
+        case 224: return launch_tc_cfg<QNN_FORM_I8, 224>(ma, mb, p, g, st);
+        case 192: return launch_tc_cfg<QNN_FORM_I8, 192>(ma, mb, p, g, st);
+        case 128: return launch_tc_cfg<QNN_FORM_I8, 128>(ma, mb, p, g, st);
+        case 64: return launch_tc_cfg<QNN_FORM_I8, 64>(ma, mb, p, g, st);
+        default: return launch_tc_cfg<QNN_FORM_I8, 32>(ma, mb, p, g, st);
     }
 }
 
