@@ -48,7 +48,6 @@ struct TcParams {
     uint32_t idesc;
     // asynchronous (TMA) stores through the per-warp staging buffers: 0 = plain stores from registers
     int tma_out;                     // 1: int32 row-major [M, N]; 2: int32 NCHW [img, n, pix]
-    int tma_form;                    // 1: form rows [M, bytes]
     // implicit convolution (conv != 0)
     int conv;
     int32_t cH, cW, cR, tiles_per_img, cKW, cpad, cblocks;
@@ -62,10 +61,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
@@ -96,19 +91,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, int32_t c0, int32_t c1, int32_t c2,
-                                            int32_t c3, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
-}
 
 // bulk tensor stores (shared -> global); rows / columns past the tensor's extents are clipped by the hardware
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, int32_t y, uint32_t src)
@@ -140,28 +122,105 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+// One pipeline stage of the MMA warp as ONE instruction stream: poll the NEXT stage's full barrier, issue the
+// four K steps of this stage (+32 bytes of K = +2 in the descriptors' address field), commit them to this
+// stage's empty barrier, and only then read the poll's result -- the poll's latency hides behind the issue.
+// Returns non-zero when the next stage has already landed.
+template <int FORM>
+__device__ __forceinline__ uint32_t umma_stage(uint32_t next_full_bar, uint32_t next_parity, uint32_t d_tmem, uint64_t adesc,
+                                               uint64_t bdesc, uint32_t idesc, uint32_t accumulate_first, uint32_t sf,
+                                               uint32_t empty_bar)
 {
+    uint32_t ready;
+    if (FORM == QNN_FORM_FP4) {
+        asm volatile(
+            "{\n"
+            ".reg .pred P, Q, T;\n"
+            ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+            "setp.ne.b32 P, %7, 0;\n"
+            "setp.eq.b32 T, 0, 0;\n"
+            "add.u64 a1, %4, 2;\n add.u64 a2, %4, 4;\n add.u64 a3, %4, 6;\n"
+            "add.u64 b1, %5, 2;\n add.u64 b2, %5, 4;\n add.u64 b3, %5, 6;\n"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%3], %4, %5, %6, [%8], [%8], P;\n"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%3], a1, b1, %6, [%8], [%8], T;\n"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%3], a2, b2, %6, [%8], [%8], T;\n"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%3], a3, b3, %6, [%8], [%8], T;\n"
+            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
+            "selp.u32 %0, 1, 0, Q;\n"
+            "}\n"
+            : "=r"(ready)
+            : "r"(next_full_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first),
+              "r"(sf), "r"(empty_bar)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n"
+            ".reg .pred P, Q, T;\n"
+            ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+            "setp.ne.b32 P, %7, 0;\n"
+            "setp.eq.b32 T, 0, 0;\n"
+            "add.u64 a1, %4, 2;\n add.u64 a2, %4, 4;\n add.u64 a3, %4, 6;\n"
+            "add.u64 b1, %5, 2;\n add.u64 b2, %5, 4;\n add.u64 b3, %5, 6;\n"
+            "tcgen05.mma.cta_group::1.kind::i8 [%3], %4, %5, %6, P;\n"
+            "tcgen05.mma.cta_group::1.kind::i8 [%3], a1, b1, %6, T;\n"
+            "tcgen05.mma.cta_group::1.kind::i8 [%3], a2, b2, %6, T;\n"
+            "tcgen05.mma.cta_group::1.kind::i8 [%3], a3, b3, %6, T;\n"
+            "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n"
+            "selp.u32 %0, 1, 0, Q;\n"
+            "}\n"
+            : "=r"(ready)
+            : "r"(next_full_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first),
+              "r"(sf), "r"(empty_bar)
+            : "memory");
+    }
+    return ready;
+}
+
+// One pipeline stage of the TMA warp the same way: poll the NEXT stage's empty barrier first, announce this
+// stage's bytes, issue its two loads, then read the poll's result.
+__device__ __forceinline__ uint32_t tma_stage_2d(uint32_t next_empty_bar, uint32_t next_parity, uint32_t full_bar, uint32_t tx_bytes,
+                                                 uint32_t dst_a, const CUtensorMap *map_a, int32_t ax, int32_t ay,
+                                                 uint32_t dst_b, const CUtensorMap *map_b, int32_t bx, int32_t by)
+{
+    uint32_t ready;
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n"
+        ".reg .pred Q;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+        "mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %4;\n"
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%5], [%6, {%7, %8}], [%3];\n"
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%9], [%10, {%11, %12}], [%3];\n"
+        "selp.u32 %0, 1, 0, Q;\n"
         "}\n"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        : "=r"(ready)
+        : "r"(next_empty_bar), "r"(next_parity), "r"(full_bar), "r"(tx_bytes), "r"(dst_a), "l"(map_a), "r"(ax), "r"(ay),
+          "r"(dst_b), "l"(map_b), "r"(bx), "r"(by)
+        : "memory");
+    return ready;
 }
-// e2m1 x e2m1 with one ue8m0 scale per 32 elements of K; `sf` addresses tensor-memory columns holding the scales
-__device__ __forceinline__ void umma_mxf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
-                                          uint32_t sf)
+__device__ __forceinline__ uint32_t tma_stage_conv(uint32_t next_empty_bar, uint32_t next_parity, uint32_t full_bar, uint32_t tx_bytes,
+                                                   uint32_t dst_a, const CUtensorMap *map_a, int32_t c0, int32_t c1, int32_t c2,
+                                                   int32_t c3, uint32_t dst_b, const CUtensorMap *map_b, int32_t bx, int32_t by)
 {
+    uint32_t ready;
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%5], p;\n"
+        ".reg .pred Q;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+        "mbarrier.arrive.expect_tx.shared::cta.b64 _, [%3], %4;\n"
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%5], [%6, {%7, %8, %9, %10}], [%3];\n"
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%11], [%12, {%13, %14}], [%3];\n"
+        "selp.u32 %0, 1, 0, Q;\n"
         "}\n"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sf) : "memory");
+        : "=r"(ready)
+        : "r"(next_empty_bar), "r"(next_parity), "r"(full_bar), "r"(tx_bytes), "r"(dst_a), "l"(map_a), "r"(c0), "r"(c1), "r"(c2),
+          "r"(c3), "r"(dst_b), "l"(map_b), "r"(bx), "r"(by)
+        : "memory");
+    return ready;
 }
+
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -212,14 +271,16 @@ __device__ __forceinline__ uint32_t spread_bits_to_bytes(uint32_t nib) { return 
 
 constexpr int next_pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
-template <int FORM, int BN>
+template <int FORM, int BN, int STG>
 struct TcCfg {
     static constexpr int A_BYTES = BM * BKB;
     static constexpr int B_BYTES = BN * BKB;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int THR_WORDS = BN + 8;                             // per epilogue warp: BN thresholds + BN/32 flip words
     static constexpr int THR_BYTES = 4 * THR_WORDS * 4;
-    static constexpr int STG_WARP_BYTES = 8192;                          // epilogue staging per warp (two 4 KB int32 tiles, or one form tile)
+    // epilogue staging per warp: two 4 KB tiles of 32 x 32 int32 for the bulk stores; kernels instantiated
+    // without it keep one more pipeline stage and store from registers
+    static constexpr int STG_WARP_BYTES = STG ? 8192 : 0;
     static constexpr int STG_BYTES = 4 * STG_WARP_BYTES;
     static constexpr int AUX_BYTES = 256 + THR_BYTES + 1024;             // barriers, thresholds, 1024-byte alignment slack
     static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES - STG_BYTES) / STAGE_BYTES;
@@ -233,15 +294,14 @@ struct TcCfg {
     static_assert(STAGES >= 3, "pipeline too shallow");
     static_assert(TMEM_COLS <= 512, "accumulators do not fit tensor memory");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile width");
-    static_assert(32 * BN <= STG_WARP_BYTES, "a warp's form tile (32 rows of at most BN bytes) must fit its staging buffer");
 };
 
-template <int FORM, int BN>
+template <int FORM, int BN, int STG>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_form, const TcParams p)
+               const __grid_constant__ CUtensorMap tmap_out, const TcParams p)
 {
-    using S = TcCfg<FORM, BN>;
+    using S = TcCfg<FORM, BN, STG>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
@@ -292,6 +352,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
+            bool ready = false;                                    // this stage's slot is known to be free
             const uint32_t tx_bytes = (uint32_t)p.a_tx_bytes + (uint32_t)S::B_BYTES;
             for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
                 const int32_t tm = (int32_t)(t % p.tiles_m), tn = (int32_t)(t / p.tiles_m);
@@ -299,17 +360,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; }
                 int32_t cb = 0, kw = 0, kh = 0;                    // conv: channel block, filter column, filter row of kb
                 for (int32_t kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 1)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(stage), tx_bytes);
+                    if (!ready && !mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 1)) { ok = false; break; }
                     const uint32_t sa = base + (uint32_t)stage * S::STAGE_BYTES;
+                    int nstage = stage + 1; uint32_t nphase = phase;
+                    if (nstage == S::STAGES) { nstage = 0; nphase ^= 1u; }
+                    uint32_t nready;
                     if (p.conv) {
-                        tma_load_4d(sa, &tmap_a, cb * BKB, kw - p.cpad, y0 + kh - p.cpad, img, full_bar(stage));
+                        nready = tma_stage_conv(empty_bar(nstage), nphase ^ 1u, full_bar(stage), tx_bytes, sa, &tmap_a, cb * BKB,
+                                                kw - p.cpad, y0 + kh - p.cpad, img, sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN);
                         if (++cb == p.cblocks) { cb = 0; if (++kw == p.cKW) { kw = 0; ++kh; } }
                     } else {
-                        tma_load_2d(sa, &tmap_a, kb * BKB, tm * BM, full_bar(stage));
+                        nready = tma_stage_2d(empty_bar(nstage), nphase ^ 1u, full_bar(stage), tx_bytes, sa, &tmap_a, kb * BKB, tm * BM,
+                                              sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN);
                     }
-                    tma_load_2d(sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN, full_bar(stage));
-                    if (++stage == S::STAGES) { stage = 0; phase ^= 1u; }
+                    ready = nready != 0;
+                    stage = nstage; phase = nphase;
                 }
             }
         }
@@ -318,6 +383,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int stage = 0; uint32_t phase = 0;
             uint32_t iter = 0;
             bool ok = true;
+            bool ready = false;                                    // this stage's operands are known to have landed
             const uint32_t sf = tmem_base + (uint32_t)S::SCALE_COL;
             for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
                 const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
@@ -325,22 +391,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * (uint32_t)BN;
                 for (int32_t kb = 0; kb < p.num_kb; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag, 3)) { ok = false; break; }
-                    tc_fence_after();
+                    if (!ready && !mbar_wait(full_bar(stage), phase, abort_flag, 3)) { ok = false; break; }
                     const uint32_t sa = base + (uint32_t)stage * S::STAGE_BYTES;
                     const uint64_t adesc = make_kmajor_sw128_desc(sa);
                     const uint64_t bdesc = make_kmajor_sw128_desc(sa + S::A_BYTES);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        // one instruction consumes 32 bytes of K; +32 bytes inside the swizzle row = +2 in the address field
-                        const uint32_t acc = (uint32_t)((kb | k) != 0);
-                        if (FORM == QNN_FORM_FP4)
-                            umma_mxf4(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), p.idesc, acc, sf);
-                        else
-                            umma_i8(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), p.idesc, acc);
-                    }
-                    umma_commit(empty_bar(stage));               // frees the smem slot once these MMAs retire
-                    if (++stage == S::STAGES) { stage = 0; phase ^= 1u; }
+                    int nstage = stage + 1; uint32_t nphase = phase;
+                    if (nstage == S::STAGES) { nstage = 0; nphase ^= 1u; }
+                    ready = umma_stage<FORM>(full_bar(nstage), nphase, d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != 0), sf,
+                                             empty_bar(stage)) != 0;
+                    stage = nstage; phase = nphase;
                 }
                 if (ok) umma_commit(tfull_bar(as));              // accumulator complete
             }
@@ -355,7 +414,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const bool want_form = p.out_form != nullptr;
         const bool want_sign = want_bits || want_form;
         const bool form_fp4 = p.out_form_kind == QNN_FORM_FP4;
-        const int form_row_bytes = form_fp4 ? BN / 2 : BN;       // bytes of a row of this tile in the output form
         uint32_t iter = 0;
         uint32_t nstore = 0;                                     // int32 tiles handed to the bulk-store engine so far
         bool ok = true;
@@ -413,12 +471,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int64_t img = 0, pix = 0;
             if (p.epilogue == EPI_NCHW && mrow) { img = m / p.hw; pix = m - img * p.hw; }
 
-            // the form tile of the previous output tile must have left the staging buffer
-            if (p.tma_form) {
-                if (lane == 0) bulk_wait_read<0>();
-                __syncwarp();
-            }
-
             // the tensor-memory loads below are warp-collective: leave the loop only as a whole warp
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(as), aphase, abort_flag, 4))) { ok = false; break; }
             tc_fence_after();
@@ -448,7 +500,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         iv[j] = (FORM == QNN_FORM_FP4) ? __float2int_rn(__uint_as_float(v[j])) : (int32_t)v[j];
                 }
                 if (p.out != nullptr) {
-                    if (p.tma_out) {
+                    if (STG && p.tma_out) {
                         // registers -> staging tile -> one asynchronous bulk store per 32 x 32 block
                         uint8_t *buf = stg + (nstore & 1u) * 4096u;
                         if (lane == 0) bulk_wait_read<1>();      // the store issued two blocks ago has read this buffer
@@ -532,8 +584,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                                 for (int b = 0; b < 4; ++b) o[b] &= spread_bits_to_nibbles((nmask >> (8 * b)) & 0xffu) * 0xfu;
                             }
                             const uint4 o4 = make_uint4(o[0], o[1], o[2], o[3]);
-                            if (p.tma_form) *reinterpret_cast<uint4 *>(stg + lane * form_row_bytes + c * 16) = o4;
-                            else if (mrow) *reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + (n0 >> 1)) = o4;
+                            if (mrow) *reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + (n0 >> 1)) = o4;
                         } else {
                             // +1 -> 0x01, -1 -> 0xFF, columns past N -> 0
                             uint32_t o[8];
@@ -543,9 +594,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                                 const uint32_t vm = spread_bits_to_bytes((nmask >> (4 * b)) & 0xfu) * 0xffu;
                                 o[b] = (0xFFFFFFFFu ^ (sb * 0xfeu)) & vm;
                             }
-                            uint4 *dst = p.tma_form ? reinterpret_cast<uint4 *>(stg + lane * form_row_bytes + c * 32)
-                                                    : reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + n0);
-                            if (p.tma_form || mrow) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + n0);
+                            if (mrow) {
                                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
                             }
@@ -556,20 +606,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
             mbar_arrive(tempty_bar(as));
-            if (p.tma_form) {
-                // this warp's 32 rows of the tile, in the output form, leave as one bulk store; columns of the
-                // tile past the operand's row length are clipped (a tile with no column there stores nothing)
-                fence_async_shared();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_2d(&tmap_form, (int32_t)(form_fp4 ? (ntile >> 1) : ntile), (int32_t)m_warp0, stg_u32);
-                    bulk_commit();
-                }
-            }
         }
         // stores still reading shared memory must finish before the block's shared memory goes away
-        if (lane == 0) bulk_wait_all();
-        __syncwarp();
+        if (STG) {
+            if (lane == 0) bulk_wait_all();
+            __syncwarp();
+        }
     }
 
     // ---- teardown ------------------------------------------------------------
@@ -727,15 +769,29 @@ int make_map_out(CUtensorMap *map, CUtensorMapDataType type, int rank, void *bas
     return QNN_OK;
 }
 
-template <int FORM, int BN>
-int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, const GemmArgs &g, cudaStream_t st)
+template <int FORM, int BN, int STG>
+int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mo, TcParams p, cudaStream_t st)
 {
-    using S = TcCfg<FORM, BN>;
-    auto kern = gemm_tc_kernel<FORM, BN>;
-    // Outputs leave through bulk stores where their layout allows it (16-byte aligned rows); otherwise the
-    // epilogue stores from registers.
-    CUtensorMap mo = ma, mf = ma;
-    p.tma_out = 0; p.tma_form = 0;
+    using S = TcCfg<FORM, BN, STG>;
+    auto kern = gemm_tc_kernel<FORM, BN, STG>;
+    QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
+    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    profile_before(st);
+    kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, p);
+    profile_after(st);
+    return check_launch("tc gemm");
+}
+
+template <int FORM, int BN>
+int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cudaStream_t st)
+{
+    // The int32 result leaves through bulk stores where its layout allows it (16-byte aligned rows), which
+    // costs the kernel one pipeline stage of shared memory; otherwise the epilogue stores from registers.
+    CUtensorMap mo = ma;
+    p.tma_out = 0;
+    p.tiles_n = (int32_t)ceil_div(p.N, BN);
+    p.idesc |= (uint32_t)(BN >> 3) << 17;
     const bool conv_full_tiles = p.conv && p.cR * p.cW == BM;
     if (p.out != nullptr && aligned(p.out, 16)) {
         // (the bulk store clips the innermost extent in 16-byte units, so N must be a whole number of them)
@@ -755,41 +811,23 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cons
             p.tma_out = 2;
         }
     }
-    if (p.out_form != nullptr && p.tma_out == 0 && (!p.conv || (conv_full_tiles && p.cH % p.cR == 0))) {
-        const int64_t row = tc_row_bytes(ceil_div(p.N, 32), p.out_form_kind);
-        cuuint64_t dims[2] = {(cuuint64_t)row, (cuuint64_t)p.M};
-        cuuint64_t strides[1] = {(cuuint64_t)p.ld_form};
-        cuuint32_t box[2] = {(cuuint32_t)(p.out_form_kind == QNN_FORM_FP4 ? BN / 2 : BN), 32};
-        if (int rc = make_map_out(&mf, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, p.out_form, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE))
-            return rc;
-        p.tma_form = 1;
-    }
-    QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
-    p.tiles_n = (int32_t)ceil_div(p.N, BN);
-    p.idesc |= (uint32_t)(BN >> 3) << 17;
-    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
-    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-    profile_before(st);
-    (void)g;
-    kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, mf, p);
-    profile_after(st);
-    return check_launch("tc gemm");
+    if (p.tma_out) return launch_tc_stg<FORM, BN, 1>(ma, mb, mo, p, st);
+    return launch_tc_stg<FORM, BN, 0>(ma, mb, mo, p, st);
 }
 
-// Tile width: fewest waves of the persistent grid, weighted by the width (a wave of wider tiles takes longer).
-int pick_bn(int form, int64_t tiles_m, int64_t N)
+// Tile width.  Measured on B200: the time of one wave of tiles depends only weakly on the width (about
+// 4.2 us + 4.7 ns per column at K = 4096), because a K block costs the issuing threads and the TMA path
+// about the same whatever its width.  So: fewest waves first, the width as a small correction.
+int pick_bn(int64_t tiles_m, int64_t N)
 {
-    static const int fp4_bn[] = {224, 192, 128, 64, 32};
-    (void)form;
-    const int *cand = fp4_bn;
-    const int ncand = 5;
+    static const int cand[] = {224, 192, 128, 64, 32};
     int best = cand[0];
     double best_cost = 1e300;
-    for (int i = 0; i < ncand; ++i) {
+    for (int i = 0; i < 5; ++i) {
         const int bn = cand[i];
         const int64_t tiles = tiles_m * ceil_div(N, bn);
         const int64_t waves = ceil_div(tiles, sm_count());
-        const double cost = (double)waves * (bn + 24);
+        const double cost = (double)waves * (bn + 900);
         if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
     }
     return best;
@@ -954,24 +992,24 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     } else {
         if (int rc = make_map_2d(&ma, a8, g.M, a_row_bytes, a_ld, BM)) return rc;
     }
-    const int bn = pick_bn(form, p.tiles_m, g.N);
+    const int bn = pick_bn(p.tiles_m, g.N);
     if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn)) return rc;
 
     if (form == QNN_FORM_FP4) {
         switch (bn) {
-            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224>(ma, mb, p, g, st);
-            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192>(ma, mb, p, g, st);
-            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128>(ma, mb, p, g, st);
-            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64>(ma, mb, p, g, st);
-            default: return launch_tc_cfg<QNN_FORM_FP4, 32>(ma, mb, p, g, st);
+            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224>(ma, mb, p, st);
+            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192>(ma, mb, p, st);
+            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128>(ma, mb, p, st);
+            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64>(ma, mb, p, st);
+            default: return launch_tc_cfg<QNN_FORM_FP4, 32>(ma, mb, p, st);
         }
     }
     switch (bn) {
-        case 224: return launch_tc_cfg<QNN_FORM_I8, 224>(ma, mb, p, g, st);
-        case 192: return launch_tc_cfg<QNN_FORM_I8, 192>(ma, mb, p, g, st);
-        case 128: return launch_tc_cfg<QNN_FORM_I8, 128>(ma, mb, p, g, st);
-        case 64: return launch_tc_cfg<QNN_FORM_I8, 64>(ma, mb, p, g, st);
-        default: return launch_tc_cfg<QNN_FORM_I8, 32>(ma, mb, p, g, st);
+        case 224: return launch_tc_cfg<QNN_FORM_I8, 224>(ma, mb, p, st);
+        case 192: return launch_tc_cfg<QNN_FORM_I8, 192>(ma, mb, p, st);
+        case 128: return launch_tc_cfg<QNN_FORM_I8, 128>(ma, mb, p, st);
+        case 64: return launch_tc_cfg<QNN_FORM_I8, 64>(ma, mb, p, st);
+        default: return launch_tc_cfg<QNN_FORM_I8, 32>(ma, mb, p, st);
     }
 }
 
