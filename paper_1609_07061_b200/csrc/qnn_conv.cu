@@ -74,16 +74,18 @@ __global__ void __launch_bounds__(256) rescale_kernel(const int32_t *__restrict_
 // taps as 0; the padding value (+1 or -1) times the weights of those taps is added back here.
 // A pixel's class says how many filter rows fall off the top / bottom and how many filter columns
 // fall off the left / right: cls = ((ty*(pad+1) + by)*(pad+1) + tx)*(pad+1) + bx.
-// corr[cls, co] = (+-1) * sum over out-of-image taps of sum_c w[co, c, tap].
+// corr[cls, co] = (+-1) * sum over out-of-image taps of sum_c w[co, c, tap]; rows are ld = Cout rounded up to 32
+// long, the pad columns zero.
 __global__ void __launch_bounds__(256) conv_border_corr_kernel(const uint32_t *__restrict__ w, int Cout, int C, int KH, int KW,
-                                                               int pad, int pad_bit, int32_t *__restrict__ corr, int classes)
+                                                               int pad, int pad_bit, int32_t *__restrict__ corr, int classes, int ld)
 {
     const int Cw = (C + 31) >> 5;
     const int pc = pad + 1;
-    const int total = classes * Cout;
+    const int total = classes * ld;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
-        const int co = e % Cout;
-        int cls = e / Cout;
+        const int co = e % ld;
+        int cls = e / ld;
+        if (co >= Cout) { corr[e] = 0; continue; }
         const int bx = cls % pc; cls /= pc;
         const int tx = cls % pc; cls /= pc;
         const int by = cls % pc; cls /= pc;
@@ -183,7 +185,8 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
         const int classes = (pad + 1) * (pad + 1) * (pad + 1) * (pad + 1);
         const size_t x_bytes = round_up((size_t)M * (size_t)cbytes, 256);
         const size_t w_bytes = round_up((size_t)Cout * (size_t)tc_row_bytes(kwords, form), 256);
-        const size_t c_bytes = round_up(sizeof(int32_t) * (size_t)classes * (size_t)Cout, 256);
+        const int corr_ld = (int)round_up((size_t)Cout, 32);
+        const size_t c_bytes = round_up(sizeof(int32_t) * (size_t)classes * (size_t)corr_ld, 256);
         if (ws != nullptr && aligned(ws, 256) && ws_bytes >= x_bytes + w_bytes + c_bytes) {
             uint8_t *xf = static_cast<uint8_t *>(ws);
             uint8_t *wf = xf + x_bytes;
@@ -194,7 +197,8 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
             if (int rc = tc_expand(x, 1, QNN_MODE_PM1, Cw, 0, M, Cw, Cw, 32, form, xf, cbytes, st)) return rc;
             if (int rc = tc_expand(w, 1, QNN_MODE_PM1, kwords, 0, Cout, kwords, kwords, 32, form, wf, tc_row_bytes(kwords, form), st))
                 return rc;
-            conv_border_corr_kernel<<<grid_for((int64_t)classes * Cout), 256, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, classes);
+            conv_border_corr_kernel<<<grid_for((int64_t)classes * corr_ld), 256, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, classes,
+                                                                                           corr_ld);
             if (int rc = check_launch("qnn_binary_conv2d border table")) return rc;
             ConvImplicit ci{};
             ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;

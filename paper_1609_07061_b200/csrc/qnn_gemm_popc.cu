@@ -235,40 +235,56 @@ __global__ void __launch_bounds__(256) gemm_popc_skinny_kernel(const uint32_t *_
     const int64_t warp0 = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const bool vec = ((lda & 3) == 0) && ((reinterpret_cast<uintptr_t>(a) & 15) == 0);
-    for (int64_t m = warp0; m < M; m += nwarps) {
-        int32_t acc[SKINNY_N];
+    // two rows per pass: their loads are in flight together
+    for (int64_t m = warp0; m < M; m += 2 * nwarps) {
+        const int64_t m2 = m + nwarps;
+        const bool has2 = m2 < M;
+        int32_t acc[SKINNY_N], acc2[SKINNY_N];
 #pragma unroll
-        for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0;
+        for (int n = 0; n < SKINNY_N; ++n) { acc[n] = 0; acc2[n] = 0; }
         const uint32_t *arow = a + m * lda;
+        const uint32_t *arow2 = a + (has2 ? m2 : m) * lda;
         for (int64_t k = (int64_t)lane * 4; k < kwords; k += 128) {
-            uint4 av;
+            uint4 av, aw;
             if (vec && k + 4 <= kwords) {
                 av = __ldcs(reinterpret_cast<const uint4 *>(arow + k));
+                aw = __ldcs(reinterpret_cast<const uint4 *>(arow2 + k));
             } else {
                 av.x = arow[k];
                 av.y = k + 1 < kwords ? arow[k + 1] : 0u;
                 av.z = k + 2 < kwords ? arow[k + 2] : 0u;
                 av.w = k + 3 < kwords ? arow[k + 3] : 0u;
+                aw.x = arow2[k];
+                aw.y = k + 1 < kwords ? arow2[k + 1] : 0u;
+                aw.z = k + 2 < kwords ? arow2[k + 2] : 0u;
+                aw.w = k + 3 < kwords ? arow2[k + 3] : 0u;
             }
 #pragma unroll
             for (int n = 0; n < SKINNY_N; ++n) {
                 if (n < N) {
                     const uint4 bv = *reinterpret_cast<const uint4 *>(bs + n * kw4 + k);
                     acc[n] += __popc(av.x ^ bv.x) + __popc(av.y ^ bv.y) + __popc(av.z ^ bv.z) + __popc(av.w ^ bv.w);
+                    acc2[n] += __popc(aw.x ^ bv.x) + __popc(aw.y ^ bv.y) + __popc(aw.z ^ bv.z) + __popc(aw.w ^ bv.w);
                 }
             }
         }
-        int32_t mine = 0;
+        int32_t mine = 0, mine2 = 0;
 #pragma unroll
         for (int n = 0; n < SKINNY_N; ++n) {
             if (n < N) {
-                int32_t v = acc[n];
+                int32_t v = acc[n], v2 = acc2[n];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == n) mine = v;
+                for (int o = 16; o > 0; o >>= 1) {
+                    v += __shfl_xor_sync(0xffffffffu, v, o);
+                    v2 += __shfl_xor_sync(0xffffffffu, v2, o);
+                }
+                if (lane == n) { mine = v; mine2 = v2; }
             }
         }
-        if (lane < N) out[m * ldo + lane] = K - 2 * mine;
+        if (lane < N) {
+            out[m * ldo + lane] = K - 2 * mine;
+            if (has2) out[m2 * ldo + lane] = K - 2 * mine2;
+        }
     }
 }
 
@@ -279,8 +295,9 @@ int launch_skinny(const PopcParams &P, cudaStream_t st)
     const size_t smem = sizeof(uint32_t) * (size_t)g.N * (size_t)kw4;
     auto kern = gemm_popc_skinny_kernel;
     if (smem > 48 * 1024) QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const int64_t need = ceil_div(g.M, 8);
-    const int64_t cap = (int64_t)sm_count() * 8;
+    // few resident blocks per SM, several rows per warp: the copy of B into shared memory is paid once per block
+    const int64_t need = ceil_div(g.M, 32);
+    const int64_t cap = (int64_t)sm_count() * 2;
     const int blocks = (int)(need < cap ? need : cap);
     profile_before(st);
     kern<<<blocks, 256, smem, st>>>(g.a, g.lda, g.b, g.ldb, g.M, (int)g.N, P.kwords, P.kll, g.out, g.ldo);

@@ -30,7 +30,8 @@ namespace {
 
 constexpr int BM = 128;              // rows of A per tile (UMMA M)
 constexpr int BKB = 128;             // bytes of K per pipeline stage = one 128-byte swizzle row
-constexpr int TC_THREADS = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int EPI_GROUPS = 2;        // epilogue warps per quarter of the accumulator's lanes
+constexpr int TC_THREADS = 64 + 128 * EPI_GROUPS;   // warp 0: TMA, warp 1: MMA + TMEM owner, the rest: epilogue
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int SMEM_LIMIT = 232448;   // 227 KB of dynamic shared memory per CTA
 
@@ -46,12 +47,14 @@ struct TcParams {
     const int32_t *thr; const uint8_t *flip; uint32_t *out_bits; int64_t ld_bits;
     uint8_t *out_form; int64_t ld_form; int out_form_kind;
     uint32_t idesc;
+    int32_t thr_clamp;               // int8 form: max |sum| + 1 when that is below 2^30 (else 0: plain compares)
     // asynchronous (TMA) stores through the per-warp staging buffers: 0 = plain stores from registers
     int tma_out;                     // 1: int32 row-major [M, N]; 2: int32 NCHW [img, n, pix]
     // implicit convolution (conv != 0)
     int conv;
     int32_t cH, cW, cR, tiles_per_img, cKW, cpad, cblocks;
     const int32_t *corr;
+    int64_t corr_ld;                 // row length of the correction table: N rounded up to 32, pad zero
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -276,12 +279,13 @@ struct TcCfg {
     static constexpr int A_BYTES = BM * BKB;
     static constexpr int B_BYTES = BN * BKB;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int THR_WORDS = BN + 8;                             // per epilogue warp: BN thresholds + BN/32 flip words
-    static constexpr int THR_BYTES = 4 * THR_WORDS * 4;
-    // epilogue staging per warp: two 4 KB tiles of 32 x 32 int32 for the bulk stores; kernels instantiated
+    static constexpr int CPW = (BN / 32 + EPI_GROUPS - 1) / EPI_GROUPS;  // 32-column chunks per epilogue warp
+    static constexpr int THR_WORDS = CPW * 32 + 8;                       // per epilogue warp: its thresholds + flip words
+    static constexpr int THR_BYTES = 4 * EPI_GROUPS * THR_WORDS * 4;
+    // epilogue staging per warp: one 4 KB tile of 32 x 32 int32 for the bulk stores; kernels instantiated
     // without it keep one more pipeline stage and store from registers
-    static constexpr int STG_WARP_BYTES = STG ? 8192 : 0;
-    static constexpr int STG_BYTES = 4 * STG_WARP_BYTES;
+    static constexpr int STG_WARP_BYTES = STG ? 4096 : 0;
+    static constexpr int STG_BYTES = 4 * EPI_GROUPS * STG_WARP_BYTES;
     static constexpr int AUX_BYTES = 256 + THR_BYTES + 1024;             // barriers, thresholds, 1024-byte alignment slack
     static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES - STG_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = MAX_STAGES > 6 ? 6 : MAX_STAGES;
@@ -320,7 +324,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128 * EPI_GROUPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -334,7 +338,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (FORM == QNN_FORM_FP4) {
         // Unit scale factors (ue8m0 exponent 127 = 2^0) in 32 columns of every lane: whatever layout the
         // instruction reads its per-block scales in, every scale it finds is 1.0.
-        if (warp >= 2) {
+        if (warp >= 2 && warp < 6) {
             const int q = warp & 3;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -346,7 +350,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         tc_fence_after();
     }
 
-    const int64_t num_tiles = (int64_t)p.tiles_m * p.tiles_n;
+    const uint32_t tiles_m = (uint32_t)p.tiles_m;
+    const uint32_t num_tiles = tiles_m * (uint32_t)p.tiles_n;          // below 2^31 (checked on the host)
 
     if (warp == 0) {
         if (lane == 0) {
@@ -354,8 +359,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             bool ok = true;
             bool ready = false;                                    // this stage's slot is known to be free
             const uint32_t tx_bytes = (uint32_t)p.a_tx_bytes + (uint32_t)S::B_BYTES;
-            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-                const int32_t tm = (int32_t)(t % p.tiles_m), tn = (int32_t)(t / p.tiles_m);
+            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
                 int32_t img = 0, y0 = 0;
                 if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; }
                 int32_t cb = 0, kw = 0, kh = 0;                    // conv: channel block, filter column, filter row of kb
@@ -385,7 +390,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             bool ok = true;
             bool ready = false;                                    // this stage's operands are known to have landed
             const uint32_t sf = tmem_base + (uint32_t)S::SCALE_COL;
-            for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
+            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
                 const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tc_fence_after();
@@ -405,43 +410,70 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
         }
     } else {
+        // EPI_GROUPS warps share each quarter of the accumulator's lanes; group g drains the 32-column chunks
+        // g, g + EPI_GROUPS, ...  One warp alone on a scheduler cannot hide the latency of its own dependent
+        // instructions, so the epilogue's time per tile falls almost linearly with the number of groups.
         const int q = warp & 3;                                  // TMEM lane quarter this warp may read
-        int32_t *thr_w = reinterpret_cast<int32_t *>(gen + S::THR_OFFSET) + q * S::THR_WORDS;   // this warp's thresholds
-        uint32_t *flip_w = reinterpret_cast<uint32_t *>(thr_w + BN);                            // and flip words
-        uint8_t *stg = gen + S::STG_OFFSET + q * S::STG_WARP_BYTES;                             // this warp's staging buffer
-        const uint32_t stg_u32 = base + (uint32_t)(S::STG_OFFSET + q * S::STG_WARP_BYTES);
+        const int grp = (warp - 2) >> 2;                         // which chunks of the tile it drains
+        const int ew = grp * 4 + q;
+        constexpr int CPW = S::CPW;                              // chunks per warp
+        int32_t *thr_w = reinterpret_cast<int32_t *>(gen + S::THR_OFFSET) + ew * S::THR_WORDS;  // this warp's thresholds
+        uint32_t *flip_w = reinterpret_cast<uint32_t *>(thr_w + CPW * 32);                      // and flip words
+        uint8_t *stg = gen + S::STG_OFFSET + ew * S::STG_WARP_BYTES;                            // this warp's staging tile
+        const uint32_t stg_u32 = base + (uint32_t)(S::STG_OFFSET + ew * S::STG_WARP_BYTES);
         const bool want_bits = p.out_bits != nullptr;
         const bool want_form = p.out_form != nullptr;
         const bool want_sign = want_bits || want_form;
         const bool form_fp4 = p.out_form_kind == QNN_FORM_FP4;
         uint32_t iter = 0;
-        uint32_t nstore = 0;                                     // int32 tiles handed to the bulk-store engine so far
         bool ok = true;
-        for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
-            const int32_t tm = (int32_t)(t % p.tiles_m), tn = (int32_t)(t / p.tiles_m);
+        // lane l holds the thresholds of columns c*32 + l of this warp's chunks c = grp + lc*EPI_GROUPS and, as bit lc,
+        // their flips
+        int32_t thr_next[CPW];
+        uint8_t flip_raw[CPW];
+        auto fetch_thresholds = [&](int64_t ncol0) {
+#pragma unroll
+            for (int lc = 0; lc < CPW; ++lc) {
+                const int64_t n = ncol0 + (grp + lc * EPI_GROUPS) * 32 + lane;
+                const bool ncol = (grp + lc * EPI_GROUPS) < BN / 32 && n < p.N;
+                // (raw values: nothing here may wait for the loads -- they are converted when they are parked)
+                const int32_t tv = ncol ? __ldg(p.thr + n) : 0;
+                thr_next[lc] = tv;
+                if (ncol && p.flip) flip_raw[lc] = __ldg(p.flip + n);
+                else flip_raw[lc] = 0;
+            }
+        };
+        if (want_sign && blockIdx.x < num_tiles) fetch_thresholds((int64_t)(blockIdx.x / tiles_m) * BN);
+        for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
+            const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
             const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
             const int64_t ntile = (int64_t)tn * BN;
 
-            // stage this tile's thresholds and flip words while the accumulator is still being produced
+            // Thresholds and flip bytes of this tile were fetched into registers one tile ago (or just before
+            // the loop): park them in this warp's shared rows, then start fetching the next tile's, so that
+            // their global-memory latency never sits between two tiles.
             if (want_sign) {
                 __syncwarp();
 #pragma unroll
-                for (int c = 0; c < BN / 32; ++c) {
-                    const int64_t n = ntile + c * 32 + lane;
-                    const bool ncol = n < p.N;
-                    int32_t tv = ncol ? __ldg(p.thr + n) : 0;
+                for (int lc = 0; lc < CPW; ++lc) {
+                    int32_t tv = thr_next[lc];
                     if (FORM == QNN_FORM_FP4) {
                         // accumulators are exact integers below 2^24 held as floats: compare there.  A threshold
                         // beyond +-2^24 decides the same way as +-2^24, which a float holds exactly.
                         tv = tv > (1 << 24) ? (1 << 24) : (tv < -(1 << 24) ? -(1 << 24) : tv);
                         tv = __float_as_int((float)tv);
+                    } else if (p.thr_clamp > 0) {
+                        // |sum| <= thr_clamp - 1 < 2^30: a threshold beyond +-thr_clamp decides like +-thr_clamp, and
+                        // sum - threshold then cannot overflow, so its sign bit is the comparison
+                        tv = tv > p.thr_clamp ? p.thr_clamp : (tv < -p.thr_clamp ? -p.thr_clamp : tv);
                     }
-                    thr_w[c * 32 + lane] = tv;
-                    const bool f = (ncol && p.flip) ? (__ldg(p.flip + n) != 0) : false;
-                    const uint32_t fw = __ballot_sync(0xffffffffu, f);
-                    if (lane == c) flip_w[c] = fw;
+                    thr_w[lc * 32 + lane] = tv;
+                    const uint32_t fw = __ballot_sync(0xffffffffu, flip_raw[lc] != 0);
+                    if (lane == lc) flip_w[lc] = fw;
                 }
                 __syncwarp();
+                const uint32_t tnext = t + gridDim.x;
+                if (tnext < num_tiles) fetch_thresholds((int64_t)(tnext / tiles_m) * BN);
             }
 
             // which output row this thread owns
@@ -475,21 +507,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(as), aphase, abort_flag, 4))) { ok = false; break; }
             tc_fence_after();
 
+            // this warp's share of the accumulator, 32 columns at a time
+            const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + as * (uint32_t)BN;
+            int nchunks = (int)((p.N - ntile + 31) >> 5);         // warp-uniform
+            nchunks = nchunks > BN / 32 ? BN / 32 : nchunks;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = grp, lc = 0; c < nchunks; c += EPI_GROUPS, ++lc) {
                 const int64_t n0 = ntile + c * 32;
-                if (n0 >= p.N) break;                            // warp-uniform
                 uint32_t v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + as * (uint32_t)BN + (uint32_t)(c * 32), v);
-                // FP4: the fp32 accumulators are exact integers; the border corrections are added in float too
-                if (any_border && cls != 0) {
-                    const int32_t *cp = p.corr + (int64_t)cls * p.N + n0;
+                tmem_ld32(tacc + (uint32_t)(c * 32), v);
+                // Border corrections, class by class: every lane reads the class's 32 values (one address per load
+                // across the warp), the lanes of that class add them.  e2m1: the fp32 accumulators are exact
+                // integers, so the correction is added in float.
+                if (any_border) {
+                    uint32_t todo = __ballot_sync(0xffffffffu, cls != 0);
+                    while (todo != 0) {
+                        const int k = __shfl_sync(0xffffffffu, cls, __ffs((int)todo) - 1);
+                        todo &= ~__ballot_sync(0xffffffffu, cls == k);
+                        const int4 *cp = reinterpret_cast<const int4 *>(p.corr + (int64_t)k * p.corr_ld + n0);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (n0 + j < p.N) {
-                            const int32_t cv = __ldg(cp + j);
-                            if (FORM == QNN_FORM_FP4) v[j] = __float_as_uint(__uint_as_float(v[j]) + (float)cv);
-                            else v[j] += (uint32_t)cv;
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            const int4 cv = __ldg(cp + j4);
+                            if (cls == k) {
+                                if (FORM == QNN_FORM_FP4) {
+                                    v[4 * j4] = __float_as_uint(__uint_as_float(v[4 * j4]) + (float)cv.x);
+                                    v[4 * j4 + 1] = __float_as_uint(__uint_as_float(v[4 * j4 + 1]) + (float)cv.y);
+                                    v[4 * j4 + 2] = __float_as_uint(__uint_as_float(v[4 * j4 + 2]) + (float)cv.z);
+                                    v[4 * j4 + 3] = __float_as_uint(__uint_as_float(v[4 * j4 + 3]) + (float)cv.w);
+                                } else {
+                                    v[4 * j4] += (uint32_t)cv.x; v[4 * j4 + 1] += (uint32_t)cv.y;
+                                    v[4 * j4 + 2] += (uint32_t)cv.z; v[4 * j4 + 3] += (uint32_t)cv.w;
+                                }
+                            }
                         }
                     }
                 }
@@ -502,8 +551,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (p.out != nullptr) {
                     if (STG && p.tma_out) {
                         // registers -> staging tile -> one asynchronous bulk store per 32 x 32 block
-                        uint8_t *buf = stg + (nstore & 1u) * 4096u;
-                        if (lane == 0) bulk_wait_read<1>();      // the store issued two blocks ago has read this buffer
+                        uint8_t *buf = stg;
+                        if (lane == 0) bulk_wait_read<0>();      // this warp's previous store has read the tile
                         __syncwarp();
                         if (p.tma_out == 1) {
                             // [row][32 columns], 16-byte chunks swizzled by the row (the tensor map's 128-byte swizzle)
@@ -519,12 +568,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         fence_async_shared();
                         __syncwarp();
                         if (lane == 0) {
-                            const uint32_t src = stg_u32 + (nstore & 1u) * 4096u;
-                            if (p.tma_out == 1) tma_store_2d(&tmap_out, (int32_t)n0, (int32_t)m_warp0, src);
-                            else tma_store_3d(&tmap_out, c_pix0, (int32_t)n0, c_img, src);
+                            if (p.tma_out == 1) tma_store_2d(&tmap_out, (int32_t)n0, (int32_t)m_warp0, stg_u32);
+                            else tma_store_3d(&tmap_out, c_pix0, (int32_t)n0, c_img, stg_u32);
                             bulk_commit();
                         }
-                        ++nstore;
                     } else if (mrow) {
                         if (p.epilogue == EPI_NCHW) {
 #pragma unroll
@@ -545,20 +592,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     }
                 }
                 if (want_sign) {
-                    const int4 *t4 = reinterpret_cast<const int4 *>(thr_w + c * 32);
+                    const int4 *t4 = reinterpret_cast<const int4 *>(thr_w + lc * 32);
                     uint32_t w = 0;
-                    if (FORM == QNN_FORM_FP4) {
+                    if (FORM == QNN_FORM_FP4 || p.thr_clamp > 0) {
                         // bit j = (acc_j >= thr_j) = NOT sign(acc_j - thr_j): one subtraction and one funnel shift per
-                        // column, last column first so that column 0 lands in bit 0
+                        // column (e2m1: in float, exact; int8: no overflow after the clamp), last column first so that
+                        // column 0 lands in bit 0; four independent byte-wide chains keep the shifts from serialising
+                        uint32_t wb[4];
 #pragma unroll
-                        for (int j4 = 7; j4 >= 0; --j4) {
-                            const int4 tt = t4[j4];              // same address in every lane: a broadcast read
-                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4 + 3]) - __int_as_float(tt.w)), w, 1);
-                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4 + 2]) - __int_as_float(tt.z)), w, 1);
-                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4 + 1]) - __int_as_float(tt.y)), w, 1);
-                            w = __funnelshift_l(__float_as_uint(__uint_as_float(v[4 * j4]) - __int_as_float(tt.x)), w, 1);
+                        for (int g4 = 0; g4 < 4; ++g4) {
+                            uint32_t x = 0;
+#pragma unroll
+                            for (int h = 1; h >= 0; --h) {
+                                const int4 tt = t4[2 * g4 + h];  // same address in every lane: a broadcast read
+                                const int j = 8 * g4 + 4 * h;
+                                if (FORM == QNN_FORM_FP4) {
+                                    x = __funnelshift_l(__float_as_uint(__uint_as_float(v[j + 3]) - __int_as_float(tt.w)), x, 1);
+                                    x = __funnelshift_l(__float_as_uint(__uint_as_float(v[j + 2]) - __int_as_float(tt.z)), x, 1);
+                                    x = __funnelshift_l(__float_as_uint(__uint_as_float(v[j + 1]) - __int_as_float(tt.y)), x, 1);
+                                    x = __funnelshift_l(__float_as_uint(__uint_as_float(v[j]) - __int_as_float(tt.x)), x, 1);
+                                } else {
+                                    x = __funnelshift_l((uint32_t)(iv[j + 3] - tt.w), x, 1);
+                                    x = __funnelshift_l((uint32_t)(iv[j + 2] - tt.z), x, 1);
+                                    x = __funnelshift_l((uint32_t)(iv[j + 1] - tt.y), x, 1);
+                                    x = __funnelshift_l((uint32_t)(iv[j] - tt.x), x, 1);
+                                }
+                            }
+                            wb[g4] = x;
                         }
-                        w = ~w;
+                        w = ~(wb[0] | (wb[1] << 8) | (wb[2] << 16) | (wb[3] << 24));
                     } else {
 #pragma unroll
                         for (int j4 = 0; j4 < 8; ++j4) {
@@ -571,7 +633,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     }
                     const int64_t left = p.N - n0;
                     const uint32_t nmask = left >= 32 ? 0xffffffffu : ((1u << (int)left) - 1u);
-                    w = (w ^ flip_w[c]) & nmask;
+                    w = (w ^ flip_w[lc]) & nmask;
                     if (want_bits && mrow) p.out_bits[m * p.ld_bits + (n0 >> 5)] = w;
                     if (want_form) {
                         if (form_fp4) {
@@ -776,6 +838,7 @@ int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMa
     auto kern = gemm_tc_kernel<FORM, BN, STG>;
     QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
     const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+    QNN_REQUIRE(tiles < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: too many output tiles");
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     profile_before(st);
     kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, p);
@@ -965,6 +1028,10 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
                         g.ld_form >= tc_row_bytes(ceil_div(g.N, 32), g.out_form_kind),
                     QNN_ERR_ALIGNMENT, "tc gemm: form output needs a 16-byte aligned base and a row stride covering N");
     }
+    {
+        const int64_t maxsum = g.K * ((1 << g.ka) - 1) * (int64_t)((1 << g.kb) - 1);
+        p.thr_clamp = maxsum + 1 < ((int64_t)1 << 30) ? (int32_t)(maxsum + 1) : 0;
+    }
     if (form == QNN_FORM_FP4) {
         // block-scaled instruction descriptor: A and B e2m1 (format 1), both K-major, ue8m0 scales, M = 128
         p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((uint32_t)(BM >> 4) << 24);
@@ -982,7 +1049,8 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
         const int R = BM / c.W < c.H ? BM / c.W : c.H;                  // image rows per tile
         QNN_REQUIRE(R >= 1 && R <= 256, QNN_ERR_UNSUPPORTED, "tc conv: bad tile height");
         p.conv = 1; p.cH = c.H; p.cW = c.W; p.cR = R; p.tiles_per_img = (int32_t)ceil_div(c.H, R);
-        p.cKW = c.KW; p.cpad = c.pad; p.cblocks = c.cblocks; p.corr = c.corr;
+        p.cKW = c.KW; p.cpad = c.pad; p.cblocks = c.cblocks; p.corr = c.corr; p.corr_ld = (int64_t)round_up((size_t)g.N, 32);
+        QNN_REQUIRE(aligned(c.corr, 16), QNN_ERR_ALIGNMENT, "tc conv: correction table must be 16-byte aligned");
         p.tiles_m = c.B * p.tiles_per_img;
         p.a_tx_bytes = R * c.W * BKB;
         QNN_REQUIRE(p.num_kb == c.KH * c.KW * c.cblocks, QNN_ERR_INVALID_ARG, "tc conv: K blocks do not match the filter");

@@ -48,7 +48,7 @@ enum Epilogue { EPI_ROWMAJOR = 0, EPI_NCHW = 1, EPI_BITS = 2 };
 struct ConvImplicit {
     int32_t B, H, W, KH, KW, pad;
     int32_t cblocks;            // 128-byte channel blocks per pixel
-    const int32_t *corr;        // [(pad+1)^4][N] border corrections, class 0 (interior) is all zero
+    const int32_t *corr;        // [(pad+1)^4][N rounded up to 32] border corrections (pad columns and class 0 zero)
 };
 
 struct GemmArgs {
