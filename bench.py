@@ -185,30 +185,19 @@ class MlpBench:
         self.flush_sink = self.flush_rd.sum()
 
     def step_calls(self, ev=None):
-        """The Algorithm-4 pass as individual C-ABI calls; `ev` (optional) brackets the dominant product."""
+        """One Algorithm-4 pass on device buffers; `ev` (optional) brackets the dominant product kernel."""
         if self.algo == self.q.QNN_ALGO_AUTO:
-            return self.step_calls_tc(ev)
+            return self.step_forward(ev)
         return self.step_calls_bits(ev)
 
-    def step_calls_tc(self, ev=None):
-        """Tensor-core chain: the uint8 input is the int8-form operand of layer 1 (Eq. 8 recomposed), hidden
-        activations travel as e2m1 values written by the previous product's threshold epilogue, the last
-        hidden layer emits packed bits for the 10-unit xor/popc head."""
-        q, M = self.q, self.M
-        I8, FP4 = q.QNN_FORM_I8, q.QNN_FORM_FP4
-        L = self.layers
-        rb = 4096 // 2
-        q.qnn_tc_gemm(q.tc_operand(self.x, DIMS[0], I8, IN_BITS, q.QNN_MODE_U01),
-                      q.tc_operand(self.w_tc[0], L[0].w_tc_ld, I8), M, DIMS[1], DIMS[0],
-                      thr=self.thr[0], out_form=self.actf[0], out_form_kind=FP4, ld_form_bytes=rb)
+    def step_forward(self, ev=None):
+        """qnn_mlp_forward with prepacked weights: the uint8 input is the int8-form operand of layer 1 (Eq. 8
+        recomposed), hidden activations travel as e2m1 values written by the previous product's threshold
+        epilogue, the last hidden layer emits packed bits for the 10-unit xor/popc head."""
+        q = self.q
         if ev is not None:
-            q.qnn_set_kernel_events(ev[0], ev[1])        # recorded by the library right around the product kernel
-        q.qnn_tc_gemm(q.tc_operand(self.actf[0], rb, FP4), q.tc_operand(self.w_tc[1], L[1].w_tc_ld, FP4), M, DIMS[2],
-                      DIMS[1], thr=self.thr[1], out_form=self.actf[1], out_form_kind=FP4, ld_form_bytes=rb)
-        q.qnn_tc_gemm(q.tc_operand(self.actf[1], rb, FP4), q.tc_operand(self.w_tc[2], L[2].w_tc_ld, FP4), M, DIMS[3],
-                      DIMS[2], thr=self.thr[2], out_bits=self.act[0], ld_words=128)
-        q.qnn_xnor_gemm(self.act[0], 128, self.packed[3], self.ldws[3], M, DIMS[4], DIMS[3], self.scores, DIMS[4],
-                        q.QNN_ALGO_POPC, None)
+            q.qnn_set_kernel_events_nth(ev[0], ev[1], 1)  # second product kernel = hidden layer 2 (10000 x 4096 x 4096)
+        q.qnn_mlp_forward(self.x, self.M, IN_BITS, self.layers, self.scores, self.algo, self.ws)
 
     def step_calls_bits(self, ev=None):
         """The pass on packed bits with a forced algorithm (plane split, per-call operand rewriting)."""

@@ -204,7 +204,11 @@ QNN_API int qnn_bitplane_gemm_threshold(const uint32_t *a, int ka, int a_mode, i
  * else QNN_FORM_I8 when the codes fit a byte, else 0 (use QNN_ALGO_POPC). */
 QNN_API int qnn_tc_form(int ka, int a_mode, int kb, int b_mode, int64_t K);
 
-/* Bytes between rows (dense) and bytes of a whole operand [rows, K] in `form`. */
+/* Recommended bytes between rows and bytes of a whole operand [rows, K] in `form`:
+ * the bytes K elements need (32 * ceil(K / 32) elements: that many bytes in
+ * QNN_FORM_I8, half as many in QNN_FORM_FP4) rounded up to whole 128-byte lines.
+ * Any multiple of 16 that covers the elements is accepted, but rows that do not
+ * start on 128-byte lines make every tile load touch twice the cache lines. */
 QNN_API int64_t qnn_tc_row_bytes(int64_t K, int form);
 QNN_API size_t qnn_tc_operand_bytes(int64_t rows, int64_t K, int form);
 
@@ -256,7 +260,7 @@ QNN_API int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_
  * inside the library image: every GPU context that loads the library holds it
  * until the process exits.  The call performs no cudaMalloc / cudaFree and
  * calls no allocating library routine.  Shapes whose scratch
- *   (M + N) * 32 * ceil(K / 32)   bytes (the M and the N term each rounded up to 256)
+ *   (M + N) * roundup(32 * ceil(K / 32), 128)   bytes (the M and the N term each rounded up to 256)
  * exceeds the array are rejected with QNN_ERR_WORKSPACE before anything runs
  * (e.g. 1024 x 1024 x 4096 fits, 4096 x 4096 x 4096 does not).
  *
@@ -384,6 +388,10 @@ QNN_API int qnn_device_status(void *stream);
  * around operand expansion or im2col), on that call's stream, and disarms
  * them.  Pass NULLs to disarm. */
 QNN_API int qnn_set_kernel_events(void *start, void *stop);
+
+/* Same, but the events go around the (nth + 1)-th matrix-product kernel this thread launches from now on
+ * (nth = 0 is the next one): lets one layer inside qnn_mlp_forward be timed. */
+QNN_API int qnn_set_kernel_events_nth(void *start, void *stop, int nth);
 
 /* Number of kernels this library has launched in this process so far (all
  * threads, all streams); a monotonically increasing bookkeeping counter. */

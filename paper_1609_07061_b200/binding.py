@@ -93,6 +93,7 @@ _SIGS = {
     "qnn_device_status": (i32, [vp]),
     "qnn_launch_count": (ctypes.c_uint64, []),
     "qnn_set_kernel_events": (i32, [vp, vp]),
+    "qnn_set_kernel_events_nth": (i32, [vp, vp, i32]),
 }
 for _name, (_res, _args) in _SIGS.items():
     _fn = getattr(_lib, _name)          # AttributeError here = the library does not export a declared symbol
@@ -316,6 +317,13 @@ def qnn_set_kernel_events(start: Optional[torch.cuda.Event], stop: Optional[torc
     a = None if start is None else start.cuda_event
     b = None if stop is None else stop.cuda_event
     _ck(_lib.qnn_set_kernel_events(a, b), "qnn_set_kernel_events")
+
+
+def qnn_set_kernel_events_nth(start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event], nth: int):
+    """As qnn_set_kernel_events, around the (nth + 1)-th product kernel launched from now on."""
+    a = None if start is None else start.cuda_event
+    b = None if stop is None else stop.cuda_event
+    _ck(_lib.qnn_set_kernel_events_nth(a, b, nth), "qnn_set_kernel_events_nth")
 
 
 def qnn_xnor_gemm_noalloc(a, lda, b, ldb, M, N, K, out, ldo):

@@ -22,7 +22,7 @@ int fail(int code, const char *fmt, ...)
 }
 
 void clear_error() { g_err[0] = 0; }
-void profile_arm(cudaEvent_t a, cudaEvent_t b);
+void profile_arm(cudaEvent_t a, cudaEvent_t b, int skip);
 
 int check_launch(const char *what)
 {
@@ -33,17 +33,20 @@ int check_launch(const char *what)
 }
 
 static thread_local cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
+static thread_local int g_ev_skip = 0;          // product kernels to let pass before the armed one
 
 void profile_before(cudaStream_t st)
 {
-    if (g_ev_start) cudaEventRecord(g_ev_start, st);
+    if (g_ev_start && g_ev_skip == 0) cudaEventRecord(g_ev_start, st);
 }
 void profile_after(cudaStream_t st)
 {
+    if (!g_ev_start) return;
+    if (g_ev_skip > 0) { --g_ev_skip; return; }
     if (g_ev_stop) cudaEventRecord(g_ev_stop, st);
     g_ev_start = g_ev_stop = nullptr;
 }
-void profile_arm(cudaEvent_t a, cudaEvent_t b) { g_ev_start = a; g_ev_stop = b; }
+void profile_arm(cudaEvent_t a, cudaEvent_t b, int skip) { g_ev_start = a; g_ev_stop = b; g_ev_skip = skip; }
 
 int sm_count()
 {
@@ -69,7 +72,15 @@ int qnn_version(void) { return QNN_VERSION; }
 int qnn_set_kernel_events(void *start, void *stop)
 {
     QNN_REQUIRE((start == nullptr) == (stop == nullptr), QNN_ERR_INVALID_ARG, "qnn_set_kernel_events: pass both events or neither");
-    qnn::profile_arm(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop));
+    qnn::profile_arm(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop), 0);
+    return QNN_OK;
+}
+
+int qnn_set_kernel_events_nth(void *start, void *stop, int nth)
+{
+    QNN_REQUIRE((start == nullptr) == (stop == nullptr), QNN_ERR_INVALID_ARG, "qnn_set_kernel_events_nth: pass both events or neither");
+    QNN_REQUIRE(nth >= 0, QNN_ERR_INVALID_ARG, "qnn_set_kernel_events_nth: nth is negative");
+    qnn::profile_arm(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop), nth);
     return QNN_OK;
 }
 

@@ -184,7 +184,8 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
         const int64_t cbytes = tc_row_bytes(Cw, form);
         const int classes = (pad + 1) * (pad + 1) * (pad + 1) * (pad + 1);
         const size_t x_bytes = round_up((size_t)M * (size_t)cbytes, 256);
-        const size_t w_bytes = round_up((size_t)Cout * (size_t)tc_row_bytes(kwords, form), 256);
+        const int64_t w_pitch = tc_row_pitch(kwords, form);
+        const size_t w_bytes = round_up((size_t)Cout * (size_t)w_pitch, 256);
         const int corr_ld = (int)round_up((size_t)Cout, 32);
         const size_t c_bytes = round_up(sizeof(int32_t) * (size_t)classes * (size_t)corr_ld, 256);
         if (ws != nullptr && aligned(ws, 256) && ws_bytes >= x_bytes + w_bytes + c_bytes) {
@@ -192,10 +193,10 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
             uint8_t *wf = xf + x_bytes;
             int32_t *corr = reinterpret_cast<int32_t *>(wf + w_bytes);
             g.a_tc = xf; g.a_tc_form = form; g.a_tc_ld = cbytes;
-            g.b_tc = wf; g.b_tc_form = form; g.b_tc_ld = tc_row_bytes(kwords, form);
+            g.b_tc = wf; g.b_tc_form = form; g.b_tc_ld = w_pitch;
             if (int rc = validate_gemm(g)) return rc;
             if (int rc = tc_expand(x, 1, QNN_MODE_PM1, Cw, 0, M, Cw, Cw, 32, form, xf, cbytes, st)) return rc;
-            if (int rc = tc_expand(w, 1, QNN_MODE_PM1, kwords, 0, Cout, kwords, kwords, 32, form, wf, tc_row_bytes(kwords, form), st))
+            if (int rc = tc_expand(w, 1, QNN_MODE_PM1, kwords, 0, Cout, kwords, kwords, 32, form, wf, w_pitch, st))
                 return rc;
             conv_border_corr_kernel<<<grid_for((int64_t)classes * corr_ld), 256, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, classes,
                                                                                            corr_ld);

@@ -74,8 +74,8 @@ int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_
             const bool fits = tc_form_holds(form, g.ka, g.a_mode) && tc_form_holds(form, g.kb, g.b_mode) &&
                               (form != QNN_FORM_FP4 || tc_pick_form(g.ka, g.a_mode, g.kb, g.b_mode, g.K) == QNN_FORM_FP4);
             const int64_t kw = g.kwords > 0 ? g.kwords : ceil_div(g.K, 32);
-            const size_t need = round_up((size_t)g.M * (size_t)tc_row_bytes(kw, form), 256) +
-                                round_up((size_t)g.N * (size_t)tc_row_bytes(kw, form), 256);
+            const size_t need = round_up((size_t)g.M * (size_t)tc_row_pitch(kw, form), 256) +
+                                round_up((size_t)g.N * (size_t)tc_row_pitch(kw, form), 256);
             if (!fits || kw == 0 || ws == nullptr || ws_bytes < need) algo = QNN_ALGO_POPC;
         }
         if (algo == QNN_ALGO_B1_MMA && !(g.ka == 1 && g.kb == 1)) algo = QNN_ALGO_POPC;
@@ -155,7 +155,7 @@ int qnn_tc_form(int ka, int a_mode, int kb, int b_mode, int64_t K)
 int64_t qnn_tc_row_bytes(int64_t K, int form)
 {
     if (K < 0 || (form != QNN_FORM_I8 && form != QNN_FORM_FP4)) return 0;
-    return tc_row_bytes(ceil_div(K, 32), form);
+    return tc_row_pitch(ceil_div(K, 32), form);
 }
 
 size_t qnn_tc_operand_bytes(int64_t rows, int64_t K, int form)
@@ -240,7 +240,7 @@ size_t qnn_workspace_bytes(int op, int64_t M, int64_t N, int64_t K, int ka, int 
     }
     if (algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_AUTO) bytes += gemm_tc_workspace_bytes(M, N, K, ka, kb);
     if (algo == QNN_ALGO_TC_FP4) {
-        const int64_t rb = tc_row_bytes(ceil_div(K, 32), QNN_FORM_FP4);
+        const int64_t rb = tc_row_pitch(ceil_div(K, 32), QNN_FORM_FP4);
         bytes += round_up((size_t)M * (size_t)rb, 256) + round_up((size_t)N * (size_t)rb, 256);
     }
     return bytes;

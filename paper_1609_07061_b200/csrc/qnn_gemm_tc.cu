@@ -693,25 +693,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // `period`/`tail` say where pad bits sit: word (w mod period) == period-1 has only `tail` valid
 // bits; every pad position expands to the value 0.
 
-// int8 form: one thread produces 16 consecutive bytes (half a source word) of a row.
+// int8 form: one thread produces 16 consecutive bytes (half a source word) of a row.  IDX is the index type:
+// 32-bit arithmetic whenever the element count allows it (the 64-bit divisions would dominate the kernel).
+template <typename IDX>
 __global__ void __launch_bounds__(256) expand_i8_kernel(const uint32_t *__restrict__ planes, int nplanes, int pm1,
                                                         int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
-                                                        int64_t period, int tail, uint8_t *__restrict__ out, int64_t out_ld)
+                                                        int64_t period64, int tail, uint8_t *__restrict__ out, int64_t out_ld)
 {
-    const int64_t chunks = kwords * 2;
-    const int64_t total = rows * chunks;
+    const IDX chunks = (IDX)(kwords * 2);
+    const IDX total = (IDX)rows * chunks;
+    const IDX period = (IDX)period64;
     const uint32_t lcode = (1u << nplanes) - 1u;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = e / chunks;
-        const int64_t ch = e - r * chunks;
-        const int64_t widx = ch >> 1;
+    for (IDX e = (IDX)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (IDX)gridDim.x * blockDim.x) {
+        const IDX r = e / chunks;
+        const IDX ch = e - r * chunks;
+        const IDX widx = ch >> 1;
         const int half = (int)(ch & 1);
-        const int valid = ((widx % period) == period - 1) ? tail : 32;
-        const uint32_t vword = (valid >= 32) ? 0xffffffffu : ((1u << valid) - 1u);
-        const uint32_t vm = (vword >> (16 * half)) & 0xffffu;
+        const bool ragged = tail < 32 && ((widx % period) == period - 1);      // this word holds pad bits
         uint32_t acc[4] = {0u, 0u, 0u, 0u};
         for (int i = 0; i < nplanes; ++i) {
-            const uint32_t w = __ldg(planes + i * plane_stride + r * ld + widx);
+            const uint32_t w = __ldg(planes + i * plane_stride + (int64_t)r * ld + widx);
             const uint32_t h = (w >> (16 * half)) & 0xffffu;
 #pragma unroll
             for (int nb = 0; nb < 4; ++nb) acc[nb] += spread_bits_to_bytes((h >> (4 * nb)) & 0xfu) << i;
@@ -721,49 +722,61 @@ __global__ void __launch_bounds__(256) expand_i8_kernel(const uint32_t *__restri
         for (int nb = 0; nb < 4; ++nb) {
             uint32_t v = acc[nb];
             if (pm1) v = __vsub4(v << 1, lcode * 0x01010101u);                  // 2q - (2^k - 1) per byte
-            o[nb] = v & (spread_bits_to_bytes((vm >> (4 * nb)) & 0xfu) * 0xffu);
+            o[nb] = v;
         }
-        *reinterpret_cast<uint4 *>(out + r * out_ld + ch * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        if (ragged) {
+            const uint32_t vm = (((1u << tail) - 1u) >> (16 * half)) & 0xffffu;
+#pragma unroll
+            for (int nb = 0; nb < 4; ++nb) o[nb] &= spread_bits_to_bytes((vm >> (4 * nb)) & 0xfu) * 0xffu;
+        }
+        *reinterpret_cast<uint4 *>(out + (int64_t)r * out_ld + (int64_t)ch * 16) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
 // e2m1 code of an integer value in {0, +-1, +-2, +-3}: sign bit 3; magnitudes 1 -> 0b010, 2 -> 0b100, 3 -> 0b101.
 // fp4 form: one thread turns one source word (per plane) into 32 nibbles = 16 bytes.
+template <typename IDX>
 __global__ void __launch_bounds__(256) expand_fp4_kernel(const uint32_t *__restrict__ planes, int nplanes, int pm1,
-                                                         int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
-                                                         int64_t period, int tail, uint8_t *__restrict__ out, int64_t out_ld)
+                                                         int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords64,
+                                                         int64_t period64, int tail, uint8_t *__restrict__ out, int64_t out_ld)
 {
-    const int64_t total = rows * kwords;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = e / kwords;
-        const int64_t w = e - r * kwords;
-        const int valid = ((w % period) == period - 1) ? tail : 32;
-        const uint32_t vword = (valid >= 32) ? 0xffffffffu : ((1u << valid) - 1u);
-        const uint32_t p0 = __ldg(planes + r * ld + w);
-        const uint32_t p1 = nplanes > 1 ? __ldg(planes + plane_stride + r * ld + w) : 0u;
+    const IDX kwords = (IDX)kwords64;
+    const IDX total = (IDX)rows * kwords;
+    const IDX period = (IDX)period64;
+    for (IDX e = (IDX)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (IDX)gridDim.x * blockDim.x) {
+        const IDX r = e / kwords;
+        const IDX w = e - r * kwords;
+        const bool ragged = tail < 32 && ((w % period) == period - 1);         // this word holds pad bits
+        const uint32_t p0 = __ldg(planes + (int64_t)r * ld + w);
+        const uint32_t p1 = nplanes > 1 ? __ldg(planes + plane_stride + (int64_t)r * ld + w) : 0u;
         uint32_t o[4];
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             const uint32_t s0 = spread_bits_to_nibbles((p0 >> (8 * b)) & 0xffu);
-            const uint32_t s1 = spread_bits_to_nibbles((p1 >> (8 * b)) & 0xffu);
-            const uint32_t vm = spread_bits_to_nibbles((vword >> (8 * b)) & 0xffu) * 0xfu;
             uint32_t code;
             if (pm1) {
                 if (nplanes == 1) {
                     code = 0xAAAAAAAAu ^ (s0 << 3);                            // bit 1 -> +1 (0x2), bit 0 -> -1 (0xA)
                 } else {
                     // value 2*q - 3 with q = s0 + 2*s1: q 0 -> -3, 1 -> -1, 2 -> +1, 3 -> +3
+                    const uint32_t s1 = spread_bits_to_nibbles((p1 >> (8 * b)) & 0xffu);
                     const uint32_t neg = (s1 ^ 0x11111111u) << 3;               // sign: negative while plane 1 is clear
                     const uint32_t three = ~(s0 ^ s1) & 0x11111111u;            // |value| = 3 when both planes agree
                     code = neg | (three * 0x5u) | ((three ^ 0x11111111u) << 1);  // 3 -> 0b101, 1 -> 0b010
                 }
             } else {
                 // unsigned code q = s0 + 2*s1: 0 -> 0, 1 -> 0b010, 2 -> 0b100, 3 -> 0b101
+                const uint32_t s1 = spread_bits_to_nibbles((p1 >> (8 * b)) & 0xffu);
                 code = (s1 << 2) | ((s0 & ~s1) << 1) | (s0 & s1);
             }
-            o[b] = code & vm;
+            o[b] = code;
         }
-        *reinterpret_cast<uint4 *>(out + r * out_ld + w * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        if (ragged) {
+            const uint32_t vword = (1u << tail) - 1u;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) o[b] &= spread_bits_to_nibbles((vword >> (8 * b)) & 0xffu) * 0xfu;
+        }
+        *reinterpret_cast<uint4 *>(out + (int64_t)r * out_ld + (int64_t)w * 16) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
@@ -899,7 +912,7 @@ int pick_bn(int64_t tiles_m, int64_t N)
 int grid_for_items(int64_t items)
 {
     const int64_t need = ceil_div(items, 256);
-    const int64_t cap = (int64_t)sm_count() * 16;
+    const int64_t cap = (int64_t)sm_count() * 32;
     return (int)(need < cap ? need : cap);
 }
 
@@ -923,18 +936,27 @@ int tc_pick_form(int ka, int a_mode, int kb, int b_mode, int64_t K)
 }
 
 int64_t tc_row_bytes(int64_t kwords, int form) { return form == QNN_FORM_FP4 ? kwords * 16 : kwords * 32; }
+int64_t tc_row_pitch(int64_t kwords, int form) { return (int64_t)round_up((size_t)tc_row_bytes(kwords, form), 128); }
 
 int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
               int64_t pad_period, int pad_tail, int form, uint8_t *dst, int64_t dst_ld, cudaStream_t st)
 {
     if (rows == 0 || kwords == 0) return QNN_OK;
     QNN_REQUIRE(tc_form_holds(form, planes, mode), QNN_ERR_UNSUPPORTED, "tc expand: %d planes do not fit form %d", planes, form);
+    const int64_t items = form == QNN_FORM_FP4 ? rows * kwords : rows * kwords * 2;
+    const bool narrow = items < ((int64_t)1 << 31);
+    const int grid = grid_for_items(items);
+    const int pm1 = mode == QNN_MODE_PM1;
     if (form == QNN_FORM_FP4) {
-        expand_fp4_kernel<<<grid_for_items(rows * kwords), 256, 0, st>>>(src, planes, mode == QNN_MODE_PM1, ld, plane_stride,
-                                                                        rows, kwords, pad_period, pad_tail, dst, dst_ld);
+        if (narrow)
+            expand_fp4_kernel<uint32_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
+        else
+            expand_fp4_kernel<int64_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
     } else {
-        expand_i8_kernel<<<grid_for_items(rows * kwords * 2), 256, 0, st>>>(src, planes, mode == QNN_MODE_PM1, ld, plane_stride,
-                                                                           rows, kwords, pad_period, pad_tail, dst, dst_ld);
+        if (narrow)
+            expand_i8_kernel<uint32_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
+        else
+            expand_i8_kernel<int64_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
     }
     return check_launch("tc expand");
 }
@@ -948,7 +970,7 @@ bool gemm_tc_supported(const GemmArgs &g)
 
 size_t gemm_tc_workspace_bytes(int64_t M, int64_t N, int64_t K, int, int)
 {
-    const int64_t rb = tc_row_bytes(ceil_div(K, 32), QNN_FORM_I8);
+    const int64_t rb = tc_row_pitch(ceil_div(K, 32), QNN_FORM_I8);
     return round_up((size_t)M * (size_t)rb, 256) + round_up((size_t)N * (size_t)rb, 256);
 }
 
@@ -987,8 +1009,9 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     int64_t a_ld = g.a_tc_ld, b_ld = g.b_tc_ld;
     int64_t a_row_bytes = row_bytes;
     size_t need = 0;
-    const size_t a_bytes = g.a_tc ? 0 : round_up((size_t)g.M * (size_t)row_bytes, 256);
-    const size_t b_bytes = g.b_tc ? 0 : round_up((size_t)g.N * (size_t)row_bytes, 256);
+    const int64_t pitch = tc_row_pitch(kwords, form);
+    const size_t a_bytes = g.a_tc ? 0 : round_up((size_t)g.M * (size_t)pitch, 256);
+    const size_t b_bytes = g.b_tc ? 0 : round_up((size_t)g.N * (size_t)pitch, 256);
     need = a_bytes + b_bytes;
     if (need > 0)
         QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= need, QNN_ERR_WORKSPACE,
@@ -1000,18 +1023,18 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     } else {
         QNN_REQUIRE(!g.conv, QNN_ERR_INVALID_ARG, "tc conv: the NHWC operand must be prepared");
         uint8_t *dst = static_cast<uint8_t *>(ws);
-        if (int rc = tc_expand(g.a, g.ka, g.a_mode, g.lda, g.a_plane_stride, g.M, kwords, period, tail, form, dst, row_bytes, st))
+        if (int rc = tc_expand(g.a, g.ka, g.a_mode, g.lda, g.a_plane_stride, g.M, kwords, period, tail, form, dst, pitch, st))
             return rc;
-        a8 = dst; a_ld = row_bytes;
+        a8 = dst; a_ld = pitch;
     }
     if (g.b_tc) {
         QNN_REQUIRE(aligned(g.b_tc, 16) && b_ld % 16 == 0 && b_ld >= row_bytes, QNN_ERR_ALIGNMENT,
                     "tc gemm: prepared B operand needs a 16-byte aligned base and row stride");
     } else {
         uint8_t *dst = static_cast<uint8_t *>(ws) + a_bytes;
-        if (int rc = tc_expand(g.b, g.kb, g.b_mode, g.ldb, g.b_plane_stride, g.N, kwords, period, tail, form, dst, row_bytes, st))
+        if (int rc = tc_expand(g.b, g.kb, g.b_mode, g.ldb, g.b_plane_stride, g.N, kwords, period, tail, form, dst, pitch, st))
             return rc;
-        b8 = dst; b_ld = row_bytes;
+        b8 = dst; b_ld = pitch;
     }
 
     TcParams p{};

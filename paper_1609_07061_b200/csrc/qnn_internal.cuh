@@ -93,6 +93,9 @@ bool gemm_tc_supported(const GemmArgs &g);
 int tc_pick_form(int ka, int a_mode, int kb, int b_mode, int64_t K);
 bool tc_form_holds(int form, int planes, int mode);
 int64_t tc_row_bytes(int64_t kwords, int form);
+// distance between rows the library itself lays operands out with: whole 128-byte lines, so that every TMA box row
+// is one line (a row pitch that is not a multiple of 128 doubles the memory requests of the loads)
+int64_t tc_row_pitch(int64_t kwords, int form);
 int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
               int64_t pad_period, int pad_tail, int form, uint8_t *dst, int64_t dst_ld, cudaStream_t st);
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st);

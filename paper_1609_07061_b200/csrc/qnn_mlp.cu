@@ -21,6 +21,18 @@ struct MlpPlan {
 
 inline bool is_tc(int algo) { return algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_TC_FP4; }
 
+// Copies a dense byte matrix [rows, K] (K a multiple of 16) to rows `pitch` bytes apart.  The tensor-core
+// product reads its operands in 128-byte boxes; rows that start on 128-byte lines halve the lines a box touches.
+__global__ void __launch_bounds__(256) repitch_rows_kernel(const uint4 *__restrict__ src, int64_t rows, int64_t k16,
+                                                           uint4 *__restrict__ dst, int64_t pitch16)
+{
+    const int64_t total = rows * k16;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = e / k16, c = e - r * k16;
+        dst[r * pitch16 + c] = __ldcs(src + e);
+    }
+}
+
 int resolve_env_algo()
 {
     const char *e = getenv("QNN_FORCE_ALGO");
@@ -124,6 +136,16 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
             const bool direct = c.form == QNN_FORM_I8 && in_bits == 8 && (ly.K % 16 == 0) && aligned(x_dev, 16);
             if (direct) {
                 g.a_tc = x_dev; g.a_tc_form = QNN_FORM_I8; g.a_tc_ld = ly.K;
+                if (ly.K % 128 != 0) {
+                    // rows of the input re-spaced to whole 128-byte lines (the plane buffer is free on this path)
+                    const int64_t pitch = p.kw0 * 32;
+                    const int64_t total = M * (ly.K / 16);
+                    const int64_t need = ceil_div(total, 256), cap = (int64_t)sm_count() * 16;
+                    repitch_rows_kernel<<<(int)(need < cap ? need : cap), 256, 0, st>>>(
+                        reinterpret_cast<const uint4 *>(x_dev), M, ly.K / 16, reinterpret_cast<uint4 *>(planes), pitch / 16);
+                    if (int rc = check_launch("mlp input re-spacing")) return rc;
+                    g.a_tc = planes; g.a_tc_ld = pitch;
+                }
             } else {
                 if (int rc = qnn_pack_planes_u8(x_dev, M, ly.K, ly.K, in_bits, planes, p.kw0, plane_stride, nullptr, st))
                     return rc;
@@ -148,7 +170,7 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
             const bool give_form = is_tc(c.algo) && is_tc(nx.algo);
             cur_bits = nullptr; cur_form = nullptr;
             if (give_form) {
-                g.out_form = buf + (p.act_bytes >> 2); g.out_form_kind = nx.form; g.ld_form = tc_row_bytes(wds, nx.form);
+                g.out_form = buf + (p.act_bytes >> 2); g.out_form_kind = nx.form; g.ld_form = tc_row_pitch(wds, nx.form);
                 cur_form = g.out_form; cur_form_kind = nx.form; cur_form_ld = g.ld_form;
             } else {
                 g.out_bits = reinterpret_cast<uint32_t *>(buf); g.ld_bits = wds;

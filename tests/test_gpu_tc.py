@@ -46,8 +46,8 @@ def test_prepack_matches_reference_encoding(q, planes, mode, form_name, rows, K)
     codes = rng.integers(0, 1 << planes, (rows, K)).astype(np.int32)
     ld = words_per_row(K) + 2
     pl = _planes_ref(codes, planes, ld)
-    rb = q.qnn_tc_row_bytes(K, form)
-    assert rb == words_per_row(K) * (32 if form == q.QNN_FORM_I8 else 16)
+    rb = words_per_row(K) * (32 if form == q.QNN_FORM_I8 else 16)      # bytes the elements need
+    assert q.qnn_tc_row_bytes(K, form) == (rb + 127) // 128 * 128     # recommended pitch: whole 128-byte lines
     ldb = rb + 16
     out = Guarded((rows, ldb), torch.uint8, fill=0x5C)
     q.qnn_tc_prepack(as_i32_words(pl).cuda(), planes, mode, ld, rows * ld, rows, K, form, out.t, ldb)
@@ -98,6 +98,7 @@ def test_tc_gemm_all_outputs(q, form_name, out_form_name, M, N, K):
     ldw = words_per_row(N) + 1
     bits = Guarded((M, ldw), torch.int32, fill=0x77777777)
     orb = q.qnn_tc_row_bytes(N, oform)
+    onb = words_per_row(N) * (32 if oform == q.QNN_FORM_I8 else 16)       # bytes the N outputs occupy
     of = Guarded((M, orb + 16), torch.uint8, fill=0x5C)
     q.qnn_tc_gemm(q.tc_operand(af, rb, form), q.tc_operand(bf, rb + 32, form), M, N, K, out.t, N + 1, dev(T), dev(flip),
                   bits.t, ldw, of.t, oform, orb + 16)
@@ -109,8 +110,8 @@ def test_tc_gemm_all_outputs(q, form_name, out_form_name, M, N, K):
     np.testing.assert_array_equal(unpack_words(words_np(bits.t), N), want_bits)
     assert (words_np(bits.t)[:, words_per_row(N):] == 0x77777777).all()
     got_f = of.t.cpu().numpy()
-    np.testing.assert_array_equal(got_f[:, :orb], form_ref(2 * want_bits.astype(np.int32) - 1, N, oform, q))
-    assert (got_f[:, orb:] == 0x5C).all()
+    np.testing.assert_array_equal(got_f[:, :onb], form_ref(2 * want_bits.astype(np.int32) - 1, N, oform, q))
+    assert (got_f[:, onb:] == 0x5C).all()
     for g in (out, bits, of):
         g.check()
 
