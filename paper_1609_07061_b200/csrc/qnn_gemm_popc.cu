@@ -215,9 +215,10 @@ __global__ void __launch_bounds__(THREADS) gemm_popc_kernel(const PopcParams P)
 }
 
 // Few output units (a classifier head: N <= 16), 1-bit x 1-bit: the work is one pass over the packed
-// activations, so the kernel is a streaming one.  B's rows sit in shared memory; a warp owns a row
-// of A, each lane xor/popc-ing every 32nd 128-bit chunk against all N rows, then the N partial
-// counts are summed across the warp.
+// activations, so the kernel is a streaming one.  B's rows sit in shared memory; a warp owns FOUR rows
+// of A at a time, eight lanes per row, each lane xor/popc-ing every eighth 128-bit chunk of its row
+// against all N rows of B; the N partial counts are then summed over the eight lanes (three shuffle
+// steps instead of five over a whole warp).
 constexpr int SKINNY_N = 16;
 __global__ void __launch_bounds__(256) gemm_popc_skinny_kernel(const uint32_t *__restrict__ a, int64_t lda,
                                                                const uint32_t *__restrict__ b, int64_t ldb, int64_t M,
@@ -225,65 +226,57 @@ __global__ void __launch_bounds__(256) gemm_popc_skinny_kernel(const uint32_t *_
                                                                int64_t ldo)
 {
     extern __shared__ __align__(16) uint32_t bs[];               // [N][kw4], kw4 = kwords rounded up to 4, zero padded
-    const int64_t kw4 = (kwords + 3) & ~(int64_t)3;
-    for (int64_t e = threadIdx.x; e < (int64_t)N * kw4; e += blockDim.x) {
-        const int64_t n = e / kw4, k = e - n * kw4;
-        bs[e] = k < kwords ? __ldg(b + n * ldb + k) : 0u;
+    const int kw4 = (int)((kwords + 3) & ~(int64_t)3);
+    for (int e = threadIdx.x; e < N * kw4; e += blockDim.x) {
+        const int n = e / kw4, k = e - n * kw4;
+        bs[e] = k < kwords ? __ldg(b + (int64_t)n * ldb + k) : 0u;
     }
     __syncthreads();
     const int lane = threadIdx.x & 31;
+    const int sub = lane >> 3;                                   // which of the warp's four rows
+    const int part = lane & 7;                                   // which eighth of the row's chunks
     const int64_t warp0 = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const bool vec = ((lda & 3) == 0) && ((reinterpret_cast<uintptr_t>(a) & 15) == 0);
-    // two rows per pass: their loads are in flight together
-    for (int64_t m = warp0; m < M; m += 2 * nwarps) {
-        const int64_t m2 = m + nwarps;
-        const bool has2 = m2 < M;
-        int32_t acc[SKINNY_N], acc2[SKINNY_N];
+    for (int64_t m0 = warp0 * 4; m0 < M; m0 += nwarps * 4) {
+        const int64_t m = m0 + sub;
+        const bool live = m < M;
+        int32_t acc[SKINNY_N];
 #pragma unroll
-        for (int n = 0; n < SKINNY_N; ++n) { acc[n] = 0; acc2[n] = 0; }
-        const uint32_t *arow = a + m * lda;
-        const uint32_t *arow2 = a + (has2 ? m2 : m) * lda;
-        for (int64_t k = (int64_t)lane * 4; k < kwords; k += 128) {
-            uint4 av, aw;
+        for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0;
+        const uint32_t *arow = a + (live ? m : m0) * lda;
+        for (int k = part * 4; k < kwords; k += 32) {
+            uint4 av;
             if (vec && k + 4 <= kwords) {
                 av = __ldcs(reinterpret_cast<const uint4 *>(arow + k));
-                aw = __ldcs(reinterpret_cast<const uint4 *>(arow2 + k));
             } else {
                 av.x = arow[k];
                 av.y = k + 1 < kwords ? arow[k + 1] : 0u;
                 av.z = k + 2 < kwords ? arow[k + 2] : 0u;
                 av.w = k + 3 < kwords ? arow[k + 3] : 0u;
-                aw.x = arow2[k];
-                aw.y = k + 1 < kwords ? arow2[k + 1] : 0u;
-                aw.z = k + 2 < kwords ? arow2[k + 2] : 0u;
-                aw.w = k + 3 < kwords ? arow2[k + 3] : 0u;
             }
 #pragma unroll
             for (int n = 0; n < SKINNY_N; ++n) {
                 if (n < N) {
                     const uint4 bv = *reinterpret_cast<const uint4 *>(bs + n * kw4 + k);
                     acc[n] += __popc(av.x ^ bv.x) + __popc(av.y ^ bv.y) + __popc(av.z ^ bv.z) + __popc(av.w ^ bv.w);
-                    acc2[n] += __popc(aw.x ^ bv.x) + __popc(aw.y ^ bv.y) + __popc(aw.z ^ bv.z) + __popc(aw.w ^ bv.w);
                 }
             }
         }
-        int32_t mine = 0, mine2 = 0;
+        int32_t lo = 0, hi = 0;                                  // lane `part` keeps units part and part + 8 of its row
 #pragma unroll
         for (int n = 0; n < SKINNY_N; ++n) {
             if (n < N) {
-                int32_t v = acc[n], v2 = acc2[n];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    v += __shfl_xor_sync(0xffffffffu, v, o);
-                    v2 += __shfl_xor_sync(0xffffffffu, v2, o);
-                }
-                if (lane == n) { mine = v; mine2 = v2; }
+                int32_t v = acc[n];
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                v += __shfl_xor_sync(0xffffffffu, v, 4);
+                if ((n & 7) == part) { if (n < 8) lo = v; else hi = v; }
             }
         }
-        if (lane < N) {
-            out[m * ldo + lane] = K - 2 * mine;
-            if (has2) out[m2 * ldo + lane] = K - 2 * mine2;
+        if (live) {
+            if (part < N) out[m * ldo + part] = K - 2 * lo;
+            if (part + 8 < N) out[m * ldo + part + 8] = K - 2 * hi;
         }
     }
 }
@@ -295,9 +288,9 @@ int launch_skinny(const PopcParams &P, cudaStream_t st)
     const size_t smem = sizeof(uint32_t) * (size_t)g.N * (size_t)kw4;
     auto kern = gemm_popc_skinny_kernel;
     if (smem > 48 * 1024) QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    // few resident blocks per SM, several rows per warp: the copy of B into shared memory is paid once per block
+    // a warp takes four rows per pass, a block 32
     const int64_t need = ceil_div(g.M, 32);
-    const int64_t cap = (int64_t)sm_count() * 2;
+    const int64_t cap = (int64_t)sm_count() * 4;
     const int blocks = (int)(need < cap ? need : cap);
     profile_before(st);
     kern<<<blocks, 256, smem, st>>>(g.a, g.lda, g.b, g.ldb, g.M, (int)g.N, P.kwords, P.kll, g.out, g.ldo);
