@@ -57,8 +57,9 @@ struct ThresholdSrc {
     }
 };
 
+// (eight resident blocks per SM: this HBM-bound kernel lives on the bytes it keeps in flight)
 template <class Src, int UNROLL, bool VEC>
-__global__ void __launch_bounds__(256) row_pack_kernel(Src src, int64_t rows, int64_t K, uint32_t *__restrict__ out,
+__global__ void __launch_bounds__(256, 8) row_pack_kernel(Src src, int64_t rows, int64_t K, uint32_t *__restrict__ out,
                                                        int64_t ld_words, int32_t *__restrict__ row_popc,
                                                        int64_t chunks_per_row)
 {
@@ -186,6 +187,47 @@ __global__ void __launch_bounds__(256) row_planes_kernel(Src src, int64_t rows, 
             }
         }
         if (row_sum != nullptr) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0 && sum) atomicAdd(row_sum + r, sum);
+        }
+    }
+}
+
+// uint8 codes, vector path (K and the row pitch multiples of 16, 16-byte aligned base): a lane loads 16
+// consecutive codes at once; bit i of every byte is gathered with one multiply per four codes
+// (0x01020408 moves the four byte-LSBs into one nibble), two neighbouring lanes make a 32-bit word.
+__global__ void __launch_bounds__(256) row_planes_u8_vec_kernel(const uint8_t *__restrict__ x, int64_t ld, int qmask,
+                                                                int64_t rows, int64_t K, int bits,
+                                                                uint32_t *__restrict__ planes, int64_t ld_words,
+                                                                int64_t plane_stride, int32_t *__restrict__ row_sum,
+                                                                int64_t chunks_per_row)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t total = rows * chunks_per_row;
+    const uint32_t qm4 = (uint32_t)qmask * 0x01010101u;
+    for (int64_t item = warp0; item < total; item += nwarps) {
+        const int64_t r = item / chunks_per_row;
+        const int64_t k0 = (item - r * chunks_per_row) * 512;
+        const int64_t k = k0 + lane * 16;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (k < K) v = __ldcs(reinterpret_cast<const uint4 *>(x + r * ld + k));
+        v.x &= qm4; v.y &= qm4; v.z &= qm4; v.w &= qm4;
+        const int64_t kw = (k0 >> 5) + (lane >> 1);
+        const bool store = ((lane & 1) == 0) && (k < K);       // K is a multiple of 16: an even lane's word holds at least 16 codes
+        for (int i = 0; i < bits; ++i) {
+            const uint32_t h = ((((v.x >> i) & 0x01010101u) * 0x01020408u) >> 24) |
+                               (((((v.y >> i) & 0x01010101u) * 0x01020408u) >> 24) << 4) |
+                               (((((v.z >> i) & 0x01010101u) * 0x01020408u) >> 24) << 8) |
+                               (((((v.w >> i) & 0x01010101u) * 0x01020408u) >> 24) << 12);
+            const uint32_t other = __shfl_xor_sync(0xffffffffu, h, 1);
+            if (store) planes[i * plane_stride + r * ld_words + kw] = h | (other << 16);
+        }
+        if (row_sum != nullptr) {
+            int sum = __dp4a(v.x, 0x01010101u, 0u) + __dp4a(v.y, 0x01010101u, 0u) + __dp4a(v.z, 0x01010101u, 0u) +
+                      __dp4a(v.w, 0x01010101u, 0u);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
             if (lane == 0 && sum) atomicAdd(row_sum + r, sum);
@@ -369,9 +411,19 @@ int qnn_pack_planes_u8(const uint8_t *x, int64_t rows, int64_t K, int64_t ldx, i
     QNN_REQUIRE(x && planes, QNN_ERR_INVALID_ARG, "qnn_pack_planes_u8: NULL pointer");
     QNN_REQUIRE(ldx >= K && ld_words >= ceil_div(K, 32) && (bits == 1 || plane_stride_words >= rows * ld_words),
                 QNN_ERR_INVALID_ARG, "qnn_pack_planes_u8: leading dimension or plane stride too small");
+    cudaStream_t st = as_stream(stream);
+    if (K % 16 == 0 && ldx % 16 == 0 && aligned(x, 16)) {
+        if (row_sum_q) QNN_CUDA(cudaMemsetAsync(row_sum_q, 0, sizeof(int32_t) * (size_t)rows, st));
+        const int64_t chunks = ceil_div(K, 512);
+        const int64_t blocks_needed = ceil_div(rows * chunks, 8);
+        const int64_t cap = (int64_t)sm_count() * 8;
+        const int blocks = (int)(blocks_needed < cap ? blocks_needed : cap);
+        row_planes_u8_vec_kernel<<<blocks, 256, 0, st>>>(x, ldx, (1 << bits) - 1, rows, K, bits, planes, ld_words,
+                                                         plane_stride_words, row_sum_q, chunks);
+        return check_launch("qnn_pack_planes_u8");
+    }
     U8Src src{x, ldx, (1 << bits) - 1};
-    return launch_row_planes(src, rows, K, bits, planes, ld_words, plane_stride_words, row_sum_q, as_stream(stream),
-                             "qnn_pack_planes_u8");
+    return launch_row_planes(src, rows, K, bits, planes, ld_words, plane_stride_words, row_sum_q, st, "qnn_pack_planes_u8");
 }
 
 int qnn_quantize_pack_sign_t(const float *w, int64_t K, int64_t N, int64_t ldw, uint32_t *out, int64_t ld_words,
