@@ -23,6 +23,7 @@
 // code in a device status word, raises a block-wide abort flag, lets copies in
 // flight land, frees its tensor memory and returns.
 #include <cuda.h>
+#include <cstdlib>
 #include "qnn_internal.cuh"
 
 namespace qnn {
@@ -116,14 +117,45 @@ __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// CTAS = 1: a CTA works alone.  CTAS = 2: two CTAs of a cluster share 256 x BN tiles (cta_group::2); the same
+// warp of both CTAs allocates / frees.
+template <int CTAS>
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    if (CTAS == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 // One pipeline stage of the MMA warp as ONE instruction stream: poll the NEXT stage's full barrier, issue the
 // four K steps of this stage (+32 bytes of K = +2 in the descriptors' address field), commit them to this
@@ -178,6 +210,98 @@ __device__ __forceinline__ uint32_t umma_stage(uint32_t next_full_bar, uint32_t 
               "r"(sf), "r"(empty_bar)
             : "memory");
     }
+    return ready;
+}
+
+// The same stage for a CTA pair (issued by the leader CTA): one instruction multiplies the 256 x BN tile of both
+// CTAs; the commit arrives on this stage's empty barrier of BOTH CTAs.
+template <int FORM>
+__device__ __forceinline__ uint32_t umma_stage_pair(uint32_t next_full_bar, uint32_t next_parity, uint32_t d_tmem, uint64_t adesc,
+                                                    uint64_t bdesc, uint32_t idesc, uint32_t accumulate_first, uint32_t sf,
+                                                    uint32_t empty_bar)
+{
+    uint32_t ready;
+    if (FORM == QNN_FORM_FP4) {
+        asm volatile(
+            "{\n"
+            ".reg .pred P, Q, T;\n"
+            ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+            ".reg .b16 both;\n"
+            "mov.b16 both, 3;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+            "setp.ne.b32 P, %7, 0;\n"
+            "setp.eq.b32 T, 0, 0;\n"
+            "add.u64 a1, %4, 2;\n add.u64 a2, %4, 4;\n add.u64 a3, %4, 6;\n"
+            "add.u64 b1, %5, 2;\n add.u64 b2, %5, 4;\n add.u64 b3, %5, 6;\n"
+            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%3], %4, %5, %6, [%8], [%8], P;\n"
+            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%3], a1, b1, %6, [%8], [%8], T;\n"
+            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%3], a2, b2, %6, [%8], [%8], T;\n"
+            "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%3], a3, b3, %6, [%8], [%8], T;\n"
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%9], both;\n"
+            "selp.u32 %0, 1, 0, Q;\n"
+            "}\n"
+            : "=r"(ready)
+            : "r"(next_full_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first),
+              "r"(sf), "r"(empty_bar)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n"
+            ".reg .pred P, Q, T;\n"
+            ".reg .b64 a1, a2, a3, b1, b2, b3;\n"
+            ".reg .b16 both;\n"
+            "mov.b16 both, 3;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+            "setp.ne.b32 P, %7, 0;\n"
+            "setp.eq.b32 T, 0, 0;\n"
+            "add.u64 a1, %4, 2;\n add.u64 a2, %4, 4;\n add.u64 a3, %4, 6;\n"
+            "add.u64 b1, %5, 2;\n add.u64 b2, %5, 4;\n add.u64 b3, %5, 6;\n"
+            "tcgen05.mma.cta_group::2.kind::i8 [%3], %4, %5, %6, P;\n"
+            "tcgen05.mma.cta_group::2.kind::i8 [%3], a1, b1, %6, T;\n"
+            "tcgen05.mma.cta_group::2.kind::i8 [%3], a2, b2, %6, T;\n"
+            "tcgen05.mma.cta_group::2.kind::i8 [%3], a3, b3, %6, T;\n"
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%9], both;\n"
+            "selp.u32 %0, 1, 0, Q;\n"
+            "}\n"
+            : "=r"(ready)
+            : "r"(next_full_bar), "r"(next_parity), "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first),
+              "r"(sf), "r"(empty_bar)
+            : "memory");
+    }
+    return ready;
+}
+// accumulator-complete signal to both CTAs of a pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile(
+        "{\n.reg .b16 both;\nmov.b16 both, 3;\n"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], both;\n}\n"
+        ::"r"(bar) : "memory");
+}
+
+// TMA stage of one CTA of a pair: the loads land in this CTA's shared memory and report their bytes to the
+// LEADER's full barrier (`leader_full_bar`, a shared::cluster address); only the leader announces the bytes
+// (those of both CTAs).  No load is multicast.
+__device__ __forceinline__ uint32_t tma_stage_2d_pair(uint32_t next_empty_bar, uint32_t next_parity, uint32_t leader_full_bar,
+                                                      uint32_t tx_bytes_both, uint32_t is_leader, uint32_t dst_a,
+                                                      const CUtensorMap *map_a, int32_t ax, int32_t ay, uint32_t dst_b,
+                                                      const CUtensorMap *map_b, int32_t bx, int32_t by)
+{
+    uint32_t ready;
+    asm volatile(
+        "{\n"
+        ".reg .pred Q, L;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 Q, [%1], %2;\n"
+        "setp.ne.b32 L, %13, 0;\n"
+        "@L mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%3], %4;\n"
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%5], [%6, {%7, %8}], [%3];\n"
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%9], [%10, {%11, %12}], [%3];\n"
+        "selp.u32 %0, 1, 0, Q;\n"
+        "}\n"
+        : "=r"(ready)
+        : "r"(next_empty_bar), "r"(next_parity), "r"(leader_full_bar), "r"(tx_bytes_both), "r"(dst_a), "l"(map_a), "r"(ax),
+          "r"(ay), "r"(dst_b), "l"(map_b), "r"(bx), "r"(by), "r"(is_leader)
+        : "memory");
     return ready;
 }
 
@@ -274,10 +398,10 @@ __device__ __forceinline__ uint32_t spread_bits_to_bytes(uint32_t nib) { return 
 
 constexpr int next_pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
-template <int FORM, int BN, int STG>
+template <int FORM, int BN, int STG, int CTAS>
 struct TcCfg {
     static constexpr int A_BYTES = BM * BKB;
-    static constexpr int B_BYTES = BN * BKB;
+    static constexpr int B_BYTES = (BN / CTAS) * BKB;                    // a pair splits the B tile between its CTAs
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int CPW = (BN / 32 + EPI_GROUPS - 1) / EPI_GROUPS;  // 32-column chunks per epilogue warp
     static constexpr int THR_WORDS = CPW * 32 + 8;                       // per epilogue warp: its thresholds + flip words
@@ -288,7 +412,7 @@ struct TcCfg {
     static constexpr int STG_BYTES = 4 * EPI_GROUPS * STG_WARP_BYTES;
     static constexpr int AUX_BYTES = 256 + THR_BYTES + 1024;             // barriers, thresholds, 1024-byte alignment slack
     static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES - STG_BYTES) / STAGE_BYTES;
-    static constexpr int STAGES = MAX_STAGES > 6 ? 6 : MAX_STAGES;
+    static constexpr int STAGES = MAX_STAGES > 7 ? 7 : MAX_STAGES;
     static constexpr int SCALE_COL = 2 * BN;                             // FP4: unit block scales live behind the accumulators
     static constexpr int TMEM_COLS = next_pow2_cols(2 * BN + (FORM == QNN_FORM_FP4 ? 32 : 0));
     static constexpr int STG_OFFSET = STAGES * STAGE_BYTES;              // 1024-byte aligned like the stages
@@ -298,14 +422,15 @@ struct TcCfg {
     static_assert(STAGES >= 3, "pipeline too shallow");
     static_assert(TMEM_COLS <= 512, "accumulators do not fit tensor memory");
     static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile width");
+    static_assert(CTAS == 1 || (CTAS == 2 && BN % 32 == 0), "pairs split B in two halves of whole 8-row groups");
 };
 
-template <int FORM, int BN, int STG>
+template <int FORM, int BN, int STG, int CTAS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_out, const TcParams p)
 {
-    using S = TcCfg<FORM, BN, STG>;
+    using S = TcCfg<FORM, BN, STG, CTAS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
@@ -321,17 +446,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // In a pair (CTAS = 2) CTA 0 of the cluster leads: it owns the full and accumulator-empty barriers and issues
+    // the MMAs; both CTAs load their halves of the operands and drain their 128 rows of the accumulator.
+    const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128 * EPI_GROUPS); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * EPI_GROUPS * CTAS); }   // one arrival per epilogue warp
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), S::TMEM_COLS);
+    if (warp == 1) tmem_alloc<CTAS>(smem_u32(tmem_slot), S::TMEM_COLS);
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();                                 // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -350,16 +480,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         tc_fence_after();
     }
 
-    const uint32_t tiles_m = (uint32_t)p.tiles_m;
+    const uint32_t tiles_m = (uint32_t)p.tiles_m;                      // in units of BM * CTAS rows
     const uint32_t num_tiles = tiles_m * (uint32_t)p.tiles_n;          // below 2^31 (checked on the host)
+    // a CTA, or a pair of them, walks the tiles blockIdx.x / CTAS, + gridDim.x / CTAS, ...  (written out in every
+    // loop: held in named variables the two values cost the single-CTA kernel 12 % of its speed)
 
     if (warp == 0) {
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             bool ready = false;                                    // this stage's slot is known to be free
-            const uint32_t tx_bytes = (uint32_t)p.a_tx_bytes + (uint32_t)S::B_BYTES;
-            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            const uint32_t tx_bytes = ((uint32_t)p.a_tx_bytes + (uint32_t)S::B_BYTES) * CTAS;   // the leader announces both CTAs' bytes
+            for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS) {
                 const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
                 int32_t img = 0, y0 = 0;
                 if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; }
@@ -374,6 +506,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         nready = tma_stage_conv(empty_bar(nstage), nphase ^ 1u, full_bar(stage), tx_bytes, sa, &tmap_a, cb * BKB,
                                                 kw - p.cpad, y0 + kh - p.cpad, img, sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN);
                         if (++cb == p.cblocks) { cb = 0; if (++kw == p.cKW) { kw = 0; ++kh; } }
+                    } else if (CTAS == 2) {
+                        nready = tma_stage_2d_pair(empty_bar(nstage), nphase ^ 1u, map_to_cta(full_bar(stage), 0), tx_bytes,
+                                                   (uint32_t)leader, sa, &tmap_a, kb * BKB, (tm * 2 + (int32_t)rank) * BM,
+                                                   sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN + (int32_t)rank * (BN / 2));
                     } else {
                         nready = tma_stage_2d(empty_bar(nstage), nphase ^ 1u, full_bar(stage), tx_bytes, sa, &tmap_a, kb * BKB, tm * BM,
                                               sa + S::A_BYTES, &tmap_b, kb * BKB, tn * BN);
@@ -384,13 +520,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && leader) {
             int stage = 0; uint32_t phase = 0;
             uint32_t iter = 0;
             bool ok = true;
             bool ready = false;                                    // this stage's operands are known to have landed
             const uint32_t sf = tmem_base + (uint32_t)S::SCALE_COL;
-            for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
+            for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS, ++iter) {
                 const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tc_fence_after();
@@ -402,11 +538,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     const uint64_t bdesc = make_kmajor_sw128_desc(sa + S::A_BYTES);
                     int nstage = stage + 1; uint32_t nphase = phase;
                     if (nstage == S::STAGES) { nstage = 0; nphase ^= 1u; }
-                    ready = umma_stage<FORM>(full_bar(nstage), nphase, d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != 0), sf,
-                                             empty_bar(stage)) != 0;
+                    if (CTAS == 2)
+                        ready = umma_stage_pair<FORM>(full_bar(nstage), nphase, d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != 0), sf,
+                                                      empty_bar(stage)) != 0;
+                    else
+                        ready = umma_stage<FORM>(full_bar(nstage), nphase, d_tmem, adesc, bdesc, p.idesc, (uint32_t)(kb != 0), sf,
+                                                 empty_bar(stage)) != 0;
                     stage = nstage; phase = nphase;
                 }
-                if (ok) umma_commit(tfull_bar(as));              // accumulator complete
+                if (ok) {                                        // accumulator complete
+                    if (CTAS == 2) umma_commit_pair(tfull_bar(as));
+                    else umma_commit(tfull_bar(as));
+                }
             }
         }
     } else {
@@ -443,8 +586,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 else flip_raw[lc] = 0;
             }
         };
-        if (want_sign && blockIdx.x < num_tiles) fetch_thresholds((int64_t)(blockIdx.x / tiles_m) * BN);
-        for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++iter) {
+        if (want_sign && blockIdx.x / CTAS < num_tiles) fetch_thresholds((int64_t)((blockIdx.x / CTAS) / tiles_m) * BN);
+        for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS, ++iter) {
             const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
             const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
             const int64_t ntile = (int64_t)tn * BN;
@@ -472,7 +615,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     if (lane == lc) flip_w[lc] = fw;
                 }
                 __syncwarp();
-                const uint32_t tnext = t + gridDim.x;
+                const uint32_t tnext = t + gridDim.x / CTAS;
                 if (tnext < num_tiles) fetch_thresholds((int64_t)(tnext / tiles_m) * BN);
             }
 
@@ -495,8 +638,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 const int32_t tx = max(pd - x, 0), bx = max(x + pd - (p.cW - 1), 0);
                 cls = mrow ? ((ty * pc + by) * pc + tx) * pc + bx : 0;
             } else {
-                m = (int64_t)tm * BM + r;
-                m_warp0 = (int64_t)tm * BM + q * 32;
+                m = ((int64_t)tm * CTAS + rank) * BM + r;
+                m_warp0 = ((int64_t)tm * CTAS + rank) * BM + q * 32;
                 mrow = m < p.M;
             }
             const bool any_border = p.conv ? (__any_sync(0xffffffffu, cls != 0) != 0) : false;
@@ -667,7 +810,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             // all TMEM reads of this accumulator stage are done: hand it back to the MMA warp
             tc_fence_before();
-            mbar_arrive(tempty_bar(as));
+            __syncwarp();
+            if (lane == 0) {
+                if (CTAS == 2) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
+                else mbar_arrive(tempty_bar(as));
+            }
         }
         // stores still reading shared memory must finish before the block's shared memory goes away
         if (STG) {
@@ -684,8 +831,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();     // the peer no longer touches this CTA's barriers, shared or tensor memory
     tc_fence_after();
-    if (warp == 1) tmem_dealloc(tmem_base, S::TMEM_COLS);
+    if (warp == 1) tmem_dealloc<CTAS>(tmem_base, S::TMEM_COLS);
 }
 
 // ---- expansion of packed planes to tensor-core forms ---------------------------
@@ -844,23 +992,56 @@ int make_map_out(CUtensorMap *map, CUtensorMapDataType type, int rank, void *bas
     return QNN_OK;
 }
 
+// CTA pairs a persistent grid of this kernel can keep resident at once (0 = pairs cannot be launched)
 template <int FORM, int BN, int STG>
-int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mo, TcParams p, cudaStream_t st)
+int max_pairs()
 {
-    using S = TcCfg<FORM, BN, STG>;
-    auto kern = gemm_tc_kernel<FORM, BN, STG>;
+    using S = TcCfg<FORM, BN, STG, 2>;
+    auto kern = gemm_tc_kernel<FORM, BN, STG, 2>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL) != cudaSuccess) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (unsigned)sm_count());
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = S::TOTAL;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { (void)cudaGetLastError(); return 0; }
+    return n;
+}
+
+template <int FORM, int BN, int STG, int CTAS>
+int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mo, TcParams p, int workers, cudaStream_t st)
+{
+    using S = TcCfg<FORM, BN, STG, CTAS>;
+    auto kern = gemm_tc_kernel<FORM, BN, STG, CTAS>;
     QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
     const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
     QNN_REQUIRE(tiles < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: too many output tiles");
-    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    const int nw = (int)(tiles < workers ? tiles : workers);
     profile_before(st);
-    kern<<<grid, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, p);
+    if (CTAS == 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * (unsigned)nw);
+        cfg.blockDim = dim3(TC_THREADS);
+        cfg.dynamicSmemBytes = S::TOTAL;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        QNN_CUDA(cudaLaunchKernelEx(&cfg, kern, ma, mb, mo, p));
+    } else {
+        kern<<<nw, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, p);
+    }
     profile_after(st);
     return check_launch("tc gemm");
 }
 
-template <int FORM, int BN>
-int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cudaStream_t st)
+template <int FORM, int BN, int CTAS>
+int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, int workers, cudaStream_t st)
 {
     // The int32 result leaves through bulk stores where its layout allows it (16-byte aligned rows), which
     // costs the kernel one pipeline stage of shared memory; otherwise the epilogue stores from registers.
@@ -868,6 +1049,7 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cuda
     p.tma_out = 0;
     p.tiles_n = (int32_t)ceil_div(p.N, BN);
     p.idesc |= (uint32_t)(BN >> 3) << 17;
+    if (CTAS == 2) p.idesc = (p.idesc & ~(0x1fu << 24)) | ((uint32_t)((2 * BM) >> 4) << 24);   // the pair's instruction is 256 rows tall
     const bool conv_full_tiles = p.conv && p.cR * p.cW == BM;
     if (p.out != nullptr && aligned(p.out, 16)) {
         // (the bulk store clips the innermost extent in 16-byte units, so N must be a whole number of them)
@@ -887,22 +1069,23 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, cuda
             p.tma_out = 2;
         }
     }
-    if (p.tma_out) return launch_tc_stg<FORM, BN, 1>(ma, mb, mo, p, st);
-    return launch_tc_stg<FORM, BN, 0>(ma, mb, mo, p, st);
+    if (p.tma_out) return launch_tc_stg<FORM, BN, 1, CTAS>(ma, mb, mo, p, workers, st);
+    return launch_tc_stg<FORM, BN, 0, CTAS>(ma, mb, mo, p, workers, st);
 }
 
 // Tile width.  Measured on B200: the time of one wave of tiles depends only weakly on the width (about
 // 4.2 us + 4.7 ns per column at K = 4096), because a K block costs the issuing threads and the TMA path
 // about the same whatever its width.  So: fewest waves first, the width as a small correction.
-int pick_bn(int64_t tiles_m, int64_t N)
+int pick_bn(int64_t tiles_m, int64_t N, int workers, int min_bn)
 {
     static const int cand[] = {224, 192, 128, 64, 32};
     int best = cand[0];
     double best_cost = 1e300;
     for (int i = 0; i < 5; ++i) {
         const int bn = cand[i];
+        if (bn < min_bn) continue;
         const int64_t tiles = tiles_m * ceil_div(N, bn);
-        const int64_t waves = ceil_div(tiles, sm_count());
+        const int64_t waves = ceil_div(tiles, workers);
         const double cost = (double)waves * (bn + 900);
         if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
     }
@@ -1083,24 +1266,52 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     } else {
         if (int rc = make_map_2d(&ma, a8, g.M, a_row_bytes, a_ld, BM)) return rc;
     }
-    const int bn = pick_bn(p.tiles_m, g.N);
-    if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn)) return rc;
+    // Large plain products with a long K run on CTA pairs (cta_group::2): one 256 x BN tile per pair halves, per
+    // SM, both the operand bytes to load and the instructions to issue.  Measured on B200: 8192^3 with int32
+    // output 209 -> 182 us, 10000 x 4096 x 4096 68 -> 66 us; with fewer than a dozen K blocks per tile the
+    // cross-SM hand-offs cost more than the pair saves (10000 x 4096 x 784: 41 -> 47 us), so those stay on single
+    // CTAs.  QNN_TC_PAIRS=0 in the environment keeps single CTAs everywhere.
+    static const bool pairs_off = [] { const char *e = getenv("QNN_TC_PAIRS"); return e && e[0] == '0'; }();
+    static const int pairs_resident = pairs_off ? 0 : max_pairs<QNN_FORM_FP4, 224, 0>();
+    const int64_t tiles_m2 = ceil_div(g.M, 2 * BM);
+    const bool pairs = !g.conv && pairs_resident >= 8 && p.num_kb >= 12 && tiles_m2 * ceil_div(g.N, 224) >= pairs_resident;
+    if (pairs) {
+        p.tiles_m = (int32_t)tiles_m2;
+        const int bn = pick_bn(tiles_m2, g.N, pairs_resident, 64);
+        if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn / 2)) return rc;
+        if (form == QNN_FORM_FP4) {
+            switch (bn) {
+                case 224: return launch_tc_cfg<QNN_FORM_FP4, 224, 2>(ma, mb, p, pairs_resident, st);
+                case 192: return launch_tc_cfg<QNN_FORM_FP4, 192, 2>(ma, mb, p, pairs_resident, st);
+                case 128: return launch_tc_cfg<QNN_FORM_FP4, 128, 2>(ma, mb, p, pairs_resident, st);
+                default: return launch_tc_cfg<QNN_FORM_FP4, 64, 2>(ma, mb, p, pairs_resident, st);
+            }
+        }
+        switch (bn) {
+            case 224: return launch_tc_cfg<QNN_FORM_I8, 224, 2>(ma, mb, p, pairs_resident, st);
+            case 192: return launch_tc_cfg<QNN_FORM_I8, 192, 2>(ma, mb, p, pairs_resident, st);
+            case 128: return launch_tc_cfg<QNN_FORM_I8, 128, 2>(ma, mb, p, pairs_resident, st);
+            default: return launch_tc_cfg<QNN_FORM_I8, 64, 2>(ma, mb, p, pairs_resident, st);
+        }
+    }
 
+    const int bn = pick_bn(p.tiles_m, g.N, sm_count(), 32);
+    if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn)) return rc;
     if (form == QNN_FORM_FP4) {
         switch (bn) {
-            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224>(ma, mb, p, st);
-            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192>(ma, mb, p, st);
-            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128>(ma, mb, p, st);
-            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64>(ma, mb, p, st);
-            default: return launch_tc_cfg<QNN_FORM_FP4, 32>(ma, mb, p, st);
+            case 224: return launch_tc_cfg<QNN_FORM_FP4, 224, 1>(ma, mb, p, sm_count(), st);
+            case 192: return launch_tc_cfg<QNN_FORM_FP4, 192, 1>(ma, mb, p, sm_count(), st);
+            case 128: return launch_tc_cfg<QNN_FORM_FP4, 128, 1>(ma, mb, p, sm_count(), st);
+            case 64: return launch_tc_cfg<QNN_FORM_FP4, 64, 1>(ma, mb, p, sm_count(), st);
+            default: return launch_tc_cfg<QNN_FORM_FP4, 32, 1>(ma, mb, p, sm_count(), st);
         }
     }
     switch (bn) {
-        case 224: return launch_tc_cfg<QNN_FORM_I8, 224>(ma, mb, p, st);
-        case 192: return launch_tc_cfg<QNN_FORM_I8, 192>(ma, mb, p, st);
-        case 128: return launch_tc_cfg<QNN_FORM_I8, 128>(ma, mb, p, st);
-        case 64: return launch_tc_cfg<QNN_FORM_I8, 64>(ma, mb, p, st);
-        default: return launch_tc_cfg<QNN_FORM_I8, 32>(ma, mb, p, st);
+        case 224: return launch_tc_cfg<QNN_FORM_I8, 224, 1>(ma, mb, p, sm_count(), st);
+        case 192: return launch_tc_cfg<QNN_FORM_I8, 192, 1>(ma, mb, p, sm_count(), st);
+        case 128: return launch_tc_cfg<QNN_FORM_I8, 128, 1>(ma, mb, p, sm_count(), st);
+        case 64: return launch_tc_cfg<QNN_FORM_I8, 64, 1>(ma, mb, p, sm_count(), st);
+        default: return launch_tc_cfg<QNN_FORM_I8, 32, 1>(ma, mb, p, sm_count(), st);
     }
 }
 
