@@ -355,8 +355,12 @@ QNN_API int qnn_mlp_forward(const uint8_t *x, int64_t M, int in_bits, const qnn_
 
 /* Same, for callers holding HOST buffers: copies x_host (pinned memory
  * recommended) to the device, runs the layers, copies the scores back to
- * scores_host and synchronises `stream`.  The workspace must also hold the
- * input and the scores: size it with qnn_mlp_workspace_bytes(..., 1). */
+ * scores_host and synchronises `stream`.  Batch rows are independent, so large
+ * batches are cut into 2 chunks whose input copies (on a copy stream the
+ * library creates once per device and keeps) overlap the previous chunk's
+ * layers; the copies start after the work already queued on `stream`.  The
+ * workspace must also hold the input and the scores: size it with
+ * qnn_mlp_workspace_bytes(..., 1). */
 QNN_API int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, const qnn_mlp_layer *layers,
                          int L, int32_t *scores_host, int algo, void *ws, size_t ws_bytes,
                          void *stream);

@@ -1017,7 +1017,14 @@ int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMa
 {
     using S = TcCfg<FORM, BN, STG, CTAS>;
     auto kern = gemm_tc_kernel<FORM, BN, STG, CTAS>;
-    QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
+    // the shared-memory opt-in is per kernel and device: asked for once, not on every launch (it costs microseconds)
+    static bool opted_in[64] = {};
+    int dev = 0;
+    QNN_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+        QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
+        if (dev >= 0 && dev < 64) opted_in[dev] = true;
+    }
     const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
     QNN_REQUIRE(tiles < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: too many output tiles");
     const int nw = (int)(tiles < workers ? tiles : workers);

@@ -3,6 +3,7 @@
 // activations ping-ponging between two workspace buffers, int32 scores last.
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include "qnn_internal.cuh"
 
 namespace qnn {
@@ -182,6 +183,21 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
     return QNN_OK;
 }
 
+// One non-blocking stream per device for the host entry point's input copies, created on first use and kept.
+cudaStream_t copy_stream()
+{
+    static std::mutex mu;
+    static cudaStream_t streams[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (streams[dev] == nullptr && cudaStreamCreateWithFlags(&streams[dev], cudaStreamNonBlocking) != cudaSuccess) {
+        (void)cudaGetLastError();
+        streams[dev] = nullptr;
+    }
+    return streams[dev];
+}
+
 }  // namespace
 }  // namespace qnn
 
@@ -227,11 +243,49 @@ int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, const qn
     char *base = static_cast<char *>(ws);
     uint8_t *x_dev = reinterpret_cast<uint8_t *>(base + p.off_x);
     int32_t *s_dev = reinterpret_cast<int32_t *>(base + p.off_scores);
-    const size_t in_bytes = (size_t)M * (size_t)layers[0].K;
-    const size_t out_bytes = sizeof(int32_t) * (size_t)M * (size_t)layers[L - 1].N;
-    QNN_CUDA(cudaMemcpyAsync(x_dev, x_host, in_bytes, cudaMemcpyHostToDevice, st));
-    if (int rc = run_mlp(x_dev, M, in_bits, layers, L, s_dev, algo, base, p, st)) return rc;
-    QNN_CUDA(cudaMemcpyAsync(scores_host, s_dev, out_bytes, cudaMemcpyDeviceToHost, st));
+    const int64_t K0 = layers[0].K, NL = layers[L - 1].N;
+
+    // Batch rows are independent, so the batch is cut into chunks whose host-to-device copies (on a copy stream
+    // of the library's own) run while the previous chunk is being computed on the caller's stream.
+    const int chunks = M >= 4096 ? 2 : 1;      // (more chunks cost more in launches than they hide in copies)
+    cudaStream_t cs = chunks > 1 ? copy_stream() : nullptr;
+    if (chunks == 1 || cs == nullptr) {
+        QNN_CUDA(cudaMemcpyAsync(x_dev, x_host, (size_t)M * (size_t)K0, cudaMemcpyHostToDevice, st));
+        if (int rc = run_mlp(x_dev, M, in_bits, layers, L, s_dev, algo, base, p, st)) return rc;
+    } else {
+        const int64_t rows_c = (int64_t)round_up((size_t)ceil_div(M, chunks), 256);   // whole 256-row tiles per chunk
+        cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+        int rc = QNN_OK;
+        for (int c = 0; c <= chunks && rc == QNN_OK; ++c)
+            if (cudaEventCreateWithFlags(&ev[c], cudaEventDisableTiming) != cudaSuccess) rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: cudaEventCreate failed");
+        if (rc == QNN_OK) {
+            // the copies start after whatever the caller already queued on its stream
+            if (cudaEventRecord(ev[chunks], st) != cudaSuccess || cudaStreamWaitEvent(cs, ev[chunks], 0) != cudaSuccess)
+                rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: stream ordering failed");
+        }
+        for (int c = 0; c < chunks && rc == QNN_OK; ++c) {
+            const int64_t r0 = c * rows_c, rows = (r0 + rows_c <= M ? rows_c : M - r0);
+            if (rows <= 0) break;
+            if (cudaMemcpyAsync(x_dev + r0 * K0, x_host + r0 * K0, (size_t)rows * (size_t)K0, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+                cudaEventRecord(ev[c], cs) != cudaSuccess)
+                rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: chunk copy failed");
+        }
+        for (int c = 0; c < chunks && rc == QNN_OK; ++c) {
+            const int64_t r0 = c * rows_c, rows = (r0 + rows_c <= M ? rows_c : M - r0);
+            if (rows <= 0) break;
+            if (cudaStreamWaitEvent(st, ev[c], 0) != cudaSuccess) { rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: stream wait failed"); break; }
+            rc = run_mlp(x_dev + r0 * K0, rows, in_bits, layers, L, s_dev + r0 * NL, algo, base, p, st);
+        }
+        if (rc != QNN_OK) {
+            cudaStreamSynchronize(cs);
+            cudaStreamSynchronize(st);
+        }
+        // (events may be destroyed while work that uses them is pending: the runtime frees them when it is done)
+        for (int c = 0; c <= chunks; ++c)
+            if (ev[c]) cudaEventDestroy(ev[c]);
+        if (rc != QNN_OK) return rc;
+    }
+    QNN_CUDA(cudaMemcpyAsync(scores_host, s_dev, sizeof(int32_t) * (size_t)M * (size_t)NL, cudaMemcpyDeviceToHost, st));
     QNN_CUDA(cudaStreamSynchronize(st));
     return QNN_OK;
 }
