@@ -197,3 +197,53 @@ def test_tc_gemm_argument_errors(q):
     with pytest.raises(q.QnnError) as ei:
         q.qnn_tc_gemm(q.tc_operand(t, 16, q.QNN_FORM_FP4, planes=3), a, 2, 2, 32, o, 2)
     assert ei.value.status == q.QNN_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("form_name,M,N,K", [("FP4", 4100, 1000, 4100), ("FP4", 5000, 777, 3104), ("I8", 4400, 900, 1600)])
+@pytest.mark.parametrize("outputs", ["int", "sign"])
+def test_tc_gemm_cta_pair_shapes(q, form_name, M, N, K, outputs):
+    """Ragged shapes large enough (and with K long enough) for the product to run on CTA pairs: 256-row tiles whose
+    second half hangs over the end of M, a last column tile of a few columns, a partial last K block.  The oracle
+    runs on sampled rows (every row position inside a pair's tile is hit) and row-sum checksums cover all outputs."""
+    form = getattr(q, "QNN_FORM_" + form_name)
+    rng = np.random.default_rng(M + N + K)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+    ld = words_per_row(K)
+    a = as_i32_words(pack_bits_ref((X >= 0).astype(np.uint8), ld)).cuda()
+    b = as_i32_words(pack_bits_ref((W >= 0).astype(np.uint8).T, ld)).cuda()
+    rb = q.qnn_tc_row_bytes(K, form)
+    af = torch.empty(M, rb, dtype=torch.uint8, device="cuda")
+    bf = torch.empty(N, rb, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(a, 1, 1, ld, 0, M, K, form, af, rb)
+    q.qnn_tc_prepack(b, 1, 1, ld, 0, N, K, form, bf, rb)
+    rows = np.unique(np.concatenate([np.arange(0, 260), np.arange(M - 300, M), rng.integers(0, M, 64)]))
+    want = oracle.xnor_gemm(X[rows], W)
+    A, B = q.tc_operand(af, rb, form), q.tc_operand(bf, rb, form)
+    if outputs == "int":
+        out = Guarded((M, N), torch.int32, fill=-7)
+        q.qnn_tc_gemm(A, B, M, N, K, out.t, N)
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        got = out.t.cpu().numpy()
+        np.testing.assert_array_equal(got[rows], want)
+        sa = np.where(X >= 0, 1, -1).astype(np.int64)
+        sw = np.where(W >= 0, 1, -1).astype(np.int64)
+        np.testing.assert_array_equal(got.sum(axis=1, dtype=np.int64), sa @ sw.sum(axis=1))
+        out.check()
+    else:
+        T = rng.integers(-30, 31, N).astype(np.int32)
+        flip = rng.integers(0, 2, N).astype(np.uint8)
+        ldw = words_per_row(N)
+        bits = Guarded((M, ldw), torch.int32, fill=0)
+        orb = q.qnn_tc_row_bytes(N, q.QNN_FORM_FP4)
+        of = Guarded((M, orb), torch.uint8, fill=0x5C)
+        q.qnn_tc_gemm(A, B, M, N, K, thr=dev(T), flip=dev(flip), out_bits=bits.t, ld_words=ldw, out_form=of.t,
+                      out_form_kind=q.QNN_FORM_FP4, ld_form_bytes=orb)
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        wb = oracle.threshold(want, T, flip)
+        np.testing.assert_array_equal(unpack_words(words_np(bits.t)[rows], N), wb)
+        onb = words_per_row(N) * 16
+        np.testing.assert_array_equal(of.t.cpu().numpy()[rows][:, :onb], form_ref(2 * wb.astype(np.int32) - 1, N, q.QNN_FORM_FP4, q))
+        bits.check(); of.check()
