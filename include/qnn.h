@@ -320,6 +320,40 @@ QNN_API int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, con
                       const int32_t *thr, const uint8_t *flip, uint32_t *out_bits, int algo, void *ws,
                       size_t ws_bytes, void *stream);
 
+/* Filter banks prepared once (static weights) for the tensor-core convolution.
+ * Applies to stride-1 "same" filters (KH = KW = 2 * pad + 1, at most 7 x 7) with
+ * C a multiple of 128 and images at most 128 pixels wide; qnn_conv_form(C) is the
+ * form such a layer multiplies in (QNN_FORM_FP4 for C % 256 == 0, else
+ * QNN_FORM_I8; 0 = not available: use qnn_binary_conv2d).
+ * qnn_conv_prepare rewrites w (qnn_pack_conv_weights layout) in that form and
+ * appends the table of what the padding value contributes per border position;
+ * `prepared` is a 256-byte aligned device buffer of qnn_conv_prepared_bytes. */
+QNN_API int qnn_conv_form(int C);
+QNN_API size_t qnn_conv_prepared_bytes(int Cout, int C, int KH, int KW, int pad);
+QNN_API int qnn_conv_prepare(const uint32_t *w, int Cout, int C, int KH, int KW, int pad, int pad_bit,
+                             void *prepared, size_t prepared_bytes, void *stream);
+
+typedef struct qnn_conv_io {
+    const void *x;        /* x_form 0: packed NHWC bits [B,H,W,ceil(C/32)] words;
+                             x_form = qnn_conv_form(C): NHWC values in that form, pixels
+                             32*ceil(C/32) elements apart (dense)                        */
+    int x_form;
+    int32_t *out_nchw;    /* int32 [B,Cout,H,W] or NULL                                  */
+    const int32_t *thr;   /* int32 [Cout], needed for out_bits / out_form               */
+    const uint8_t *flip;  /* uint8 [Cout] or NULL                                        */
+    uint32_t *out_bits;   /* packed NHWC bits [B,H,W,ceil(Cout/32)] or NULL              */
+    void *out_form;       /* the same signs as NHWC values in out_form_kind (dense), the
+                             next convolution's x, or NULL                               */
+    int out_form_kind;
+} qnn_conv_io;
+
+/* Section 5 with a prepared filter bank: same result as qnn_binary_conv2d
+ * (stride 1, the pad and pad_bit given to qnn_conv_prepare).  A workspace of
+ * B*H*W * 32*ceil(C/32) bytes (int8 form; half for e2m1) is needed only when x is
+ * given as packed bits. */
+QNN_API int qnn_binary_conv2d_prepared(const qnn_conv_io *io, int B, int C, int H, int W, const void *prepared,
+                                       int Cout, int KH, int KW, int pad, void *ws, size_t ws_bytes, void *stream);
+
 /* ------------------------------------------------------------------------- */
 /* Algorithm 4 runner                                                         */
 /* ------------------------------------------------------------------------- */

@@ -52,6 +52,11 @@ class qnn_tc_output(ctypes.Structure):
                 ("out_form", vp), ("out_form_kind", i32), ("ld_form_bytes", i64)]
 
 
+class qnn_conv_io(ctypes.Structure):
+    _fields_ = [("x", vp), ("x_form", i32), ("out_nchw", vp), ("thr", vp), ("flip", vp), ("out_bits", vp),
+                ("out_form", vp), ("out_form_kind", i32)]
+
+
 class qnn_mlp_layer(ctypes.Structure):
     _fields_ = [("w", vp), ("ldw", i64), ("K", i64), ("N", i64), ("thr", vp), ("flip", vp),
                 ("w_tc", vp), ("w_tc_ld", i64), ("w_tc_form", i32)]
@@ -84,6 +89,10 @@ _SIGS = {
     "qnn_fold_bn": (i32, [vp, vp, vp, vp, ctypes.c_double, i64, vp, vp]),
     "qnn_rescale_f32": (i32, [vp, i64, i64, i64, f32, vp, vp, f32, vp, i64, vp]),
     "qnn_binary_conv2d": (i32, [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, vp, sz, vp]),
+    "qnn_conv_form": (i32, [i32]),
+    "qnn_conv_prepared_bytes": (sz, [i32, i32, i32, i32, i32]),
+    "qnn_conv_prepare": (i32, [vp, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
+    "qnn_binary_conv2d_prepared": (i32, [ctypes.POINTER(qnn_conv_io), i32, i32, i32, i32, vp, i32, i32, i32, i32, vp, sz, vp]),
     "qnn_mlp_forward": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
     "qnn_mlp_forward_host": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
     "qnn_mlp_layer_form": (i32, [ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
@@ -242,6 +251,27 @@ def qnn_binary_conv2d(x, B, C, H, W, w, Cout, KH, KW, stride, pad, pad_bit, out_
     wp, wb = _ws(ws)
     _ck(_lib.qnn_binary_conv2d(_p(x), B, C, H, W, _p(w), Cout, KH, KW, stride, pad, pad_bit, _p(out_nchw), _p(thr),
                                _p(flip), _p(out_bits), algo, wp, wb, _stream()), "qnn_binary_conv2d")
+
+
+def qnn_conv_form(C) -> int:
+    return int(_lib.qnn_conv_form(C))
+
+
+def qnn_conv_prepared_bytes(Cout, C, KH, KW, pad) -> int:
+    return int(_lib.qnn_conv_prepared_bytes(Cout, C, KH, KW, pad))
+
+
+def qnn_conv_prepare(w, Cout, C, KH, KW, pad, pad_bit, prepared):
+    _ck(_lib.qnn_conv_prepare(_p(w), Cout, C, KH, KW, pad, pad_bit, _p(prepared), prepared.numel() * prepared.element_size(),
+                              _stream()), "qnn_conv_prepare")
+
+
+def qnn_binary_conv2d_prepared(x, x_form, B, C, H, W, prepared, Cout, KH, KW, pad, out_nchw=None, thr=None, flip=None,
+                               out_bits=None, out_form=None, out_form_kind=0, ws=None):
+    io = qnn_conv_io(_p(x), x_form, _p(out_nchw), _p(thr), _p(flip), _p(out_bits), _p(out_form), out_form_kind)
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_binary_conv2d_prepared(ctypes.byref(io), B, C, H, W, _p(prepared), Cout, KH, KW, pad, wp, wb, _stream()),
+        "qnn_binary_conv2d_prepared")
 
 
 def make_mlp_layers(ws: Sequence[torch.Tensor], ldws: Sequence[int], Ks: Sequence[int], Ns: Sequence[int],

@@ -76,31 +76,35 @@ __global__ void __launch_bounds__(256) rescale_kernel(const int32_t *__restrict_
 // fall off the left / right: cls = ((ty*(pad+1) + by)*(pad+1) + tx)*(pad+1) + bx.
 // corr[cls, co] = (+-1) * sum over out-of-image taps of sum_c w[co, c, tap]; rows are ld = Cout rounded up to 32
 // long, the pad columns zero.
-__global__ void __launch_bounds__(256) conv_border_corr_kernel(const uint32_t *__restrict__ w, int Cout, int C, int KH, int KW,
+__global__ void __launch_bounds__(128) conv_border_corr_kernel(const uint32_t *__restrict__ w, int Cout, int C, int KH, int KW,
                                                                int pad, int pad_bit, int32_t *__restrict__ corr, int classes, int ld)
 {
+    // one block per output channel (and per pad column): first the sum of every tap's weights, then the classes
+    __shared__ int32_t tap_sum[64];
+    const int co = blockIdx.x;
+    const int taps = KH * KW;
+    if (co >= Cout) {
+        for (int cls = threadIdx.x; cls < classes; cls += blockDim.x) corr[cls * ld + co] = 0;
+        return;
+    }
     const int Cw = (C + 31) >> 5;
+    for (int t = threadIdx.x; t < taps; t += blockDim.x) tap_sum[t] = 0;
+    __syncthreads();
+    const uint32_t *wp = w + (int64_t)co * taps * Cw;
+    for (int e = threadIdx.x; e < taps * Cw; e += blockDim.x) atomicAdd(&tap_sum[e / Cw], 2 * __popc(__ldg(wp + e)));
+    __syncthreads();
     const int pc = pad + 1;
-    const int total = classes * ld;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < total; e += gridDim.x * blockDim.x) {
-        const int co = e % ld;
-        int cls = e / ld;
-        if (co >= Cout) { corr[e] = 0; continue; }
+    for (int c0 = threadIdx.x; c0 < classes; c0 += blockDim.x) {
+        int cls = c0;
         const int bx = cls % pc; cls /= pc;
         const int tx = cls % pc; cls /= pc;
         const int by = cls % pc; cls /= pc;
         const int ty = cls;
         int32_t sum = 0;
         for (int kh = 0; kh < KH; ++kh)
-            for (int kw = 0; kw < KW; ++kw) {
-                const bool oob = kh < ty || kh >= KH - by || kw < tx || kw >= KW - bx;
-                if (!oob) continue;
-                const uint32_t *wp = w + ((int64_t)co * KH * KW + kh * KW + kw) * Cw;
-                int32_t ones = 0;
-                for (int cw = 0; cw < Cw; ++cw) ones += __popc(__ldg(wp + cw));
-                sum += 2 * ones - C;
-            }
-        corr[e] = pad_bit ? sum : -sum;
+            for (int kw = 0; kw < KW; ++kw)
+                if (kh < ty || kh >= KH - by || kw < tx || kw >= KW - bx) sum += tap_sum[kh * KW + kw] - C;
+        corr[c0 * ld + co] = pad_bit ? sum : -sum;
     }
 }
 
@@ -109,6 +113,41 @@ inline int grid_for(int64_t total)
     const int64_t need = ceil_div(total, 256);
     const int64_t cap = (int64_t)sm_count() * 16;
     return (int)(need < cap ? need : cap);
+}
+
+// Where the prepared form of a filter bank lives: weights in tensor-core form, then the border table.
+struct ConvPrep {
+    int form;
+    int64_t kwords, w_pitch;
+    int classes, corr_ld;
+    size_t w_bytes, c_bytes;
+};
+
+// The implicit tensor-core path takes stride-1 "same" filters (at most 7 x 7: 64 taps), images at most 128 pixels wide
+// and whole 128-byte channel blocks per pixel: 256 channels as e2m1 values, 128 as int8.  want_form = 0: the best form.
+bool conv_prep_layout(int Cout, int C, int KH, int KW, int pad, int want_form, ConvPrep *l)
+{
+    if (KH != 2 * pad + 1 || KW != 2 * pad + 1 || pad > 3 || (int64_t)KH * KW * C >= (1 << 24)) return false;
+    int form = 0;
+    if (C % 256 == 0 && want_form != QNN_FORM_I8) form = QNN_FORM_FP4;
+    else if (C % 128 == 0 && want_form != QNN_FORM_FP4) form = QNN_FORM_I8;
+    if (form == 0) return false;
+    l->form = form;
+    l->kwords = (int64_t)KH * KW * ceil_div(C, 32);
+    l->w_pitch = tc_row_pitch(l->kwords, form);
+    l->classes = (pad + 1) * (pad + 1) * (pad + 1) * (pad + 1);
+    l->corr_ld = (int)round_up((size_t)Cout, 32);
+    l->w_bytes = round_up((size_t)Cout * (size_t)l->w_pitch, 256);
+    l->c_bytes = round_up(sizeof(int32_t) * (size_t)l->classes * (size_t)l->corr_ld, 256);
+    return true;
+}
+
+int conv_prepare_into(const uint32_t *w, int Cout, int C, int KH, int KW, int pad, int pad_bit, const ConvPrep &l, uint8_t *wf,
+                      int32_t *corr, cudaStream_t st)
+{
+    if (int rc = tc_expand(w, 1, QNN_MODE_PM1, l.kwords, 0, Cout, l.kwords, l.kwords, 32, l.form, wf, l.w_pitch, st)) return rc;
+    conv_border_corr_kernel<<<l.corr_ld, 128, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, l.classes, l.corr_ld);
+    return check_launch("conv border table");
 }
 
 }  // namespace
@@ -167,49 +206,34 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
     g.thr = thr; g.flip = flip; g.out_bits = out_bits; g.ld_bits = ceil_div(Cout, 32);
 
     // ---- implicit GEMM on the tensor cores: no im2col matrix ------------------------------------
-    // Needs a stride-1 "same" filter, an image row that fits a 128-pixel tile and whole 128-byte
-    // channel blocks per pixel (256 channels as e2m1 values, 128 as int8).
-    int form = 0;
-    if (stride == 1 && KH == 2 * pad + 1 && KW == 2 * pad + 1 && pad <= 3 && W <= 128 && (int64_t)KH * KW * C < (1 << 24)) {
-        if (C % 256 == 0 && algo != QNN_ALGO_TC_I8) form = QNN_FORM_FP4;
-        else if (C % 128 == 0 && algo != QNN_ALGO_TC_FP4) form = QNN_FORM_I8;
-    }
-    if (algo == QNN_ALGO_AUTO) {
+    ConvPrep lay{};
+    bool implicit = stride == 1 && W <= 128 && algo != QNN_ALGO_POPC && algo != QNN_ALGO_B1_MMA &&
+                    conv_prep_layout(Cout, C, KH, KW, pad, algo == QNN_ALGO_TC_I8 ? QNN_FORM_I8 : (algo == QNN_ALGO_TC_FP4 ? QNN_FORM_FP4 : 0), &lay);
+    if (implicit && algo == QNN_ALGO_AUTO) {
         const int pick = qnn_select_algo(M, Cout, g.K, 1, 1, QNN_MODE_PM1, QNN_MODE_PM1);
-        if (pick != QNN_ALGO_TC_FP4 && pick != QNN_ALGO_TC_I8) form = 0;
-    } else if (algo == QNN_ALGO_POPC || algo == QNN_ALGO_B1_MMA) {
-        form = 0;
+        implicit = pick == QNN_ALGO_TC_FP4 || pick == QNN_ALGO_TC_I8;
     }
-    if (form != 0) {
-        const int64_t cbytes = tc_row_bytes(Cw, form);
-        const int classes = (pad + 1) * (pad + 1) * (pad + 1) * (pad + 1);
+    if (implicit) {
+        const int64_t cbytes = tc_row_bytes(Cw, lay.form);
         const size_t x_bytes = round_up((size_t)M * (size_t)cbytes, 256);
-        const int64_t w_pitch = tc_row_pitch(kwords, form);
-        const size_t w_bytes = round_up((size_t)Cout * (size_t)w_pitch, 256);
-        const int corr_ld = (int)round_up((size_t)Cout, 32);
-        const size_t c_bytes = round_up(sizeof(int32_t) * (size_t)classes * (size_t)corr_ld, 256);
-        if (ws != nullptr && aligned(ws, 256) && ws_bytes >= x_bytes + w_bytes + c_bytes) {
+        if (ws != nullptr && aligned(ws, 256) && ws_bytes >= x_bytes + lay.w_bytes + lay.c_bytes) {
             uint8_t *xf = static_cast<uint8_t *>(ws);
             uint8_t *wf = xf + x_bytes;
-            int32_t *corr = reinterpret_cast<int32_t *>(wf + w_bytes);
-            g.a_tc = xf; g.a_tc_form = form; g.a_tc_ld = cbytes;
-            g.b_tc = wf; g.b_tc_form = form; g.b_tc_ld = w_pitch;
+            int32_t *corr = reinterpret_cast<int32_t *>(wf + lay.w_bytes);
+            g.a_tc = xf; g.a_tc_form = lay.form; g.a_tc_ld = cbytes;
+            g.b_tc = wf; g.b_tc_form = lay.form; g.b_tc_ld = lay.w_pitch;
             if (int rc = validate_gemm(g)) return rc;
-            if (int rc = tc_expand(x, 1, QNN_MODE_PM1, Cw, 0, M, Cw, Cw, 32, form, xf, cbytes, st)) return rc;
-            if (int rc = tc_expand(w, 1, QNN_MODE_PM1, kwords, 0, Cout, kwords, kwords, 32, form, wf, w_pitch, st))
-                return rc;
-            conv_border_corr_kernel<<<grid_for((int64_t)classes * corr_ld), 256, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, classes,
-                                                                                           corr_ld);
-            if (int rc = check_launch("qnn_binary_conv2d border table")) return rc;
+            if (int rc = tc_expand(x, 1, QNN_MODE_PM1, Cw, 0, M, Cw, Cw, 32, lay.form, xf, cbytes, st)) return rc;
+            if (int rc = conv_prepare_into(w, Cout, C, KH, KW, pad, pad_bit, lay, wf, corr, st)) return rc;
             ConvImplicit ci{};
             ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;
             ci.cblocks = (int32_t)(cbytes / 128);
             ci.corr = corr;
             g.conv = &ci;
-            return launch_gemm_tc(g, form, nullptr, 0, st);
+            return launch_gemm_tc(g, lay.form, nullptr, 0, st);
         }
         QNN_REQUIRE(algo == QNN_ALGO_AUTO, QNN_ERR_WORKSPACE,
-                    "qnn_binary_conv2d: workspace of at least %zu bytes (256-byte aligned) required", x_bytes + w_bytes + c_bytes);
+                    "qnn_binary_conv2d: workspace of at least %zu bytes (256-byte aligned) required", x_bytes + lay.w_bytes + lay.c_bytes);
     }
 
     // ---- packed im2col + matrix product ------------------------------------------------------------
@@ -224,6 +248,85 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
     im2col_bits_kernel<<<grid_for(total), 256, 0, st>>>(x, B, C, H, W, KH, KW, stride, pad, pad_bit, Ho, Wo, col, total);
     if (int rc = check_launch("qnn_binary_conv2d im2col")) return rc;
     return run_gemm(g, algo, static_cast<char *>(ws) + col_bytes, ws_bytes - col_bytes, st);
+}
+
+size_t qnn_conv_prepared_bytes(int Cout, int C, int KH, int KW, int pad)
+{
+    ConvPrep l{};
+    if (Cout <= 0 || C <= 0 || !conv_prep_layout(Cout, C, KH, KW, pad, 0, &l)) return 0;
+    return l.w_bytes + l.c_bytes;
+}
+
+int qnn_conv_prepare(const uint32_t *w, int Cout, int C, int KH, int KW, int pad, int pad_bit, void *prepared, size_t prepared_bytes,
+                     void *stream)
+{
+    QNN_REQUIRE(w && prepared, QNN_ERR_INVALID_ARG, "qnn_conv_prepare: NULL pointer");
+    QNN_REQUIRE(Cout >= 1 && C >= 1 && (pad_bit == 0 || pad_bit == 1), QNN_ERR_INVALID_ARG, "qnn_conv_prepare: bad sizes or pad_bit");
+    ConvPrep l{};
+    QNN_REQUIRE(conv_prep_layout(Cout, C, KH, KW, pad, 0, &l), QNN_ERR_UNSUPPORTED,
+                "qnn_conv_prepare: needs a stride-1 'same' filter up to 7 x 7 and C a multiple of 128; use qnn_binary_conv2d");
+    QNN_REQUIRE(aligned(prepared, 256) && prepared_bytes >= l.w_bytes + l.c_bytes, QNN_ERR_WORKSPACE,
+                "qnn_conv_prepare: buffer of at least %zu bytes (256-byte aligned) required", l.w_bytes + l.c_bytes);
+    uint8_t *wf = static_cast<uint8_t *>(prepared);
+    return conv_prepare_into(w, Cout, C, KH, KW, pad, pad_bit, l, wf, reinterpret_cast<int32_t *>(wf + l.w_bytes), as_stream(stream));
+}
+
+int qnn_conv_form(int C)
+{
+    return C > 0 && C % 256 == 0 ? QNN_FORM_FP4 : (C > 0 && C % 128 == 0 ? QNN_FORM_I8 : 0);
+}
+
+int qnn_binary_conv2d_prepared(const qnn_conv_io *io, int B, int C, int H, int W, const void *prepared, int Cout, int KH, int KW,
+                               int pad, void *ws, size_t ws_bytes, void *stream)
+{
+    QNN_REQUIRE(io != nullptr && prepared != nullptr, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: NULL descriptor");
+    QNN_REQUIRE(B >= 0 && C >= 1 && H >= 0 && W >= 0 && Cout >= 1, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: bad size");
+    if (B == 0 || H == 0 || W == 0) return QNN_OK;
+    ConvPrep l{};
+    QNN_REQUIRE(conv_prep_layout(Cout, C, KH, KW, pad, 0, &l) && W <= 128, QNN_ERR_UNSUPPORTED,
+                "qnn_binary_conv2d_prepared: needs a stride-1 'same' filter up to 7 x 7, C a multiple of 128 and W <= 128");
+    QNN_REQUIRE(io->x != nullptr, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: NULL input");
+    QNN_REQUIRE(io->x_form == 0 || io->x_form == l.form, QNN_ERR_INVALID_ARG,
+                "qnn_binary_conv2d_prepared: input form %d, but this filter bank multiplies in form %d", io->x_form, l.form);
+    QNN_REQUIRE(io->out_nchw || io->out_bits || io->out_form, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: no output buffer");
+    QNN_REQUIRE(!(io->out_bits || io->out_form) || io->thr, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: thresholds required");
+    cudaStream_t st = as_stream(stream);
+    const int64_t Cw = ceil_div(C, 32);
+    const int64_t M = (int64_t)B * H * W;
+    const int64_t cbytes = tc_row_bytes(Cw, l.form);
+    const uint8_t *wf = static_cast<const uint8_t *>(prepared);
+
+    GemmArgs g{};
+    g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;
+    g.M = M; g.N = Cout; g.K = (int64_t)KH * KW * C; g.kwords = l.kwords;
+    g.pad_period = Cw; g.pad_tail = 32;
+    g.epilogue = EPI_NCHW; g.out = io->out_nchw; g.hw = (int64_t)H * W;
+    g.thr = io->thr; g.flip = io->flip; g.out_bits = io->out_bits; g.ld_bits = ceil_div(Cout, 32);
+    if (io->out_form) {
+        g.out_form = io->out_form; g.out_form_kind = io->out_form_kind;
+        g.ld_form = tc_row_bytes(ceil_div(Cout, 32), io->out_form_kind);      // dense NHWC: the next layer's pixels
+    }
+    g.b_tc = wf; g.b_tc_form = l.form; g.b_tc_ld = l.w_pitch;
+    if (io->x_form != 0) {
+        g.a_tc = io->x;
+    } else {
+        const size_t x_bytes = round_up((size_t)M * (size_t)cbytes, 256);
+        QNN_REQUIRE(ws != nullptr && aligned(ws, 256) && ws_bytes >= x_bytes, QNN_ERR_WORKSPACE,
+                    "qnn_binary_conv2d_prepared: workspace of at least %zu bytes (256-byte aligned) required", x_bytes);
+        g.a_tc = ws;
+    }
+    g.a_tc_form = l.form; g.a_tc_ld = cbytes;
+    if (int rc = validate_gemm(g)) return rc;
+    if (io->x_form == 0)
+        if (int rc = tc_expand(static_cast<const uint32_t *>(io->x), 1, QNN_MODE_PM1, Cw, 0, M, Cw, Cw, 32, l.form,
+                               static_cast<uint8_t *>(ws), cbytes, st))
+            return rc;
+    ConvImplicit ci{};
+    ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;
+    ci.cblocks = (int32_t)(cbytes / 128);
+    ci.corr = reinterpret_cast<const int32_t *>(wf + l.w_bytes);
+    g.conv = &ci;
+    return launch_gemm_tc(g, l.form, nullptr, 0, st);
 }
 
 }  // extern "C"

@@ -275,3 +275,85 @@ def test_square_large_sampled_and_checksums(q, n, algo):
     sw = oracle.sign(W).astype(np.int64)
     np.testing.assert_array_equal(got.sum(axis=1, dtype=np.int64), sa @ sw.sum(axis=1))
     np.testing.assert_array_equal(got.sum(axis=0, dtype=np.int64), sa.sum(axis=0) @ sw)
+
+
+@pytest.mark.parametrize("B,C,H,W,Co,KS,pad_bit", [(2, 256, 16, 16, 256, 3, 1), (2, 128, 13, 12, 70, 3, 0), (1, 256, 7, 20, 33, 5, 1),
+                                                  (3, 512, 8, 8, 128, 1, 1)])
+@pytest.mark.parametrize("x_as_form", [False, True])
+def test_conv2d_prepared_filter_bank(q, B, C, H, W, Co, KS, pad_bit, x_as_form):
+    """Filter bank prepared once (tensor-core form + border table), input as packed bits or already in form;
+    int32, packed-bit and form outputs of one call against the oracle."""
+    pad = KS // 2
+    rng = np.random.default_rng(B + C + H + Co + KS)
+    X = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    Wt = rng.uniform(-1, 1, (Co, C, KS, KS)).astype(np.float32)
+    T = rng.integers(-16, 17, Co).astype(np.int32)
+    flip = rng.integers(0, 2, Co).astype(np.uint8)
+    want = oracle.conv2d(oracle.sign(X), oracle.sign(Wt), 1, pad, 1 if pad_bit else -1)
+    cw = words_per_row(C)
+    xb = torch.zeros(B, H, W, cw, dtype=torch.int32, device="cuda")
+    wb = torch.zeros(Co, KS * KS * cw, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_sign_nchw(dev(X), B, C, H, W, xb)
+    q.qnn_pack_conv_weights(dev(Wt), Co, C, KS, KS, wb)
+    form = q.qnn_conv_form(C)
+    assert form in (q.QNN_FORM_FP4, q.QNN_FORM_I8)
+    prep = torch.empty(q.qnn_conv_prepared_bytes(Co, C, KS, KS, pad), dtype=torch.uint8, device="cuda")
+    q.qnn_conv_prepare(wb, Co, C, KS, KS, pad, pad_bit, prep)
+    pix_bytes = cw * (32 if form == q.QNN_FORM_I8 else 16)
+    x_arg, x_form, ws = xb, 0, torch.empty(B * H * W * pix_bytes + 256, dtype=torch.uint8, device="cuda")
+    if x_as_form:
+        xf = torch.empty(B * H * W, pix_bytes, dtype=torch.uint8, device="cuda")
+        q.qnn_tc_prepack(xb, 1, q.QNN_MODE_PM1, cw, 0, B * H * W, C, form, xf, pix_bytes)
+        x_arg, x_form, ws = xf, form, None
+    out = Guarded((B, Co, H, W), torch.int32, fill=-7)
+    bits = Guarded((B, H, W, words_per_row(Co)), torch.int32, fill=0)
+    oform = q.QNN_FORM_FP4
+    onb = words_per_row(Co) * 16
+    of = Guarded((B * H * W, onb), torch.uint8, fill=0x5C)
+    q.qnn_binary_conv2d_prepared(x_arg, x_form, B, C, H, W, prep, Co, KS, KS, pad, out.t, dev(T), dev(flip), bits.t, of.t,
+                                 oform, ws)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    np.testing.assert_array_equal(out.t.cpu().numpy(), want)
+    rows = want.transpose(0, 2, 3, 1).reshape(-1, Co)
+    wbits = oracle.threshold(rows, T, flip)
+    np.testing.assert_array_equal(unpack_words(words_np(bits.t).reshape(-1, words_per_row(Co)), Co), wbits)
+    # form output: e2m1 nibbles of the thresholded signs, pad columns zero
+    E2M1 = {0: 0x0, 1: 0x2, -1: 0xA}
+    vals = np.zeros((rows.shape[0], words_per_row(Co) * 32), np.int32)
+    vals[:, :Co] = 2 * wbits.astype(np.int32) - 1
+    nib = np.vectorize(E2M1.__getitem__)(vals).astype(np.uint8)
+    np.testing.assert_array_equal(of.t.cpu().numpy(), (nib[:, 0::2] | (nib[:, 1::2] << 4)).astype(np.uint8))
+    for gbuf in (out, bits, of):
+        gbuf.check()
+
+
+def test_conv2d_prepared_chain_two_layers(q):
+    """conv -> threshold -> conv with the activations handed over in tensor-core form (no packed bits in between)."""
+    rng = np.random.default_rng(5)
+    B, C, H, W, C1, C2 = 2, 256, 8, 8, 256, 40
+    X = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    W1 = rng.uniform(-1, 1, (C1, C, 3, 3)).astype(np.float32)
+    W2 = rng.uniform(-1, 1, (C2, C1, 3, 3)).astype(np.float32)
+    T = rng.integers(-16, 17, C1).astype(np.int32)
+    s1 = oracle.conv2d(oracle.sign(X), oracle.sign(W1), 1, 1, 1)
+    h = np.where(s1 >= T[None, :, None, None], 1, -1).astype(np.int32)
+    want = oracle.conv2d(h, oracle.sign(W2), 1, 1, 1)
+    FP4 = q.QNN_FORM_FP4
+    xb = torch.zeros(B, H, W, C // 32, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_sign_nchw(dev(X), B, C, H, W, xb)
+    preps = []
+    for Wt, (co, ci) in ((W1, (C1, C)), (W2, (C2, C1))):
+        wb = torch.zeros(co, 9 * ci // 32, dtype=torch.int32, device="cuda")
+        q.qnn_pack_conv_weights(dev(Wt), co, ci, 3, 3, wb)
+        pr = torch.empty(q.qnn_conv_prepared_bytes(co, ci, 3, 3, 1), dtype=torch.uint8, device="cuda")
+        q.qnn_conv_prepare(wb, co, ci, 3, 3, 1, 1, pr)
+        preps.append(pr)
+    hf = torch.empty(B * H * W, C1 // 2, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(B * H * W * C // 2 + 256, dtype=torch.uint8, device="cuda")
+    q.qnn_binary_conv2d_prepared(xb, 0, B, C, H, W, preps[0], C1, 3, 3, 1, thr=dev(T), out_form=hf, out_form_kind=FP4, ws=ws)
+    out = torch.empty(B, C2, H, W, dtype=torch.int32, device="cuda")
+    q.qnn_binary_conv2d_prepared(hf, FP4, B, C1, H, W, preps[1], C2, 3, 3, 1, out_nchw=out)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), want)
