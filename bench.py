@@ -315,6 +315,18 @@ def run_extras(q, bench, peaks, algo):
     ms, best = _time_op(lambda: q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, out, N, algo, ws), flush)
     rec("c1_xnor_gemm_100x4096x4096", ms, best, bytes_=(M + N) * ld * 4 + M * N * 4, ops=2.0 * M * N * K)
 
+    # static weights rewritten once in tensor-core form (qnn_tc_prepack); per call only the activations are
+    form = q.qnn_tc_form(1, q.QNN_MODE_PM1, 1, q.QNN_MODE_PM1, K)
+    rb = q.qnn_tc_row_bytes(K, form)
+    wf = torch.empty(N, rb, dtype=torch.uint8, device="cuda"); af = torch.empty(M, rb, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(b, 1, q.QNN_MODE_PM1, ld, 0, N, K, form, wf, rb)
+
+    def warm_prepacked():
+        q.qnn_tc_prepack(a, 1, q.QNN_MODE_PM1, ld, 0, M, K, form, af, rb)
+        q.qnn_tc_gemm(q.tc_operand(af, rb, form), q.tc_operand(wf, rb, form), M, N, K, out, N)
+    ms, best = _time_op(warm_prepacked, flush)
+    rec("c1_xnor_gemm_100x4096x4096_prepacked_weights", ms, best, bytes_=(M + N) * ld * 4 + M * N * 4, ops=2.0 * M * N * K)
+
     def cold():
         q.qnn_quantize_pack_sign(Xd, M, K, K, a, ld)
         q.qnn_quantize_pack_sign_t(Wd, K, N, N, b, ld)
@@ -353,6 +365,16 @@ def run_extras(q, bench, peaks, algo):
         ms, best = _time_op(lambda: q.qnn_bitplane_gemm(ap, 2, q.QNN_MODE_U01, ld, M * ld, bp, 1, q.QNN_MODE_PM1, ld, 0,
                                                         M, N, K, o, N, algo, w3), flush)
         rec(f"c3_fc{6 + i}_2bit_x_1bit_{M}x{N}x{K}", ms, best, ops=2.0 * M * N * K * 2)
+        f3 = q.qnn_tc_form(2, q.QNN_MODE_U01, 1, q.QNN_MODE_PM1, K)
+        rb3 = q.qnn_tc_row_bytes(K, f3)
+        wf3 = torch.empty(N, rb3, dtype=torch.uint8, device="cuda"); af3 = torch.empty(M, rb3, dtype=torch.uint8, device="cuda")
+        q.qnn_tc_prepack(bp, 1, q.QNN_MODE_PM1, ld, 0, N, K, f3, wf3, rb3)
+
+        def fc_prepacked():
+            q.qnn_tc_prepack(ap, 2, q.QNN_MODE_U01, ld, M * ld, M, K, f3, af3, rb3)
+            q.qnn_tc_gemm(q.tc_operand(af3, rb3, f3, 2, q.QNN_MODE_U01), q.tc_operand(wf3, rb3, f3), M, N, K, o, N)
+        ms, best = _time_op(fc_prepacked, flush)
+        rec(f"c3_fc{6 + i}_prepacked_weights", ms, best, ops=2.0 * M * N * K * 2)
 
     # config 4: CIFAR conv
     wl4 = workloads.cifar_conv()
@@ -372,6 +394,17 @@ def run_extras(q, bench, peaks, algo):
     rec("c4_conv3x3_int32_out", ms, best, ops=ops4)
     ms, best = _time_op(lambda: q.qnn_binary_conv2d(xb, B, C, H, Wd_, wb, Co, 3, 3, 1, 1, 1, None, t4, None, ob, algo, w4), flush)
     rec("c4_conv3x3_threshold_bits_out", ms, best, ops=ops4)
+    prep = torch.empty(q.qnn_conv_prepared_bytes(Co, C, 3, 3, 1), dtype=torch.uint8, device="cuda")
+    q.qnn_conv_prepare(wb, Co, C, 3, 3, 1, 1, prep)
+    f4 = q.qnn_conv_form(C)
+    xf4 = torch.empty(B * H * Wd_, q.qnn_tc_row_bytes(C, f4), dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(xb, 1, q.QNN_MODE_PM1, C // 32, 0, B * H * Wd_, C, f4, xf4, xf4.shape[1])
+    of4 = torch.empty(B * H * Wd_, q.qnn_tc_row_bytes(Co, f4), dtype=torch.uint8, device="cuda")
+    ms, best = _time_op(lambda: q.qnn_binary_conv2d_prepared(xb, 0, B, C, H, Wd_, prep, Co, 3, 3, 1, out_nchw=o4, ws=w4), flush)
+    rec("c4_conv3x3_prepared_filters_int32_out", ms, best, ops=ops4)
+    ms, best = _time_op(lambda: q.qnn_binary_conv2d_prepared(xf4, f4, B, C, H, Wd_, prep, Co, 3, 3, 1, thr=t4, out_form=of4,
+                                                              out_form_kind=f4), flush)
+    rec("c4_conv3x3_prepared_filters_form_in_form_out", ms, best, ops=ops4, note="mid-network layer: activations arrive and leave in tensor-core form")
 
     # config 5: LSTM gate 4b x 4b and the square sweep
     wl5 = workloads.lstm_gate()
