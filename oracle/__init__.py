@@ -18,6 +18,11 @@ Pins (what each routine is checked against, other than itself) live in
   conv2d          library conv2d in float64 on +-1 tensors padded with +1,
                   the 1x1 case against the matrix product, all-ones input
   mlp_forward     Algorithm 4 step by step with the routines above
+  maxpool2x2      library max_pool2d in float64; the identity that pooling the
+                  integer sums and then thresholding equals OR (AND where the
+                  comparison is flipped) of the thresholded bits, by brute force
+  convnet_forward Table 7 layer by layer against a float64 library chain
+                  (conv2d, max_pool2d, comparisons)
   rescale         float64 numpy expression
 """
 from __future__ import annotations
@@ -191,6 +196,48 @@ def conv2d(X, Wt, stride: int = 1, pad: int = 1, pad_value: int = 1) -> np.ndarr
     rc = _load().qo_conv2d(_ptr(X), _ptr(Wt), B, C, H, W, Cout, KH, KW, stride, pad, pad_value, _ptr(out))
     _check(rc, "conv2d")
     return out
+
+
+def maxpool2x2(x) -> np.ndarray:
+    """2 x 2 / stride 2 max-pooling of an int32 [B,C,H,W] tensor (Table 7); odd tails dropped."""
+    x = _c(x, np.int32)
+    B, C, H, W = x.shape
+    out = np.empty((B, C, H // 2, W // 2), np.int32)
+    _check(_load().qo_maxpool2x2(_ptr(x), B, C, H, W, _ptr(out)), "maxpool2x2")
+    return out
+
+
+def convnet_forward(x, layers) -> np.ndarray:
+    """The ConvNet of Table 7 at inference, in the table's order: convolution, (2 x 2 max-pooling,)
+    batch norm folded to a threshold, binarisation; then the fully connected layers of Algorithm 4.
+
+    x: integer codes [B,C,H,W] (8-bit pixels).  layers: dicts with
+      kind 'conv': W +-1 int32 [Cout,C,k,k], pad, pad_value (what a tap outside the image reads:
+                   0 for the pixel codes of the first layer, +1 for +-1 activations), pool (bool)
+      kind 'fc'  : W +-1 int32 [K,N]; the first one reads the last feature map flattened in
+                   (h, w, c) order
+      T, flip    : folded thresholds of the layer; T None on the last layer (integer scores).
+    Returns the last layer's int32 result."""
+    a = _c(x, np.int32)
+    for i, ly in enumerate(layers):
+        if ly["kind"] == "conv":
+            s = conv2d(a, ly["W"], 1, ly["pad"], ly["pad_value"])
+            if ly.get("pool"):
+                s = maxpool2x2(s)
+            if ly.get("T") is None:
+                return s
+            Bq, Co, Ho, Wo = s.shape
+            rows = s.transpose(0, 2, 3, 1).reshape(-1, Co)
+            bits = threshold(rows, ly["T"], ly.get("flip"))
+            a = np.where(bits.reshape(Bq, Ho, Wo, Co) != 0, 1, -1).astype(np.int32).transpose(0, 3, 1, 2)
+        else:
+            if a.ndim == 4:
+                a = a.transpose(0, 2, 3, 1).reshape(a.shape[0], -1)
+            s = int_gemm(a, ly["W"])
+            if ly.get("T") is None:
+                return s
+            a = np.where(threshold(s, ly["T"], ly.get("flip")) != 0, 1, -1).astype(np.int32)
+    return a
 
 
 def mlp_forward(x, Ws: Sequence[np.ndarray], Ts: Sequence[np.ndarray],

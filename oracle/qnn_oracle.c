@@ -223,6 +223,26 @@ int qo_conv2d(const int32_t *X, const int32_t *Wt, int B, int C, int H, int W, i
     return overflow;
 }
 
+/* 2 x 2 max-pooling with stride 2 of an int32 [B,C,H,W] tensor, the pooling that
+ * Table 7 places between a convolution and its batch norm.  A trailing odd row
+ * or column is dropped: out is [B,C,H/2,W/2] (integer division). */
+int qo_maxpool2x2(const int32_t *x, int B, int C, int H, int W, int32_t *out)
+{
+    if (B < 0 || C < 0 || H < 0 || W < 0) return 2;
+    const int Ho = H / 2, Wo = W / 2;
+    for (int64_t bc = 0; bc < (int64_t)B * C; ++bc)
+        for (int y = 0; y < Ho; ++y)
+            for (int xo = 0; xo < Wo; ++xo) {
+                const int32_t *p = x + (bc * H + 2 * y) * W + 2 * xo;
+                int32_t m = p[0];
+                if (p[1] > m) m = p[1];
+                if (p[W] > m) m = p[W];
+                if (p[W + 1] > m) m = p[W + 1];
+                out[(bc * Ho + y) * Wo + xo] = m;
+            }
+    return 0;
+}
+
 /* Algorithm 4 in full for an MLP whose input is an unsigned integer code
  * (8-bit pixels in the paper):
  *   layer 1:      a_1 = x . W_1            (integer x, +-1 weights; Eq. 8)

@@ -117,6 +117,50 @@ def cifar_conv(B: int = 128, C: int = 256, H: int = 16, W: int = 16, Cout: int =
     return ConvWorkload(X, Wt, T, 1, 1)
 
 
+@dataclass
+class ConvNetWorkload:
+    """The CIFAR-10 ConvNet of Table 7: 8-bit RGB images, three pairs of 3x3 'same' convolutions
+    (the second of each pair followed by 2x2 max-pooling), then fully connected layers."""
+    X: torch.Tensor                     # [B, 3, H, W] uint8
+    conv_W: List[torch.Tensor]          # fp32 [Cout, C, 3, 3], to be sign-binarised
+    conv_pool: List[bool]               # 2x2 max-pooling after this convolution
+    fc_W: List[torch.Tensor]            # fp32 [K, N]; the first reads the feature map in (h, w, c) order
+    Ts: List[torch.Tensor]              # int32 thresholds, one per layer but the last
+    flips: List[torch.Tensor]           # uint8 0/1 per channel, same layers
+
+
+def cifar_convnet(B: int = 128, H: int = 32, W: int = 32, widths: Tuple[int, ...] = (128, 128, 256, 256, 512, 512),
+                  fc: Tuple[int, ...] = (1024, 1024, 10), in_ch: int = 3, seed: int = 5, stream: int = 0,
+                  flip_share: float = 0.25) -> ConvNetWorkload:
+    """Weights, thresholds and flips come from stream 0, the images from ``stream``.  Thresholds of the
+    pooled layers are centred near the typical maximum of four sums (about sqrt(K)) so that the bits stay mixed."""
+    gw = _gen(seed, 0)
+    X = torch.randint(0, 256, (B, in_ch, H, W), generator=gw, dtype=torch.uint8)
+    conv_W, conv_pool, Ts, flips = [], [], [], []
+    c, h, w = in_ch, H, W
+    for i, co in enumerate(widths):
+        conv_W.append(_uniform_pm1(gw, co, c, 3, 3))
+        pool = (i % 2 == 1)
+        conv_pool.append(pool)
+        shift = int(round((9 * c) ** 0.5)) if pool else 0
+        Ts.append(_thresholds(gw, co) + shift)
+        flips.append((torch.rand(co, generator=gw) < flip_share).to(torch.uint8))
+        c = co
+        if pool:
+            h, w = h // 2, w // 2
+    k = c * h * w
+    fc_W = []
+    for j, n in enumerate(fc):
+        fc_W.append(_uniform_pm1(gw, k, n))
+        if j < len(fc) - 1:
+            Ts.append(_thresholds(gw, n))
+            flips.append((torch.rand(n, generator=gw) < flip_share).to(torch.uint8))
+        k = n
+    if stream != 0:
+        X = torch.randint(0, 256, (B, in_ch, H, W), generator=_gen(seed, stream), dtype=torch.uint8)
+    return ConvNetWorkload(X, conv_W, conv_pool, fc_W, Ts, flips)
+
+
 def square_gemm(n: int, seed: int = 4) -> FcLayer:
     """Square binary GEMM M=N=K=n with N(0,1) operands (the paper timed 8192^3)."""
     g = _gen(seed, n)

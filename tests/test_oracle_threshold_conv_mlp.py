@@ -106,6 +106,98 @@ def test_mlp_flip():
     np.testing.assert_array_equal(got, want)
 
 
+@pytest.mark.parametrize("B,C,H,W", [(2, 3, 4, 6), (1, 5, 7, 5), (3, 1, 2, 2), (1, 2, 3, 4)])
+def test_maxpool_vs_library(B, C, H, W):
+    rng = np.random.default_rng(H * 10 + W)
+    x = rng.integers(-500, 500, (B, C, H, W)).astype(np.int32)
+    want = F.max_pool2d(torch.from_numpy(x).double(), 2).numpy().astype(np.int32)
+    got = oracle.maxpool2x2(x)
+    assert got.shape == (B, C, H // 2, W // 2)
+    np.testing.assert_array_equal(got, want)
+    assert oracle.maxpool2x2(x[:, :, :1, :]).shape == (B, C, 0, W // 2)      # a single row has no window
+
+
+def test_threshold_of_pooled_sums_is_or_and_of_bits():
+    """Thresholding is monotone in the sum, so the bit of a window's maximum is the OR of the four
+    pixels' bits, and the AND where the channel's comparison is flipped (every window checked)."""
+    rng = np.random.default_rng(11)
+    B, C, H, W = 2, 6, 6, 8
+    s = rng.integers(-20, 20, (B, C, H, W)).astype(np.int32)
+    T = rng.integers(-10, 10, C).astype(np.int32)
+    flip = np.array([0, 1, 0, 1, 1, 0], np.uint8)
+    rows = lambda t: t.transpose(0, 2, 3, 1).reshape(-1, C)
+    pooled_bits = oracle.threshold(rows(oracle.maxpool2x2(s)), T, flip).reshape(B, H // 2, W // 2, C)
+    bits = oracle.threshold(rows(s), T, flip).reshape(B, H, W, C)
+    for b in range(B):
+        for y in range(H // 2):
+            for x in range(W // 2):
+                win = bits[b, 2 * y:2 * y + 2, 2 * x:2 * x + 2, :].reshape(4, C)
+                for c in range(C):
+                    want = win[:, c].min() if flip[c] else win[:, c].max()
+                    assert pooled_bits[b, y, x, c] == want
+
+
+def test_first_layer_conv_on_pixel_codes_vs_library():
+    """8-bit codes times +-1 weights with a zero border (Table 7's first layer; Eq. 8 summed over planes)."""
+    rng = np.random.default_rng(5)
+    x = rng.integers(0, 256, (2, 3, 6, 5)).astype(np.int32)
+    w = np.where(rng.standard_normal((4, 3, 3, 3)) >= 0, 1, -1).astype(np.int32)
+    want = F.conv2d(torch.from_numpy(x).double(), torch.from_numpy(w).double(), padding=1).numpy()
+    got = oracle.conv2d(x, w, 1, 1, 0)
+    np.testing.assert_array_equal(got, want.astype(np.int32))
+    # plane by plane (Eq. 8): the same sums from the eight bit planes of the codes
+    acc = np.zeros_like(got)
+    for i in range(8):
+        acc += (1 << i) * oracle.conv2d(oracle.bit_plane(x, i).astype(np.int32), w, 1, 1, 0)
+    np.testing.assert_array_equal(acc, got)
+
+
+def _convnet_layers(wl):
+    layers, t = [], 0
+    for i, (Wc, pool) in enumerate(zip(wl.conv_W, wl.conv_pool)):
+        layers.append(dict(kind="conv", W=oracle.sign(Wc.numpy()), pad=1, pad_value=0 if i == 0 else 1, pool=pool,
+                           T=wl.Ts[t].numpy(), flip=wl.flips[t].numpy()))
+        t += 1
+    for j, Wf in enumerate(wl.fc_W):
+        last = j == len(wl.fc_W) - 1
+        layers.append(dict(kind="fc", W=oracle.sign(Wf.numpy()), T=None if last else wl.Ts[t].numpy(),
+                           flip=None if last else wl.flips[t].numpy()))
+        t += 0 if last else 1
+    return layers
+
+
+def test_convnet_forward_vs_library_chain():
+    """Table 7 layer by layer with float64 library calls: conv2d on a padded tensor, max_pool2d, comparisons."""
+    wl = workloads.cifar_convnet(B=3, H=8, W=8, widths=(8, 8, 16, 16), fc=(24, 10), seed=5)
+    layers = _convnet_layers(wl)
+    got = oracle.convnet_forward(wl.X.numpy().astype(np.int32), layers)
+    a = wl.X.double()
+    for ly in layers:
+        if ly["kind"] == "conv":
+            ap = F.pad(a, (1, 1, 1, 1), value=float(ly["pad_value"]))
+            s = F.conv2d(ap, torch.from_numpy(ly["W"]).double())
+            if ly["pool"]:
+                s = F.max_pool2d(s, 2)
+            ge = s >= torch.from_numpy(ly["T"]).double()[None, :, None, None]
+            bit = ge ^ (torch.from_numpy(ly["flip"]) != 0)[None, :, None, None]
+            a = torch.where(bit, 1.0, -1.0).double()
+        else:
+            if a.dim() == 4:
+                a = a.permute(0, 2, 3, 1).reshape(a.shape[0], -1)
+            s = a @ torch.from_numpy(ly["W"]).double()
+            if ly["T"] is not None:
+                bit = (s >= torch.from_numpy(ly["T"]).double()[None, :]) ^ (torch.from_numpy(ly["flip"]) != 0)[None, :]
+                a = torch.where(bit, 1.0, -1.0).double()
+    assert got.shape == (3, 10)
+    np.testing.assert_array_equal(got, s.numpy().astype(np.int32))
+    # the chain is live: changing one pixel changes the scores
+    x2 = wl.X.numpy().astype(np.int32).copy()
+    x2[:, :, 0, 0] = 255 - x2[:, :, 0, 0]
+    assert not np.array_equal(oracle.convnet_forward(x2, layers), got)
+    # both kinds of channel occur, so both the OR and the AND side of pooling are exercised
+    assert any(f.any() for f in wl.flips) and any((f == 0).any() for f in wl.flips)
+
+
 def test_rescale():
     rng = np.random.default_rng(1)
     p = rng.integers(-1000, 1000, (4, 6)).astype(np.int32)
