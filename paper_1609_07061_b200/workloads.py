@@ -131,9 +131,9 @@ class ConvNetWorkload:
 
 def cifar_convnet(B: int = 128, H: int = 32, W: int = 32, widths: Tuple[int, ...] = (128, 128, 256, 256, 512, 512),
                   fc: Tuple[int, ...] = (1024, 1024, 10), in_ch: int = 3, seed: int = 5, stream: int = 0,
-                  flip_share: float = 0.25) -> ConvNetWorkload:
-    """Weights, thresholds and flips come from stream 0, the images from ``stream``.  Thresholds of the
-    pooled layers are centred near the typical maximum of four sums (about sqrt(K)) so that the bits stay mixed."""
+                  flip_share: float = 0.25, thr: int = 64) -> ConvNetWorkload:
+    """Weights, thresholds and flips come from stream 0, the images from ``stream``.  Thresholds are uniform in [-thr, thr]
+    (narrow layers need a small thr to keep the bits data dependent); those of the pooled layers are centred near the typical maximum of four sums (about sqrt(K)) so that the bits stay mixed."""
     gw = _gen(seed, 0)
     X = torch.randint(0, 256, (B, in_ch, H, W), generator=gw, dtype=torch.uint8)
     conv_W, conv_pool, Ts, flips = [], [], [], []
@@ -143,7 +143,7 @@ def cifar_convnet(B: int = 128, H: int = 32, W: int = 32, widths: Tuple[int, ...
         pool = (i % 2 == 1)
         conv_pool.append(pool)
         shift = int(round((9 * c) ** 0.5)) if pool else 0
-        Ts.append(_thresholds(gw, co) + shift)
+        Ts.append(_thresholds(gw, co, -thr, thr) + shift)
         flips.append((torch.rand(co, generator=gw) < flip_share).to(torch.uint8))
         c = co
         if pool:
@@ -153,7 +153,7 @@ def cifar_convnet(B: int = 128, H: int = 32, W: int = 32, widths: Tuple[int, ...
     for j, n in enumerate(fc):
         fc_W.append(_uniform_pm1(gw, k, n))
         if j < len(fc) - 1:
-            Ts.append(_thresholds(gw, n))
+            Ts.append(_thresholds(gw, n, -thr, thr))
             flips.append((torch.rand(n, generator=gw) < flip_share).to(torch.uint8))
         k = n
     if stream != 0:

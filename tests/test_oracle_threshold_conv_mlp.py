@@ -168,7 +168,7 @@ def _convnet_layers(wl):
 
 def test_convnet_forward_vs_library_chain():
     """Table 7 layer by layer with float64 library calls: conv2d on a padded tensor, max_pool2d, comparisons."""
-    wl = workloads.cifar_convnet(B=3, H=8, W=8, widths=(8, 8, 16, 16), fc=(24, 10), seed=5)
+    wl = workloads.cifar_convnet(B=3, H=8, W=8, widths=(8, 8, 16, 16), fc=(24, 10), seed=5, thr=3)
     layers = _convnet_layers(wl)
     got = oracle.convnet_forward(wl.X.numpy().astype(np.int32), layers)
     a = wl.X.double()
