@@ -55,7 +55,7 @@
 extern "C" {
 #endif
 
-#define QNN_VERSION 200
+#define QNN_VERSION 210
 
 /* status codes */
 #define QNN_OK 0
@@ -401,6 +401,81 @@ QNN_API int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, 
 
 QNN_API size_t qnn_mlp_workspace_bytes(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int algo,
                                int host_io);
+
+/* ------------------------------------------------------------------------- */
+/* The ConvNet of Table 7                                                     */
+/* ------------------------------------------------------------------------- */
+
+/* First layer of Table 7: a stride-1 convolution of 8-bit pixel codes with +-1
+ * filters, i.e. Eq. 8 summed over the eight bit planes:
+ *   out[b,co,y,x] = sum_{c,kh,kw} q[b,c,y+kh-pad,x+kw-pad] * w[co,c,kh,kw],
+ * a tap outside the image reading pad_code (0 = the zero border of a 'same'
+ * convolution).  Runs as an im2col of the codes and one int8 tensor-core product.
+ *   x         device, uint8 [B,C,H,W]
+ *   w         device, packed filters as qnn_pack_conv_weights writes them
+ *   out_nchw  device, int32 [B,Cout,Ho,Wo] or NULL (Ho = H + 2 pad - KH + 1)
+ *   thr/flip  folded batch norm, needed for out_bits / out_form
+ *   out_bits  device, packed NHWC bits [B,Ho,Wo,ceil(Cout/32)] or NULL
+ *   out_form  device, the same signs as NHWC values in out_form_kind
+ *             (QNN_FORM_*; pixels 32*ceil(Cout/32) elements apart), or NULL
+ *   ws        256-byte aligned scratch of qnn_conv2d_u8_workspace_bytes(...)
+ * Errors: INVALID_ARG, UNSUPPORTED (KH*KW*C > 8192), WORKSPACE, CUDA. */
+QNN_API size_t qnn_conv2d_u8_workspace_bytes(int B, int C, int H, int W, int Cout, int KH, int KW, int pad);
+QNN_API int qnn_conv2d_u8(const uint8_t *x, int B, int C, int H, int W, const uint32_t *w, int Cout, int KH, int KW,
+                          int pad, int pad_code, int32_t *out_nchw, const int32_t *thr, const uint8_t *flip,
+                          uint32_t *out_bits, void *out_form, int out_form_kind, void *ws, size_t ws_bytes,
+                          void *stream);
+
+/* 2 x 2 / stride 2 max-pooling placed between a convolution and its batch norm
+ * (Table 7), applied AFTER the folded threshold: since the threshold is
+ * monotone in the sum, the bit of a window's largest sum is the OR of its four
+ * bits, and the AND for channels with flip[c] != 0.  A trailing odd row or
+ * column is dropped.
+ *   bits      device, packed NHWC bits [B,H,W,ceil(C/32)] (pad bits zero)
+ *   flip      device, uint8 [C] (the flip given to the threshold) or NULL
+ *   out_bits  device, [B,H/2,W/2,ceil(C/32)] or NULL
+ *   out_form  device, the pooled signs as NHWC values in out_form_kind, or NULL */
+QNN_API int qnn_maxpool2x2_bits(const uint32_t *bits, int B, int H, int W, int C, const uint8_t *flip,
+                                uint32_t *out_bits, void *out_form, int out_form_kind, void *stream);
+
+#define QNN_LAYER_CONV_U8 1 /* first layer: 8-bit codes x +-1 filters, zero border        */
+#define QNN_LAYER_CONV 2    /* +-1 x +-1 'same' convolution, border value +1              */
+#define QNN_LAYER_FC 3      /* fully connected +-1 x +-1                                   */
+
+/* One layer of a ConvNet (a HOST struct; the pointers inside are device pointers). */
+typedef struct qnn_net_layer {
+    int kind;            /* QNN_LAYER_*                                                     */
+    int C;               /* convolution: input channels; FC: inputs                        */
+    int Cout;            /* convolution: output channels; FC: units                        */
+    int ksize;           /* convolution: ksize x ksize filter, ksize = 2 * pad + 1         */
+    int pad;
+    int pool;            /* convolution: 1 = 2 x 2 max-pooling before the threshold        */
+    const uint32_t *w;   /* convolution: qnn_pack_conv_weights layout [Cout, k*k*ceil(C/32)];
+                            FC after a convolution: the same layout for a [Cout, C', H', W']
+                            filter covering the whole feature map (inputs in (h, w, c)
+                            order, each pixel padded to whole words); FC after an FC layer:
+                            [Cout, ceil(C/32)]                                              */
+    const int32_t *thr;  /* int32 [Cout]; NULL only on the last layer                      */
+    const uint8_t *flip; /* uint8 [Cout] or NULL                                           */
+} qnn_net_layer;
+
+/* Table 7 at inference, layer by layer on one stream: convolution, optional
+ * pooling, folded batch norm + binarisation (Algorithm 4's a^b), then the fully
+ * connected layers; the last layer (FC) returns int32 scores [B, Cout].
+ * Convolutions with C a multiple of 128 and images up to 128 wide run as
+ * implicit products on the tensor cores from filter banks prepared once by
+ * qnn_convnet_prepare (activations pass between them in tensor-core form);
+ * other shapes take the packed im2col path.
+ *   x         device, uint8 [B, layers[0].C, H, W]
+ *   prepared  device, written by qnn_convnet_prepare for the same layers, H, W
+ *   ws        256-byte aligned scratch of qnn_convnet_workspace_bytes(...)
+ * Errors: INVALID_ARG (layers that do not chain), UNSUPPORTED, WORKSPACE, CUDA. */
+QNN_API size_t qnn_convnet_prepared_bytes(int H, int W, const qnn_net_layer *layers, int n);
+QNN_API int qnn_convnet_prepare(int H, int W, const qnn_net_layer *layers, int n, void *prepared,
+                                size_t prepared_bytes, void *stream);
+QNN_API size_t qnn_convnet_workspace_bytes(int B, int H, int W, const qnn_net_layer *layers, int n);
+QNN_API int qnn_convnet_forward(const uint8_t *x, int B, int H, int W, const qnn_net_layer *layers, int n,
+                                const void *prepared, int32_t *scores, void *ws, size_t ws_bytes, void *stream);
 
 /* ------------------------------------------------------------------------- */
 /* Workspace, status                                                          */

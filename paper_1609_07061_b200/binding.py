@@ -23,6 +23,7 @@ QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA, QNN_ALGO_TC_FP4 =
 QNN_FORM_I8, QNN_FORM_FP4 = 1, 2
 QNN_MODE_U01, QNN_MODE_PM1 = 0, 1
 QNN_OP_XNOR_GEMM, QNN_OP_BITPLANE_GEMM, QNN_OP_CONV2D, QNN_OP_MLP = 1, 2, 3, 4
+QNN_LAYER_CONV_U8, QNN_LAYER_CONV, QNN_LAYER_FC = 1, 2, 3
 QNN_NOALLOC_SCRATCH_BYTES = 8 << 20
 
 
@@ -62,6 +63,11 @@ class qnn_mlp_layer(ctypes.Structure):
                 ("w_tc", vp), ("w_tc_ld", i64), ("w_tc_form", i32)]
 
 
+class qnn_net_layer(ctypes.Structure):
+    _fields_ = [("kind", i32), ("C", i32), ("Cout", i32), ("ksize", i32), ("pad", i32), ("pool", i32),
+                ("w", vp), ("thr", vp), ("flip", vp)]
+
+
 _SIGS = {
     "qnn_version": (i32, []),
     "qnn_status_string": (ctypes.c_char_p, [i32]),
@@ -93,6 +99,13 @@ _SIGS = {
     "qnn_conv_prepared_bytes": (sz, [i32, i32, i32, i32, i32]),
     "qnn_conv_prepare": (i32, [vp, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
     "qnn_binary_conv2d_prepared": (i32, [ctypes.POINTER(qnn_conv_io), i32, i32, i32, i32, vp, i32, i32, i32, i32, vp, sz, vp]),
+    "qnn_conv2d_u8_workspace_bytes": (sz, [i32, i32, i32, i32, i32, i32, i32, i32]),
+    "qnn_conv2d_u8": (i32, [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]),
+    "qnn_maxpool2x2_bits": (i32, [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]),
+    "qnn_convnet_prepared_bytes": (sz, [i32, i32, ctypes.POINTER(qnn_net_layer), i32]),
+    "qnn_convnet_prepare": (i32, [i32, i32, ctypes.POINTER(qnn_net_layer), i32, vp, sz, vp]),
+    "qnn_convnet_workspace_bytes": (sz, [i32, i32, i32, ctypes.POINTER(qnn_net_layer), i32]),
+    "qnn_convnet_forward": (i32, [vp, i32, i32, i32, ctypes.POINTER(qnn_net_layer), i32, vp, vp, vp, sz, vp]),
     "qnn_mlp_forward": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
     "qnn_mlp_forward_host": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
     "qnn_mlp_layer_form": (i32, [ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
@@ -324,6 +337,112 @@ def qnn_mlp_forward_host(x_host, M, in_bits, layers, scores_host, algo=QNN_ALGO_
     wp, wb = _ws(ws)
     _ck(_lib.qnn_mlp_forward_host(_p(x_host), M, in_bits, layers, len(layers), _p(scores_host), algo, wp, wb,
                                   _stream()), "qnn_mlp_forward_host")
+
+
+def qnn_conv2d_u8_workspace_bytes(B, C, H, W, Cout, KH, KW, pad) -> int:
+    return int(_lib.qnn_conv2d_u8_workspace_bytes(B, C, H, W, Cout, KH, KW, pad))
+
+
+def qnn_conv2d_u8(x, B, C, H, W, w, Cout, KH, KW, pad, pad_code=0, out_nchw=None, thr=None, flip=None, out_bits=None,
+                  out_form=None, out_form_kind=0, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_conv2d_u8(_p(x), B, C, H, W, _p(w), Cout, KH, KW, pad, pad_code, _p(out_nchw), _p(thr), _p(flip),
+                           _p(out_bits), _p(out_form), out_form_kind, wp, wb, _stream()), "qnn_conv2d_u8")
+
+
+def qnn_maxpool2x2_bits(bits, B, H, W, C, flip=None, out_bits=None, out_form=None, out_form_kind=0):
+    _ck(_lib.qnn_maxpool2x2_bits(_p(bits), B, H, W, C, _p(flip), _p(out_bits), _p(out_form), out_form_kind, _stream()),
+        "qnn_maxpool2x2_bits")
+
+
+def make_net_layers(specs):
+    """specs: dicts with kind, C, Cout, and (conv) ksize, pad, pool; w, thr, flip device tensors (thr None on the last)."""
+    arr = (qnn_net_layer * len(specs))()
+    for i, sp in enumerate(specs):
+        arr[i].kind = sp["kind"]
+        arr[i].C = sp["C"]
+        arr[i].Cout = sp["Cout"]
+        arr[i].ksize = sp.get("ksize", 0)
+        arr[i].pad = sp.get("pad", 0)
+        arr[i].pool = 1 if sp.get("pool") else 0
+        arr[i].w = _p(sp["w"])
+        arr[i].thr = _p(sp.get("thr"))
+        arr[i].flip = _p(sp.get("flip"))
+    return arr
+
+
+class ConvNet:
+    """A Table 7 network on the device: packed weights, layer structs, prepared filter banks (argument marshalling only)."""
+
+    def __init__(self, in_ch, H, W, conv_W, conv_pool, fc_W, Ts, flips):
+        """conv_W: fp32 [Cout,C,k,k] tensors; fc_W: fp32 [K,N], the first with K in (h, w, c) order of the last
+        feature map; Ts / flips: per layer but the last (flips may hold None)."""
+        self.H, self.W = H, W
+        self.keep, specs = [], []
+        c, h, w, t = in_ch, H, W, 0
+        for i, (Wc, pool) in enumerate(zip(conv_W, conv_pool)):
+            co, ci, k, _ = Wc.shape
+            wb = torch.zeros(co, k * k * ((ci + 31) // 32), dtype=torch.int32, device="cuda")
+            qnn_pack_conv_weights(Wc.cuda().contiguous(), co, ci, k, k, wb)
+            specs.append(dict(kind=QNN_LAYER_CONV_U8 if i == 0 else QNN_LAYER_CONV, C=ci, Cout=co, ksize=k, pad=k // 2,
+                              pool=pool, w=wb, thr=Ts[t].cuda(), flip=None if flips[t] is None else flips[t].cuda()))
+            t += 1
+            c = co
+            if pool:
+                h, w = h // 2, w // 2
+        first = True
+        for j, Wf in enumerate(fc_W):
+            K, N = Wf.shape
+            last = j == len(fc_W) - 1
+            if first and len(conv_W) > 0:
+                # inputs in (h, w, c) order, every pixel padded to whole words: the packed layout of an h x w filter
+                w4 = Wf.reshape(h, w, c, N).permute(3, 2, 0, 1).contiguous().cuda()
+                wb = torch.zeros(N, h * w * ((c + 31) // 32), dtype=torch.int32, device="cuda")
+                qnn_pack_conv_weights(w4, N, c, h, w, wb)
+            else:
+                ld = (K + 31) // 32
+                wb = torch.zeros(N, ld, dtype=torch.int32, device="cuda")
+                qnn_quantize_pack_sign_t(Wf.cuda().contiguous(), K, N, N, wb, ld)
+            first = False
+            specs.append(dict(kind=QNN_LAYER_FC, C=K, Cout=N, w=wb, thr=None if last else Ts[t].cuda(),
+                              flip=None if (last or flips[t] is None) else flips[t].cuda()))
+            t += 0 if last else 1
+        self.n_out = specs[-1]["Cout"]
+        self.keep = specs
+        self.layers = make_net_layers(specs)
+        nb = qnn_convnet_prepared_bytes(H, W, self.layers)
+        if nb == 0:
+            raise QnnError(QNN_ERR_INVALID_ARG, "qnn_convnet_prepared_bytes")
+        self.prepared = torch.empty(nb, dtype=torch.uint8, device="cuda")
+        qnn_convnet_prepare(H, W, self.layers, self.prepared)
+
+    def workspace(self, B) -> torch.Tensor:
+        nb = qnn_convnet_workspace_bytes(B, self.H, self.W, self.layers)
+        if nb == 0 and B > 0:
+            raise QnnError(QNN_ERR_INVALID_ARG, "qnn_convnet_workspace_bytes")
+        return torch.empty(max(nb, 256), dtype=torch.uint8, device="cuda")
+
+    def forward(self, x, scores, ws):
+        qnn_convnet_forward(x, x.shape[0], self.H, self.W, self.layers, self.prepared, scores, ws)
+
+
+def qnn_convnet_prepared_bytes(H, W, layers) -> int:
+    return int(_lib.qnn_convnet_prepared_bytes(H, W, layers, len(layers)))
+
+
+def qnn_convnet_prepare(H, W, layers, prepared):
+    _ck(_lib.qnn_convnet_prepare(H, W, layers, len(layers), _p(prepared), prepared.numel() * prepared.element_size(), _stream()),
+        "qnn_convnet_prepare")
+
+
+def qnn_convnet_workspace_bytes(B, H, W, layers) -> int:
+    return int(_lib.qnn_convnet_workspace_bytes(B, H, W, layers, len(layers)))
+
+
+def qnn_convnet_forward(x, B, H, W, layers, prepared, scores, ws=None):
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_convnet_forward(_p(x), B, H, W, layers, len(layers), _p(prepared), _p(scores), wp, wb, _stream()),
+        "qnn_convnet_forward")
 
 
 def qnn_workspace_bytes(op, M, N, K, ka=1, kb=1, algo=QNN_ALGO_AUTO) -> int:

@@ -115,13 +115,15 @@ inline int grid_for(int64_t total)
     return (int)(need < cap ? need : cap);
 }
 
-// Where the prepared form of a filter bank lives: weights in tensor-core form, then the border table.
-struct ConvPrep {
-    int form;
-    int64_t kwords, w_pitch;
-    int classes, corr_ld;
-    size_t w_bytes, c_bytes;
-};
+int conv_prepare_into(const uint32_t *w, int Cout, int C, int KH, int KW, int pad, int pad_bit, const ConvPrep &l, uint8_t *wf,
+                      int32_t *corr, cudaStream_t st)
+{
+    if (int rc = tc_expand(w, 1, QNN_MODE_PM1, l.kwords, 0, Cout, l.kwords, l.kwords, 32, l.form, wf, l.w_pitch, st)) return rc;
+    conv_border_corr_kernel<<<l.corr_ld, 128, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, l.classes, l.corr_ld);
+    return check_launch("conv border table");
+}
+
+}  // namespace
 
 // The implicit tensor-core path takes stride-1 "same" filters (at most 7 x 7: 64 taps), images at most 128 pixels wide
 // and whole 128-byte channel blocks per pixel: 256 channels as e2m1 values, 128 as int8.  want_form = 0: the best form.
@@ -142,15 +144,6 @@ bool conv_prep_layout(int Cout, int C, int KH, int KW, int pad, int want_form, C
     return true;
 }
 
-int conv_prepare_into(const uint32_t *w, int Cout, int C, int KH, int KW, int pad, int pad_bit, const ConvPrep &l, uint8_t *wf,
-                      int32_t *corr, cudaStream_t st)
-{
-    if (int rc = tc_expand(w, 1, QNN_MODE_PM1, l.kwords, 0, Cout, l.kwords, l.kwords, 32, l.form, wf, l.w_pitch, st)) return rc;
-    conv_border_corr_kernel<<<l.corr_ld, 128, 0, st>>>(w, Cout, C, KH, KW, pad, pad_bit, corr, l.classes, l.corr_ld);
-    return check_launch("conv border table");
-}
-
-}  // namespace
 }  // namespace qnn
 
 using namespace qnn;

@@ -385,17 +385,6 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr)
     return d;
 }
 
-// bit i of the low byte of x -> bit 4*i (one bit per nibble)
-__device__ __forceinline__ uint32_t spread_bits_to_nibbles(uint32_t x)
-{
-    x = (x | (x << 12)) & 0x000F000Fu;
-    x = (x | (x << 6)) & 0x03030303u;
-    x = (x | (x << 3)) & 0x11111111u;
-    return x;
-}
-// bit i of the low nibble of x -> bit 8*i (one bit per byte)
-__device__ __forceinline__ uint32_t spread_bits_to_bytes(uint32_t nib) { return (nib * 0x00204081u) & 0x01010101u; }
-
 constexpr int next_pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
 template <int FORM, int BN, int STG, int CTAS>

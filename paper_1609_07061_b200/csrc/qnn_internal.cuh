@@ -96,8 +96,51 @@ int64_t tc_row_bytes(int64_t kwords, int form);
 // distance between rows the library itself lays operands out with: whole 128-byte lines, so that every TMA box row
 // is one line (a row pitch that is not a multiple of 128 doubles the memory requests of the loads)
 int64_t tc_row_pitch(int64_t kwords, int form);
+// Prepared filter bank of the implicit tensor-core convolution: weights in tensor-core form, then the border table.
+struct ConvPrep {
+    int form;
+    int64_t kwords, w_pitch;
+    int classes, corr_ld;
+    size_t w_bytes, c_bytes;
+};
+bool conv_prep_layout(int Cout, int C, int KH, int KW, int pad, int want_form, ConvPrep *l);
 int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
               int64_t pad_period, int pad_tail, int form, uint8_t *dst, int64_t dst_ld, cudaStream_t st);
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st);
+
+#ifdef __CUDACC__
+// bit i of the low byte of x -> bit 4*i (one bit per nibble)
+__device__ __forceinline__ uint32_t spread_bits_to_nibbles(uint32_t x)
+{
+    x = (x | (x << 12)) & 0x000F000Fu;
+    x = (x | (x << 6)) & 0x03030303u;
+    x = (x | (x << 3)) & 0x11111111u;
+    return x;
+}
+// bit i of the low nibble of x -> bit 8*i (one bit per byte)
+__device__ __forceinline__ uint32_t spread_bits_to_bytes(uint32_t nib) { return (nib * 0x00204081u) & 0x01010101u; }
+
+// 32 sign bits as 32 e2m1 values (+1 -> 0x2, -1 -> 0xA; elements outside `valid` -> 0), element 2i in the low nibble of byte i
+__device__ __forceinline__ uint4 signs_to_fp4(uint32_t w, uint32_t valid)
+{
+    uint32_t o[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+        o[b] = (0xAAAAAAAAu ^ (spread_bits_to_nibbles((w >> (8 * b)) & 0xffu) << 3)) &
+               (spread_bits_to_nibbles((valid >> (8 * b)) & 0xffu) * 0xfu);
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+// 32 sign bits as 32 int8 values (+1 -> 0x01, -1 -> 0xFF; elements outside `valid` -> 0): bytes 0..15 and 16..31
+__device__ __forceinline__ void signs_to_i8(uint32_t w, uint32_t valid, uint4 &lo, uint4 &hi)
+{
+    uint32_t o[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b)
+        o[b] = (0xFFFFFFFFu ^ (spread_bits_to_bytes((w >> (4 * b)) & 0xfu) * 0xfeu)) &
+               (spread_bits_to_bytes((valid >> (4 * b)) & 0xfu) * 0xffu);
+    lo = make_uint4(o[0], o[1], o[2], o[3]);
+    hi = make_uint4(o[4], o[5], o[6], o[7]);
+}
+#endif
 
 }  // namespace qnn
