@@ -30,16 +30,22 @@ __global__ void __launch_bounds__(256) im2col_u8_kernel(const uint8_t *__restric
         const int yo = (int)(t % Ho);
         const int64_t b = t / Ho;
         uint32_t o[4] = {0u, 0u, 0u, 0u};
+        // (kh, kw, c) of the first byte by division, of the others by counting on
+        int k = piece * 16;
+        int tap = k / C, c = k - tap * C;
+        int kh = tap / KW, kw = tap - kh * KW;
+        const uint8_t *img = x + b * C * H * W;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int k = piece * 16 + j;
+        for (int j = 0; j < 16; ++j, ++k) {
             if (k < K) {
-                const int tap = k / C, c = k - tap * C;
-                const int kh = tap / KW, kw = tap - kh * KW;
                 const int yi = yo + kh - pad, xi = xo + kw - pad;
                 uint32_t v = (uint32_t)pad_code;
-                if (yi >= 0 && yi < H && xi >= 0 && xi < W) v = __ldg(x + ((b * C + c) * H + yi) * W + xi);
+                if (yi >= 0 && yi < H && xi >= 0 && xi < W) v = __ldg(img + (c * H + yi) * W + xi);
                 o[j >> 2] |= v << (8 * (j & 3));
+                if (++c == C) {
+                    c = 0;
+                    if (++kw == KW) { kw = 0; ++kh; }
+                }
             }
         }
         reinterpret_cast<uint4 *>(dst)[e] = make_uint4(o[0], o[1], o[2], o[3]);

@@ -54,6 +54,7 @@ struct TcParams {
     // implicit convolution (conv != 0)
     int conv;
     int32_t cH, cW, cR, tiles_per_img, cKW, cpad, cblocks;
+    int32_t cG, cB;             // images per tile (> 1 only when a whole image is at most half a tile), images in all
     const int32_t *corr;
     int64_t corr_ld;                 // row length of the correction table: N rounded up to 32, pad zero
 };
@@ -348,6 +349,12 @@ __device__ __forceinline__ uint32_t tma_stage_conv(uint32_t next_empty_bar, uint
     return ready;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while the kernel
+// before it is still draining; it must not touch that kernel's results (or buffers that kernel still reads) before
+// griddep_wait() returns, which is when every earlier kernel has completed and its writes are visible.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -435,6 +442,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // the next kernel in the stream may be scheduled as soon as SMs free up; it waits for this grid where it needs to
+    griddep_launch_dependents();
     // In a pair (CTAS = 2) CTA 0 of the cluster leads: it owns the full and accumulator-empty barriers and issues
     // the MMAs; both CTAs load their halves of the operands and drain their 128 rows of the accumulator.
     const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
@@ -469,6 +478,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         tc_fence_after();
     }
 
+    // Everything above (barriers, tensor memory, scales) touched only this CTA's own state and overlapped the tail of
+    // the previous kernel; from here on global memory is read and written.
+    griddep_wait();
+
     const uint32_t tiles_m = (uint32_t)p.tiles_m;                      // in units of BM * CTAS rows
     const uint32_t num_tiles = tiles_m * (uint32_t)p.tiles_n;          // below 2^31 (checked on the host)
     // a CTA, or a pair of them, walks the tiles blockIdx.x / CTAS, + gridDim.x / CTAS, ...  (written out in every
@@ -483,7 +496,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS) {
                 const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
                 int32_t img = 0, y0 = 0;
-                if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; }
+                if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; img *= p.cG; }
                 int32_t cb = 0, kw = 0, kh = 0;                    // conv: channel block, filter column, filter row of kb
                 for (int32_t kb = 0; kb < p.num_kb; ++kb) {
                     if (!ready && !mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 1)) { ok = false; break; }
@@ -614,14 +627,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             bool mrow;
             int32_t cls = 0, c_img = 0, c_pix0 = 0;
             if (p.conv) {
-                c_img = tm / p.tiles_per_img;
-                const int32_t y0 = (tm - c_img * p.tiles_per_img) * p.cR;
-                const int32_t y = y0 + r / p.cW;
-                const int32_t x = r % p.cW;
-                mrow = (r < p.cR * p.cW) && (y < p.cH);
+                // a tile is cR rows of one image, or cG whole images one after the other
+                const int32_t tile_img = tm / p.tiles_per_img;
+                const int32_t y0 = (tm - tile_img * p.tiles_per_img) * p.cR;
+                const int32_t gi = r / (p.cR * p.cW), rem = r - gi * (p.cR * p.cW);
+                const int32_t y = y0 + rem / p.cW;
+                const int32_t x = rem % p.cW;
+                c_img = tile_img * p.cG + gi;
+                mrow = (gi < p.cG) && (y < p.cH) && (c_img < p.cB);
                 m = ((int64_t)c_img * p.cH + y) * p.cW + x;
                 c_pix0 = y0 * p.cW + q * 32;
-                m_warp0 = (int64_t)c_img * p.cH * p.cW + c_pix0;
+                m_warp0 = (int64_t)tile_img * p.cG * p.cH * p.cW + c_pix0;
                 const int32_t pd = p.cpad, pc = pd + 1;
                 const int32_t ty = max(pd - y, 0), by = max(y + pd - (p.cH - 1), 0);
                 const int32_t tx = max(pd - x, 0), bx = max(x + pd - (p.cW - 1), 0);
@@ -953,13 +969,13 @@ int make_map_2d(CUtensorMap *map, const void *base, int64_t rows, int64_t row_by
 }
 
 // 4-D NHWC byte tensor [B, H, W, cbytes]; box = 128 bytes x W x box_h x 1
-int make_map_nhwc(CUtensorMap *map, const void *base, int B, int H, int W, int64_t cbytes, int box_h)
+int make_map_nhwc(CUtensorMap *map, const void *base, int B, int H, int W, int64_t cbytes, int box_h, int box_b)
 {
     EncodeTiledFn fn = encode_fn();
     QNN_REQUIRE(fn != nullptr, QNN_ERR_CUDA, "tc conv: cuTensorMapEncodeTiled is not available from this driver");
     cuuint64_t dims[4] = {(cuuint64_t)cbytes, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
     cuuint64_t strides[3] = {(cuuint64_t)cbytes, (cuuint64_t)cbytes * W, (cuuint64_t)cbytes * W * H};
-    cuuint32_t box[4] = {(cuuint32_t)BKB, (cuuint32_t)W, (cuuint32_t)box_h, 1};
+    cuuint32_t box[4] = {(cuuint32_t)BKB, (cuuint32_t)W, (cuuint32_t)box_h, (cuuint32_t)box_b};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1018,19 +1034,29 @@ int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMa
     QNN_REQUIRE(tiles < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: too many output tiles");
     const int nw = (int)(tiles < workers ? tiles : workers);
     profile_before(st);
-    if (CTAS == 2) {
+    {
+        // programmatic stream serialisation: the grid may be scheduled while the previous kernel drains (the kernel
+        // calls griddepcontrol.wait before it touches global memory); QNN_PDL=0 in the environment turns it off
+        static const bool pdl = [] { const char *e = getenv("QNN_PDL"); return !(e && e[0] == '0'); }();
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * (unsigned)nw);
+        cfg.gridDim = dim3((unsigned)(CTAS * nw));
         cfg.blockDim = dim3(TC_THREADS);
         cfg.dynamicSmemBytes = S::TOTAL;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
+        cudaLaunchAttribute attr[2];
+        unsigned na = 0;
+        if (CTAS == 2) {
+            attr[na].id = cudaLaunchAttributeClusterDimension;
+            attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+            ++na;
+        }
+        if (pdl) {
+            attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[na].val.programmaticStreamSerializationAllowed = 1;
+            ++na;
+        }
+        cfg.attrs = attr; cfg.numAttrs = na;
         QNN_CUDA(cudaLaunchKernelEx(&cfg, kern, ma, mb, mo, p));
-    } else {
-        kern<<<nw, TC_THREADS, S::TOTAL, st>>>(ma, mb, mo, p);
     }
     profile_after(st);
     return check_launch("tc gemm");
@@ -1046,7 +1072,7 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, int 
     p.tiles_n = (int32_t)ceil_div(p.N, BN);
     p.idesc |= (uint32_t)(BN >> 3) << 17;
     if (CTAS == 2) p.idesc = (p.idesc & ~(0x1fu << 24)) | ((uint32_t)((2 * BM) >> 4) << 24);   // the pair's instruction is 256 rows tall
-    const bool conv_full_tiles = p.conv && p.cR * p.cW == BM;
+    const bool conv_full_tiles = p.conv && p.cR * p.cW == BM && p.cG == 1;
     if (p.out != nullptr && aligned(p.out, 16)) {
         // (the bulk store clips the innermost extent in 16-byte units, so N must be a whole number of them)
         if (!p.conv && p.epilogue == EPI_ROWMAJOR && p.ldo % 4 == 0 && p.N % 4 == 0) {
@@ -1250,15 +1276,18 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
                     QNN_ERR_UNSUPPORTED, "tc conv: implicit path needs a stride-1 'same' filter and W <= 128");
         const int R = BM / c.W < c.H ? BM / c.W : c.H;                  // image rows per tile
         QNN_REQUIRE(R >= 1 && R <= 256, QNN_ERR_UNSUPPORTED, "tc conv: bad tile height");
+        // feature maps of at most half a tile: several whole images per tile
+        const int G = (R == c.H && BM / (c.H * c.W) >= 2) ? BM / (c.H * c.W) : 1;
         p.conv = 1; p.cH = c.H; p.cW = c.W; p.cR = R; p.tiles_per_img = (int32_t)ceil_div(c.H, R);
+        p.cG = G; p.cB = c.B;
         p.cKW = c.KW; p.cpad = c.pad; p.cblocks = c.cblocks; p.corr = c.corr; p.corr_ld = (int64_t)round_up((size_t)g.N, 32);
         QNN_REQUIRE(aligned(c.corr, 16), QNN_ERR_ALIGNMENT, "tc conv: correction table must be 16-byte aligned");
-        p.tiles_m = c.B * p.tiles_per_img;
-        p.a_tx_bytes = R * c.W * BKB;
+        p.tiles_m = (int32_t)ceil_div(c.B, G) * p.tiles_per_img;
+        p.a_tx_bytes = G * R * c.W * BKB;
         QNN_REQUIRE(p.num_kb == c.KH * c.KW * c.cblocks, QNN_ERR_INVALID_ARG, "tc conv: K blocks do not match the filter");
         QNN_REQUIRE(g.M == (int64_t)c.B * c.H * c.W, QNN_ERR_INVALID_ARG, "tc conv: M does not match the image geometry");
         QNN_REQUIRE(a_ld == (int64_t)c.cblocks * BKB, QNN_ERR_INVALID_ARG, "tc conv: pixels must be whole 128-byte channel blocks apart");
-        if (int rc = make_map_nhwc(&ma, a8, c.B, c.H, c.W, (int64_t)c.cblocks * BKB, R)) return rc;
+        if (int rc = make_map_nhwc(&ma, a8, c.B, c.H, c.W, (int64_t)c.cblocks * BKB, R, G)) return rc;
     } else {
         if (int rc = make_map_2d(&ma, a8, g.M, a_row_bytes, a_ld, BM)) return rc;
     }
