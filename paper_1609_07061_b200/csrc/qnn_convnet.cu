@@ -214,6 +214,9 @@ struct LayerPlan {
     // FC: how its input rows are laid out
     int64_t kwords, pad_period;
     int pad_tail;
+    int fc_form;                // FC: tensor-core form its prepared weights are kept in (0 = none)
+    int64_t fc_pitch;           // bytes between prepared weight rows
+    bool fc_tc;                 // FC: runs on the tensor cores at this batch size
 };
 
 struct NetPlan {
@@ -284,8 +287,14 @@ int plan_net(int B, int H, int W, const qnn_net_layer *layers, int n, NetPlan *p
             } else {
                 lp.kwords = ceil_div(ly.C, 32);
             }
-            const size_t g = qnn_workspace_bytes(QNN_OP_XNOR_GEMM, B, ly.Cout, lp.kwords * 32, 1, 1, QNN_ALGO_AUTO);
-            if (g > gen) gen = g;
+            // weights are also kept in tensor-core form; with both operands ready the tensor cores win from about
+            // 2^24 products on (no operand-rewriting launches), below that the CUDA-core kernel's shorter start does
+            lp.fc_form = tc_pick_form(1, QNN_MODE_PM1, 1, QNN_MODE_PM1, ly.C);
+            if (lp.fc_form != 0) {
+                lp.fc_pitch = tc_row_pitch(lp.kwords, lp.fc_form);
+                lp.prep_bytes = (size_t)ly.Cout * (size_t)lp.fc_pitch;
+                lp.fc_tc = (double)B * (double)ly.Cout * (double)ly.C >= 16777216.0;
+            }
             lp.out_rows = B;
             lp.out_cw = (int)ceil_div(ly.Cout, 32);
             prev_c = 0;
@@ -296,7 +305,7 @@ int plan_net(int B, int H, int W, const qnn_net_layer *layers, int n, NetPlan *p
         prep += round_up(lp.prep_bytes, 256);
         if (i < n - 1) {
             const size_t bb = round_up((size_t)lp.out_rows * lp.out_cw * 4, 256);
-            const size_t fb = round_up((size_t)lp.out_rows * lp.out_cw * 32, 256);
+            const size_t fb = round_up((size_t)lp.out_rows * round_up((size_t)lp.out_cw * 32, 128), 256);   // rows on 128-byte lines
             if (bb > bits) bits = bb;
             if (fb > form) form = fb;
         }
@@ -397,6 +406,12 @@ int qnn_convnet_prepare(int H, int W, const qnn_net_layer *layers, int n, void *
         } else if (ly.kind == QNN_LAYER_CONV && lp.fast) {
             if (int rc = qnn_conv_prepare(ly.w, ly.Cout, ly.C, ly.ksize, ly.ksize, ly.pad, 1, base + lp.prep_off, lp.prep_bytes, stream))
                 return rc;
+        } else if (ly.kind == QNN_LAYER_FC && lp.fc_form != 0) {
+            const int64_t period = lp.pad_period > 0 ? lp.pad_period : lp.kwords;
+            const int tail = lp.pad_period > 0 ? lp.pad_tail : (int)(ly.C - 32 * (lp.kwords - 1));
+            if (int rc = tc_expand(ly.w, 1, QNN_MODE_PM1, lp.kwords, 0, ly.Cout, lp.kwords, period, tail, lp.fc_form, base + lp.prep_off,
+                                   lp.fc_pitch, st))
+                return rc;
         }
     }
     return QNN_OK;
@@ -422,29 +437,62 @@ int qnn_convnet_forward(const uint8_t *x, int B, int H, int W, const qnn_net_lay
     const uint32_t *cur_bits = nullptr;
     const void *cur_form = nullptr;
     int cur_kind = 0;
+    int64_t cur_form_ld = 0;
+    // the form layer i reads its input in: a tensor-core layer its operand form, everything else packed bits (0)
+    auto in_form = [&](int i) -> int {
+        if (i >= n) return 0;
+        if (layers[i].kind == QNN_LAYER_CONV && p.l[i].fast) return p.l[i].prep.form;
+        if (layers[i].kind == QNN_LAYER_FC && p.l[i].fc_tc) return p.l[i].fc_form;
+        return 0;
+    };
 
     for (int i = 0; i < n; ++i) {
         const qnn_net_layer &ly = layers[i];
         const LayerPlan &lp = p.l[i];
         const bool last = i == n - 1;
         // what the next layer reads: a fast convolution its form, everything else packed bits
-        const int want_form = (!last && layers[i + 1].kind == QNN_LAYER_CONV && p.l[i + 1].fast) ? p.l[i + 1].prep.form : 0;
+        const int want_form = in_form(i + 1);
         uint32_t *act_bits = reinterpret_cast<uint32_t *>(wsb + p.off_act[i & 1]);
         void *act_form = wsb + p.off_act[i & 1] + p.act_bits_bytes;
 
         if (ly.kind == QNN_LAYER_FC) {
             GemmArgs g{};
-            g.a = cur_bits; g.lda = lp.kwords; g.b = ly.w; g.ldb = lp.kwords;
             g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;
-            g.M = B; g.N = ly.Cout; g.K = ly.C; g.kwords = lp.kwords;
-            if (lp.pad_period > 0) { g.pad_period = lp.pad_period; g.pad_tail = lp.pad_tail; }
+            g.M = B; g.N = ly.Cout; g.K = ly.C;
+            if (lp.pad_period > 0) { g.kwords = lp.kwords; g.pad_period = lp.pad_period; g.pad_tail = lp.pad_tail; }
             if (last) {
                 g.epilogue = EPI_ROWMAJOR; g.out = scores; g.ldo = ly.Cout;
             } else {
-                g.epilogue = EPI_BITS; g.thr = ly.thr; g.flip = ly.flip; g.out_bits = act_bits; g.ld_bits = lp.out_cw;
+                g.epilogue = EPI_BITS; g.thr = ly.thr; g.flip = ly.flip;
+                if (want_form != 0 && lp.fc_tc) {
+                    g.out_form = act_form; g.out_form_kind = want_form; g.ld_form = tc_row_pitch(lp.out_cw, want_form);
+                } else {
+                    g.out_bits = act_bits; g.ld_bits = lp.out_cw;
+                }
             }
-            if (int rc = run_gemm(g, QNN_ALGO_AUTO, gen, p.gen_bytes, st)) return rc;
-            cur_bits = act_bits; cur_form = nullptr; cur_kind = 0;
+            if (lp.fc_tc && cur_form != nullptr && cur_kind == lp.fc_form) {
+                g.a_tc = cur_form; g.a_tc_form = cur_kind; g.a_tc_ld = cur_form_ld;
+                g.b_tc = prep + lp.prep_off; g.b_tc_form = lp.fc_form; g.b_tc_ld = lp.fc_pitch;
+                if (int rc = validate_gemm(g)) return rc;
+                if (int rc = launch_gemm_tc(g, lp.fc_form, nullptr, 0, st)) return rc;
+            } else {
+                QNN_REQUIRE(cur_bits != nullptr, QNN_ERR_INVALID_ARG, "convnet: layer %d has no packed input", i);
+                g.a = cur_bits; g.lda = lp.kwords; g.b = ly.w; g.ldb = lp.kwords;
+                if (int rc = run_gemm(g, QNN_ALGO_POPC, nullptr, 0, st)) return rc;
+            }
+            if (g.out_form != nullptr) {
+                cur_bits = nullptr; cur_form = act_form; cur_kind = want_form; cur_form_ld = g.ld_form;
+            } else {
+                // a CUDA-core layer feeding a tensor-core one: rewrite its bits in the form the next layer reads
+                cur_bits = act_bits; cur_form = nullptr; cur_kind = 0;
+                if (!last && want_form != 0) {
+                    const int64_t cw = lp.out_cw, ld = tc_row_pitch(cw, want_form);
+                    if (int rc = tc_expand(act_bits, 1, QNN_MODE_PM1, cw, 0, B, cw, cw, ly.Cout - 32 * ((int)cw - 1), want_form,
+                                           static_cast<uint8_t *>(act_form), ld, st))
+                        return rc;
+                    cur_bits = nullptr; cur_form = act_form; cur_kind = want_form; cur_form_ld = ld;
+                }
+            }
             continue;
         }
 
@@ -490,6 +538,7 @@ int qnn_convnet_forward(const uint8_t *x, int B, int H, int W, const qnn_net_lay
         cur_bits = want_form ? nullptr : act_bits;
         cur_form = want_form ? act_form : nullptr;
         cur_kind = want_form;
+        cur_form_ld = want_form ? tc_row_bytes(lp.out_cw, want_form) * (layers[i + 1].kind == QNN_LAYER_FC ? (int64_t)lp.Ho * lp.Wo : 1) : 0;
     }
     return QNN_OK;
 }
