@@ -648,8 +648,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 mrow = m < p.M;
             }
             const bool any_border = p.conv ? (__any_sync(0xffffffffu, cls != 0) != 0) : false;
-            int64_t img = 0, pix = 0;
-            if (p.epilogue == EPI_NCHW && mrow) { img = m / p.hw; pix = m - img * p.hw; }
+            int64_t img = 0, pix = 0;                            // where an int32 NCHW result of this row goes
+            if (p.epilogue == EPI_NCHW && mrow && p.out != nullptr) {
+                if (p.conv) { img = c_img; pix = m - (int64_t)c_img * p.cH * p.cW; }
+                else { img = m / p.hw; pix = m - img * p.hw; }
+            }
 
             // the tensor-memory loads below are warp-collective: leave the loop only as a whole warp
             if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(as), aphase, abort_flag, 4))) { ok = false; break; }
@@ -664,29 +667,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 const int64_t n0 = ntile + c * 32;
                 uint32_t v[32];
                 tmem_ld32(tacc + (uint32_t)(c * 32), v);
-                // Border corrections, class by class: every lane reads the class's 32 values (one address per load
-                // across the warp), the lanes of that class add them.  e2m1: the fp32 accumulators are exact
-                // integers, so the correction is added in float.
+                // Border corrections.  e2m1: the fp32 accumulators are exact integers, so the correction is added in float.
                 if (any_border) {
-                    uint32_t todo = __ballot_sync(0xffffffffu, cls != 0);
-                    while (todo != 0) {
-                        const int k = __shfl_sync(0xffffffffu, cls, __ffs((int)todo) - 1);
-                        todo &= ~__ballot_sync(0xffffffffu, cls == k);
-                        const int4 *cp = reinterpret_cast<const int4 *>(p.corr + (int64_t)k * p.corr_ld + n0);
+                    // every lane adds the row of its own class (class 0, the interior, is a row of zeros): eight
+                    // independent loads, lanes of one class sharing their addresses
+                    const int4 *cp = reinterpret_cast<const int4 *>(p.corr + (int64_t)cls * p.corr_ld + n0);
+                    int4 cv[8];
 #pragma unroll
-                        for (int j4 = 0; j4 < 8; ++j4) {
-                            const int4 cv = __ldg(cp + j4);
-                            if (cls == k) {
-                                if (FORM == QNN_FORM_FP4) {
-                                    v[4 * j4] = __float_as_uint(__uint_as_float(v[4 * j4]) + (float)cv.x);
-                                    v[4 * j4 + 1] = __float_as_uint(__uint_as_float(v[4 * j4 + 1]) + (float)cv.y);
-                                    v[4 * j4 + 2] = __float_as_uint(__uint_as_float(v[4 * j4 + 2]) + (float)cv.z);
-                                    v[4 * j4 + 3] = __float_as_uint(__uint_as_float(v[4 * j4 + 3]) + (float)cv.w);
-                                } else {
-                                    v[4 * j4] += (uint32_t)cv.x; v[4 * j4 + 1] += (uint32_t)cv.y;
-                                    v[4 * j4 + 2] += (uint32_t)cv.z; v[4 * j4 + 3] += (uint32_t)cv.w;
-                                }
-                            }
+                    for (int j4 = 0; j4 < 8; ++j4) cv[j4] = __ldg(cp + j4);
+#pragma unroll
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        if (FORM == QNN_FORM_FP4) {
+                            v[4 * j4] = __float_as_uint(__uint_as_float(v[4 * j4]) + (float)cv[j4].x);
+                            v[4 * j4 + 1] = __float_as_uint(__uint_as_float(v[4 * j4 + 1]) + (float)cv[j4].y);
+                            v[4 * j4 + 2] = __float_as_uint(__uint_as_float(v[4 * j4 + 2]) + (float)cv[j4].z);
+                            v[4 * j4 + 3] = __float_as_uint(__uint_as_float(v[4 * j4 + 3]) + (float)cv[j4].w);
+                        } else {
+                            v[4 * j4] += (uint32_t)cv[j4].x; v[4 * j4 + 1] += (uint32_t)cv[j4].y;
+                            v[4 * j4 + 2] += (uint32_t)cv[j4].z; v[4 * j4 + 3] += (uint32_t)cv[j4].w;
                         }
                     }
                 }
