@@ -406,6 +406,26 @@ def run_extras(q, bench, peaks, algo):
                                                               out_form_kind=f4), flush)
     rec("c4_conv3x3_prepared_filters_form_in_form_out", ms, best, ops=ops4, note="mid-network layer: activations arrive and leave in tensor-core form")
 
+    # the whole CIFAR-10 ConvNet of Table 7 (first layer on 8-bit pixels, pooled thresholds, FC head), one call per pass
+    for Bn in (128, 1024):
+        wln = workloads.cifar_convnet(B=Bn)
+        net = q.ConvNet(3, 32, 32, wln.conv_W, wln.conv_pool, wln.fc_W, wln.Ts, wln.flips)
+        wsn = net.workspace(Bn)
+        xn = wln.X.cuda()
+        sn = torch.zeros(Bn, net.n_out, dtype=torch.int32, device="cuda")
+        opsn, c_, h_, w_ = 0.0, 3, 32, 32
+        for Wc, pool in zip(wln.conv_W, wln.conv_pool):
+            opsn += 2.0 * Bn * h_ * w_ * Wc.shape[0] * 9 * c_ * (8 if c_ == 3 else 1)
+            c_ = Wc.shape[0]
+            if pool:
+                h_, w_ = h_ // 2, w_ // 2
+        for Wf in wln.fc_W:
+            opsn += 2.0 * Bn * Wf.shape[0] * Wf.shape[1]
+        ms, best = _time_op(lambda: net.forward(xn, sn, wsn), flush)
+        rec(f"table7_convnet_forward_batch{Bn}", ms, best, ops=opsn,
+            note=f"{Bn / ms * 1e3:.0f} images/s; 6 conv + 3 FC layers in one qnn_convnet_forward call, weights prepared once")
+        del net, wsn, xn, sn
+
     # config 5: LSTM gate 4b x 4b and the square sweep
     wl5 = workloads.lstm_gate()
     M, K = wl5.X.shape; N = wl5.W.shape[1]; ld = K // 32
