@@ -126,15 +126,15 @@ int conv_prepare_into(const uint32_t *w, int Cout, int C, int KH, int KW, int pa
 }  // namespace
 
 // The implicit tensor-core path takes stride-1 "same" filters (at most 7 x 7: 64 taps), images at most 128 pixels wide
-// and whole 128-byte channel blocks per pixel: 256 channels as e2m1 values, 128 as int8.  want_form = 0: the best form.
+// and whole channel blocks per pixel: multiples of 128 channels as e2m1 values (128-byte blocks when C is a multiple
+// of 256, else 64-byte blocks), or as int8 (128-byte blocks) when that form is asked for.  want_form = 0: the best form.
 bool conv_prep_layout(int Cout, int C, int KH, int KW, int pad, int want_form, ConvPrep *l)
 {
     if (KH != 2 * pad + 1 || KW != 2 * pad + 1 || pad > 3 || (int64_t)KH * KW * C >= (1 << 24)) return false;
-    int form = 0;
-    if (C % 256 == 0 && want_form != QNN_FORM_I8) form = QNN_FORM_FP4;
-    else if (C % 128 == 0 && want_form != QNN_FORM_FP4) form = QNN_FORM_I8;
-    if (form == 0) return false;
+    if (C % 128 != 0) return false;
+    const int form = want_form == QNN_FORM_I8 ? QNN_FORM_I8 : QNN_FORM_FP4;
     l->form = form;
+    l->kblk = (form == QNN_FORM_FP4 && C % 256 != 0) ? 64 : 128;
     l->kwords = (int64_t)KH * KW * ceil_div(C, 32);
     l->w_pitch = tc_row_pitch(l->kwords, form);
     l->classes = (pad + 1) * (pad + 1) * (pad + 1) * (pad + 1);
@@ -220,7 +220,7 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
             if (int rc = conv_prepare_into(w, Cout, C, KH, KW, pad, pad_bit, lay, wf, corr, st)) return rc;
             ConvImplicit ci{};
             ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;
-            ci.cblocks = (int32_t)(cbytes / 128);
+            ci.cblocks = (int32_t)(cbytes / lay.kblk); ci.kblk = lay.kblk;
             ci.corr = corr;
             g.conv = &ci;
             return launch_gemm_tc(g, lay.form, nullptr, 0, st);
@@ -266,7 +266,7 @@ int qnn_conv_prepare(const uint32_t *w, int Cout, int C, int KH, int KW, int pad
 
 int qnn_conv_form(int C)
 {
-    return C > 0 && C % 256 == 0 ? QNN_FORM_FP4 : (C > 0 && C % 128 == 0 ? QNN_FORM_I8 : 0);
+    return C > 0 && C % 128 == 0 ? QNN_FORM_FP4 : 0;
 }
 
 int qnn_binary_conv2d_prepared(const qnn_conv_io *io, int B, int C, int H, int W, const void *prepared, int Cout, int KH, int KW,
@@ -316,7 +316,7 @@ int qnn_binary_conv2d_prepared(const qnn_conv_io *io, int B, int C, int H, int W
             return rc;
     ConvImplicit ci{};
     ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;
-    ci.cblocks = (int32_t)(cbytes / 128);
+    ci.cblocks = (int32_t)(cbytes / l.kblk); ci.kblk = l.kblk;
     ci.corr = reinterpret_cast<const int32_t *>(wf + l.w_bytes);
     g.conv = &ci;
     return launch_gemm_tc(g, l.form, nullptr, 0, st);

@@ -47,7 +47,8 @@ enum Epilogue { EPI_ROWMAJOR = 0, EPI_NCHW = 1, EPI_BITS = 2 };
 // out-of-image reads return zero; `corr` adds back what the padding value contributes.
 struct ConvImplicit {
     int32_t B, H, W, KH, KW, pad;
-    int32_t cblocks;            // 128-byte channel blocks per pixel
+    int32_t cblocks;            // channel blocks per pixel
+    int32_t kblk;               // bytes per channel block: 128 (0 means 128), or 64 for 128 e2m1 channels
     const int32_t *corr;        // [(pad+1)^4][N rounded up to 32] border corrections (pad columns and class 0 zero)
 };
 
@@ -99,6 +100,7 @@ int64_t tc_row_pitch(int64_t kwords, int form);
 // Prepared filter bank of the implicit tensor-core convolution: weights in tensor-core form, then the border table.
 struct ConvPrep {
     int form;
+    int kblk;                   // bytes of one channel block of a pixel (128, or 64: 128 e2m1 channels)
     int64_t kwords, w_pitch;
     int classes, corr_ld;
     size_t w_bytes, c_bytes;
