@@ -282,6 +282,27 @@ def _time_op(fn, flush, reps=7, warm=3):
     return statistics.median(ts), min(ts)
 
 
+def convnet_record(q, Bn, flush, rec, reps=7):
+    """Times one qnn_convnet_forward call of the Table 7 network at batch Bn (weights prepared once, L2 flushed)."""
+    from paper_1609_07061_b200 import workloads
+    wln = workloads.cifar_convnet(B=Bn)
+    net = q.ConvNet(3, 32, 32, wln.conv_W, wln.conv_pool, wln.fc_W, wln.Ts, wln.flips)
+    wsn = net.workspace(Bn)
+    xn = wln.X.cuda()
+    sn = torch.zeros(Bn, net.n_out, dtype=torch.int32, device="cuda")
+    opsn, c_, h_, w_ = 0.0, 3, 32, 32
+    for Wc, pool in zip(wln.conv_W, wln.conv_pool):
+        opsn += 2.0 * Bn * h_ * w_ * Wc.shape[0] * 9 * c_ * (8 if c_ == 3 else 1)
+        c_ = Wc.shape[0]
+        if pool:
+            h_, w_ = h_ // 2, w_ // 2
+    for Wf in wln.fc_W:
+        opsn += 2.0 * Bn * Wf.shape[0] * Wf.shape[1]
+    ms, best = _time_op(lambda: net.forward(xn, sn, wsn), flush, reps=reps)
+    rec(f"table7_convnet_forward_batch{Bn}", ms, best, ops=opsn,
+        note=f"{Bn / ms * 1e3:.0f} images/s; 6 conv + 3 FC layers in one qnn_convnet_forward call, weights prepared once")
+
+
 def run_extras(q, bench, peaks, algo):
     """Other paper-shaped workloads, one record each (device time, L2 flushed): packers against the HBM
     roofline, products in binary Tops/s."""
@@ -408,23 +429,7 @@ def run_extras(q, bench, peaks, algo):
 
     # the whole CIFAR-10 ConvNet of Table 7 (first layer on 8-bit pixels, pooled thresholds, FC head), one call per pass
     for Bn in (128, 1024):
-        wln = workloads.cifar_convnet(B=Bn)
-        net = q.ConvNet(3, 32, 32, wln.conv_W, wln.conv_pool, wln.fc_W, wln.Ts, wln.flips)
-        wsn = net.workspace(Bn)
-        xn = wln.X.cuda()
-        sn = torch.zeros(Bn, net.n_out, dtype=torch.int32, device="cuda")
-        opsn, c_, h_, w_ = 0.0, 3, 32, 32
-        for Wc, pool in zip(wln.conv_W, wln.conv_pool):
-            opsn += 2.0 * Bn * h_ * w_ * Wc.shape[0] * 9 * c_ * (8 if c_ == 3 else 1)
-            c_ = Wc.shape[0]
-            if pool:
-                h_, w_ = h_ // 2, w_ // 2
-        for Wf in wln.fc_W:
-            opsn += 2.0 * Bn * Wf.shape[0] * Wf.shape[1]
-        ms, best = _time_op(lambda: net.forward(xn, sn, wsn), flush)
-        rec(f"table7_convnet_forward_batch{Bn}", ms, best, ops=opsn,
-            note=f"{Bn / ms * 1e3:.0f} images/s; 6 conv + 3 FC layers in one qnn_convnet_forward call, weights prepared once")
-        del net, wsn, xn, sn
+        convnet_record(q, Bn, flush, rec)
 
     # config 5: LSTM gate 4b x 4b and the square sweep
     wl5 = workloads.lstm_gate()
@@ -461,6 +466,8 @@ def main():
     ap.add_argument("--algo", default="auto", choices=["auto", "popc", "tc_i8", "b1_mma", "tc_fp4"])
     ap.add_argument("--no-extras", action="store_true", help="skip the per-config extra records")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--convnet-only", type=int, default=0, metavar="BATCH",
+                    help="time only the Table 7 ConvNet forward at this batch and print its record (one GPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -471,6 +478,18 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     from paper_1609_07061_b200 import binding as q
+    if args.convnet_only > 0:
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+        def flush():
+            flush_buf.fill_(1)
+            flush_buf.sum()
+        out = []
+        convnet_record(q, args.convnet_only, flush, lambda name, ms, best, bytes_=None, ops=None, note=None: out.append(
+            {"name": name, "ms": round(ms, 5), "ms_best": round(best, 5), "binary_Tops": round(ops / ms / 1e9, 2), "note": note}),
+            reps=max(args.steps if args.steps != 200 else 7, 1))
+        print(json.dumps(out[0]))
+        return
     rank, world, local = _dist_setup(args.gpus)
     algo = {"auto": q.QNN_ALGO_AUTO, "popc": q.QNN_ALGO_POPC, "tc_i8": q.QNN_ALGO_TC_I8, "b1_mma": q.QNN_ALGO_B1_MMA,
             "tc_fp4": q.QNN_ALGO_TC_FP4}[args.algo]
