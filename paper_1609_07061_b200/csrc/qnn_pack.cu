@@ -10,7 +10,9 @@ namespace qnn {
 // Row-major packing: source [rows, K] -> words [rows, ceil(K/32)].
 // A warp owns a (row, chunk) pair; a chunk is 128*UNROLL elements.  Each lane
 // loads UNROLL 16-byte vectors (4 elements each), turns each into a nibble and
-// the warp ORs the nibbles of 8 neighbouring lanes into one word.
+// the warp ORs the nibbles of 8 neighbouring lanes into one word.  Sources give
+// a vector either in one step (nibble) or as a raw load and a later conversion
+// (raw, nib_of), which lets a full chunk's loads be issued back to back.
 // --------------------------------------------------------------------------
 
 struct SignSrc {
@@ -23,6 +25,11 @@ struct SignSrc {
         const float4 v = __ldcs(reinterpret_cast<const float4 *>(x + r * ld + k));
         return (uint32_t)(v.x >= 0.0f) | ((uint32_t)(v.y >= 0.0f) << 1) | ((uint32_t)(v.z >= 0.0f) << 2) |
                ((uint32_t)(v.w >= 0.0f) << 3);
+    }
+    __device__ __forceinline__ int4 raw(int64_t r, int64_t k) const { return __ldcs(reinterpret_cast<const int4 *>(x + r * ld + k)); }
+    __device__ __forceinline__ uint32_t nib_of(const int4 v, int64_t) const
+    {
+        return (uint32_t)(__int_as_float(v.x) >= 0.0f) | ((uint32_t)(__int_as_float(v.y) >= 0.0f) << 1) | ((uint32_t)(__int_as_float(v.z) >= 0.0f) << 2) | ((uint32_t)(__int_as_float(v.w) >= 0.0f) << 3);
     }
     __host__ bool vector_ok() const { return (ld % 4 == 0) && aligned(x, 16); }
 };
@@ -51,15 +58,29 @@ struct ThresholdSrc {
         }
         return n;
     }
+    __device__ __forceinline__ int4 raw(int64_t r, int64_t k) const { return __ldcs(reinterpret_cast<const int4 *>(s + r * ld + k)); }
+    __device__ __forceinline__ uint32_t nib_of(const int4 v, int64_t k) const
+    {
+        const int4 t = __ldg(reinterpret_cast<const int4 *>(thr + k));
+        uint32_t n = (uint32_t)(v.x >= t.x) | ((uint32_t)(v.y >= t.y) << 1) | ((uint32_t)(v.z >= t.z) << 2) | ((uint32_t)(v.w >= t.w) << 3);
+        if (flip) {
+            const uint32_t f = __ldg(reinterpret_cast<const uint32_t *>(flip + k));
+            n ^= (uint32_t)((f & 0xffu) != 0) | ((uint32_t)((f & 0xff00u) != 0) << 1) | ((uint32_t)((f & 0xff0000u) != 0) << 2) | ((uint32_t)((f & 0xff000000u) != 0) << 3);
+        }
+        return n;
+    }
     __host__ bool vector_ok() const
     {
         return (ld % 4 == 0) && aligned(s, 16) && aligned(thr, 16) && (!flip || aligned(flip, 4));
     }
 };
 
-// (eight resident blocks per SM: this HBM-bound kernel lives on the bytes it keeps in flight)
+// This HBM-bound kernel lives on the bytes it keeps in flight: a full chunk's UNROLL 16-byte loads are all issued
+// before the first one is used (64 registers at four resident blocks per SM hold them).  Measured on B200,
+// 10000 x 4096: sign 38.9 -> 30.7 us, threshold 47.1 -> 38.9 us against eight blocks of 32-register threads with
+// four loads each; sixteen loads, or three or six blocks, are slower.
 template <class Src, int UNROLL, bool VEC>
-__global__ void __launch_bounds__(256, 8) row_pack_kernel(Src src, int64_t rows, int64_t K, uint32_t *__restrict__ out,
+__global__ void __launch_bounds__(256, 4) row_pack_kernel(Src src, int64_t rows, int64_t K, uint32_t *__restrict__ out,
                                                        int64_t ld_words, int32_t *__restrict__ row_popc,
                                                        int64_t chunks_per_row)
 {
@@ -72,18 +93,26 @@ __global__ void __launch_bounds__(256, 8) row_pack_kernel(Src src, int64_t rows,
         const int64_t r = item / chunks_per_row;
         const int64_t k0 = (item - r * chunks_per_row) * CHUNK;
         uint32_t nib[UNROLL];
+        if (VEC && k0 + CHUNK <= K) {
+            int4 raw[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const int64_t k = k0 + u * 128 + lane * 4;
-            uint32_t n = 0;
-            if (VEC && k + 4 <= K) {
-                n = src.nibble(r, k);
-            } else {
+            for (int u = 0; u < UNROLL; ++u) raw[u] = src.raw(r, k0 + u * 128 + lane * 4);
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (k + j < K) n |= src.bit(r, k + j) << j;
+            for (int u = 0; u < UNROLL; ++u) nib[u] = src.nib_of(raw[u], k0 + u * 128 + lane * 4);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int64_t k = k0 + u * 128 + lane * 4;
+                uint32_t n = 0;
+                if (VEC && k + 4 <= K) {
+                    n = src.nibble(r, k);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (k + j < K) n |= src.bit(r, k + j) << j;
+                }
+                nib[u] = n;
             }
-            nib[u] = n;
         }
         int pc = 0;
 #pragma unroll
@@ -112,11 +141,11 @@ static int launch_row_pack(const Src &src, int64_t rows, int64_t K, uint32_t *ou
 {
     if (rows == 0 || K == 0) return QNN_OK;
     if (row_popc) QNN_CUDA(cudaMemsetAsync(row_popc, 0, sizeof(int32_t) * (size_t)rows, st));
-    constexpr int UNROLL = 4;
+    constexpr int UNROLL = 8;
     const int64_t chunks = ceil_div(K, 128 * UNROLL);
     const int64_t warps = rows * chunks;
     const int64_t blocks_needed = ceil_div(warps, 8);
-    const int64_t cap = (int64_t)sm_count() * 8;
+    const int64_t cap = (int64_t)sm_count() * 4;
     const int blocks = (int)(blocks_needed < cap ? blocks_needed : cap);
     if (src.vector_ok())
         row_pack_kernel<Src, UNROLL, true><<<blocks, 256, 0, st>>>(src, rows, K, out, ld_words, row_popc, chunks);
