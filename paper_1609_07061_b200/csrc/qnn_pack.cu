@@ -322,6 +322,27 @@ __global__ void __launch_bounds__(128) trans_pack_kernel(const float *__restrict
         for (int c = 0; c < 4; ++c) word[p][c] = 0;
     int sum[4] = {0, 0, 0, 0};
     const int64_t kbase = kw * 32;
+    if (VEC && n0 + 4 <= N && kbase + 32 <= K) {
+        // whole word, whole vectors: sixteen loads issued before the first is converted, twice (measured on B200,
+        // 4096 x 4096: 26.6 -> 18.4 us; the unrolled loop below keeps only a few loads in flight)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float4 t[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) t[j] = __ldcs(reinterpret_cast<const float4 *>(src + (kbase + h * 16 + j) * ldw + n0));
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float v[4] = {t[j].x, t[j].y, t[j].z, t[j].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int q = code(v[c]);
+                    sum[c] += q;
+#pragma unroll
+                    for (int p = 0; p < NB; ++p) word[p][c] |= (uint32_t)((q >> p) & 1) << (h * 16 + j);
+                }
+            }
+        }
+    } else
 #pragma unroll 8
     for (int j = 0; j < 32; ++j) {
         const int64_t k = kbase + j;
