@@ -245,21 +245,33 @@ __global__ void __launch_bounds__(256) gemm_popc_skinny_kernel(const uint32_t *_
 #pragma unroll
         for (int n = 0; n < SKINNY_N; ++n) acc[n] = 0;
         const uint32_t *arow = a + (live ? m : m0) * lda;
-        for (int k = part * 4; k < kwords; k += 32) {
-            uint4 av;
-            if (vec && k + 4 <= kwords) {
-                av = __ldcs(reinterpret_cast<const uint4 *>(arow + k));
-            } else {
-                av.x = arow[k];
-                av.y = k + 1 < kwords ? arow[k + 1] : 0u;
-                av.z = k + 2 < kwords ? arow[k + 2] : 0u;
-                av.w = k + 3 < kwords ? arow[k + 3] : 0u;
+        // four 16-byte pieces of the row per lane are loaded before any of them is used: the kernel is a stream over A,
+        // and one load in flight per lane leaves it waiting out a memory latency per piece
+        for (int k0 = part * 4; k0 < kwords; k0 += 128) {
+            uint4 av[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = k0 + 32 * u;
+                if (vec && k + 4 <= kwords) {
+                    av[u] = __ldcs(reinterpret_cast<const uint4 *>(arow + k));
+                } else {
+                    av[u].x = k < kwords ? arow[k] : 0u;
+                    av[u].y = k + 1 < kwords ? arow[k + 1] : 0u;
+                    av[u].z = k + 2 < kwords ? arow[k + 2] : 0u;
+                    av[u].w = k + 3 < kwords ? arow[k + 3] : 0u;
+                }
             }
 #pragma unroll
-            for (int n = 0; n < SKINNY_N; ++n) {
-                if (n < N) {
-                    const uint4 bv = *reinterpret_cast<const uint4 *>(bs + n * kw4 + k);
-                    acc[n] += __popc(av.x ^ bv.x) + __popc(av.y ^ bv.y) + __popc(av.z ^ bv.z) + __popc(av.w ^ bv.w);
+            for (int u = 0; u < 4; ++u) {
+                const int k = k0 + 32 * u;
+                if (k < kwords) {
+#pragma unroll
+                    for (int n = 0; n < SKINNY_N; ++n) {
+                        if (n < N) {
+                            const uint4 bv = *reinterpret_cast<const uint4 *>(bs + n * kw4 + k);
+                            acc[n] += __popc(av[u].x ^ bv.x) + __popc(av[u].y ^ bv.y) + __popc(av[u].z ^ bv.z) + __popc(av[u].w ^ bv.w);
+                        }
+                    }
                 }
             }
         }
