@@ -283,6 +283,31 @@ def _time_op(fn, flush, reps=7, warm=3):
     return statistics.median(ts), min(ts)
 
 
+def _time_graph(fn, flush, n=100, reps=5):
+    """Per-call device time (ms) of n back-to-back calls of fn() captured in one CUDA graph: what remains of a small
+    operation once launch latency is amortised (the calls inside a replay run warm)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(n):
+                fn()
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); g.replay(); b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b) / n)
+    return statistics.median(ts), min(ts)
+
+
 def convnet_record(q, Bn, flush, rec, reps=7):
     """Times one qnn_convnet_forward call of the Table 7 network at batch Bn (weights prepared once, L2 flushed)."""
     from paper_1609_07061_b200 import workloads
@@ -356,6 +381,17 @@ def run_extras(q, bench, peaks, algo):
     ms, best = _time_op(cold, flush)
     rec("c1_layer_cold_weights", ms, best, bytes_=(M * K + K * N) * 4.0 + 2 * (M + N) * ld * 4 + M * N * 4,
         ops=2.0 * M * N * K)
+
+    # Items whose roofline time is below a few microseconds cannot approach it in a single launch (a launch alone costs
+    # 3-5 us): the same calls 100 times back to back inside one CUDA graph show what is left without the launch latency.
+    ms, best = _time_graph(lambda: q.qnn_quantize_pack_sign(Xd, M, K, K, a, ld), flush)
+    rec("c1_pack_X_100x4096_x100_in_one_graph", ms, best, bytes_=M * K * 4.125, note="per call; 100 calls in one CUDA graph")
+    ms, best = _time_graph(lambda: q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, out, N, algo, ws), flush)
+    rec("c1_xnor_gemm_100x4096x4096_x100_in_one_graph", ms, best, bytes_=(M + N) * ld * 4 + M * N * 4, ops=2.0 * M * N * K,
+        note="per call; 100 calls in one CUDA graph")
+    ms, best = _time_graph(warm_prepacked, flush)
+    rec("c1_xnor_gemm_prepacked_weights_x100_in_one_graph", ms, best, bytes_=(M + N) * ld * 4 + M * N * 4, ops=2.0 * M * N * K,
+        note="per call; 100 calls in one CUDA graph")
     del Xd, Wd
 
     # large row-major sign pack and standalone threshold pack (HBM-bound steps on tensors >= 32 MB)

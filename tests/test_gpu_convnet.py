@@ -170,3 +170,31 @@ def test_convnet_argument_errors(q):
     with pytest.raises(q.QnnError) as e:
         q.qnn_convnet_forward(wl.X.cuda(), 2, 8, 8, net.layers, net.prepared, scores, torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
     assert e.value.status == q.QNN_ERR_INVALID_ARG
+
+
+def test_network_runners_replay_from_a_cuda_graph(q):
+    """Both whole-network calls are allocation-free and asynchronous: captured once in a CUDA graph, a replay
+    must reproduce the oracle's scores (the tensor-core kernels inside are launched with programmatic stream
+    serialisation, which the capture has to carry over)."""
+    B = 64
+    wl = workloads.cifar_convnet(B=B, H=16, W=16, widths=(128, 128, 256, 256), fc=(256, 10), seed=5, thr=24)
+    net = q.ConvNet(3, 16, 16, wl.conv_W, wl.conv_pool, wl.fc_W, wl.Ts, wl.flips)
+    ws = net.workspace(B)
+    x = wl.X.cuda()
+    scores = torch.zeros(B, net.n_out, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        net.forward(x, scores, ws)                    # first call outside the capture (one-time kernel attributes)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            net.forward(x, scores, ws)
+    torch.cuda.synchronize()
+    want = oracle.convnet_forward(wl.X.numpy().astype(np.int32), _oracle_layers(wl))
+    for _ in range(3):
+        scores.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        np.testing.assert_array_equal(scores.cpu().numpy(), want)
