@@ -18,6 +18,8 @@ Pins (what each routine is checked against, other than itself) live in
   conv2d          library conv2d in float64 on +-1 tensors padded with +1,
                   the 1x1 case against the matrix product, all-ones input
   mlp_forward     Algorithm 4 step by step with the routines above
+  ap2 / log_quant float64 round(log2|x|) away from ties, exact powers of two, the factor-sqrt(2)
+                  bound, monotonicity, clipping, zero / infinities / NaN
   maxpool2x2      library max_pool2d in float64; the identity that pooling the
                   integer sums and then thresholding equals OR (AND where the
                   comparison is flipped) of the thresholded bits, by brute force
@@ -196,6 +198,23 @@ def conv2d(X, Wt, stride: int = 1, pad: int = 1, pad_value: int = 1) -> np.ndarr
     rc = _load().qo_conv2d(_ptr(X), _ptr(Wt), B, C, H, W, Cout, KH, KW, stride, pad, pad_value, _ptr(out))
     _check(rc, "conv2d")
     return out
+
+
+def ap2_exponent(x) -> np.ndarray:
+    """round(log2|x|) of AP2 (Algorithm 2's caption); INT32_MIN for 0, INT32_MAX for inf / NaN."""
+    x = _c(x, np.float32)
+    e = np.empty(x.shape, np.int32)
+    _check(_load().qo_ap2_exponent(_ptr(x), ctypes.c_int64(x.size), _ptr(e)), "ap2_exponent")
+    return e
+
+
+def log_quant(x, emin: int, emax: int) -> np.ndarray:
+    """Eq. 10 with magnitudes clipped to [2^emin, 2^emax], as integers sign * 2^(e - emin)."""
+    x = _c(x, np.float32)
+    v = np.empty(x.shape, np.int32)
+    _check(_load().qo_log_quant(_ptr(x), ctypes.c_int64(x.size), ctypes.c_int(emin), ctypes.c_int(emax), _ptr(v)),
+           "log_quant")
+    return v
 
 
 def maxpool2x2(x) -> np.ndarray:

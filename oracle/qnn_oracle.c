@@ -158,6 +158,47 @@ int qo_planewise_gemm(const int32_t *QA, int ka, const int32_t *B, int64_t M, in
     return overflow;
 }
 
+/* AP2 (caption of Algorithm 2): AP2(x) = sign(x) * 2^round(log2|x|), returned as the exponent e = round(log2|x|).
+ * |x| = m * 2^f with m in [1, 2) (frexpf gives m/2 and f+1): log2|x| = f + log2 m, and log2 m >= 1/2 exactly when
+ * m >= sqrt(2).  sqrt(2) is not a float, so no input sits on the tie: m rounds up when it is above the largest
+ * float below sqrt(2).  x = 0 has no logarithm: e = INT32_MIN (it clips to the smallest level in Eq. 10);
+ * infinities and NaN give INT32_MAX (they clip to the largest). */
+static int32_t ap2_exponent(float x)
+{
+    float ax = fabsf(x);
+    if (!(ax == ax) || isinf(ax)) return INT32_MAX;
+    if (ax == 0.0f) return INT32_MIN;
+    int f;
+    float half_m = frexpf(ax, &f);          /* ax = half_m * 2^f, half_m in [0.5, 1) */
+    float m = half_m * 2.0f;                /* exact */
+    int32_t e = f - 1;
+    const float below_sqrt2 = 1.41421353816986083984375f;   /* largest float < sqrt(2) */
+    if (m > below_sqrt2) e += 1;
+    return e;
+}
+
+int qo_ap2_exponent(const float *x, int64_t n, int32_t *e)
+{
+    if (n < 0) return 2;
+    for (int64_t i = 0; i < n; ++i) e[i] = ap2_exponent(x[i]);
+    return 0;
+}
+
+/* Eq. 10: LogQuant(x) = Clip(AP2(x), minV, maxV) with minV = 2^emin, maxV = 2^emax as bounds on the magnitude.
+ * The result is returned as the integer v = sign * 2^(e - emin), e = clamp(round(log2|x|), emin, emax), i.e. the
+ * quantised value in units of minV: |v| in {1, 2, 4, ..., 2^(emax-emin)}; sign as in Eq. 1 (x >= 0 gives +1). */
+int qo_log_quant(const float *x, int64_t n, int emin, int emax, int32_t *v)
+{
+    if (n < 0 || emax < emin || emax - emin > 30) return 2;
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t e = ap2_exponent(x[i]);
+        if (e < emin) e = emin;
+        if (e > emax) e = emax;
+        v[i] = sgn(x[i]) * (int32_t)(1 << (e - emin));
+    }
+    return 0;
+}
+
 /* Algorithm 4: a^b = Sign(BatchNorm(a, theta)) with the batch-norm folded to a
  * per-channel integer comparison: bit = (s >= T[n]) xor flip[n].  Output is
  * one byte (0/1) per element, not packed.  flip may be NULL (all zero). */

@@ -121,3 +121,57 @@ def test_lstm_levels_roundtrip_and_real_product():
     got = oracle.int_gemm(va, vb)
     real = wl.X.numpy().astype(np.float64) @ wl.W.numpy().astype(np.float64)
     np.testing.assert_allclose(got / 225.0, real, atol=1e-4)
+
+
+def test_ap2_exponent_pins():
+    """AP2(x) = sign(x) 2^round(log2|x|): float64 logarithms away from ties, closed forms at and around them."""
+    rng = np.random.default_rng(7)
+    x = (rng.standard_normal(20000) * np.exp(rng.uniform(-20, 20, 20000))).astype(np.float32)
+    x = x[x != 0]
+    l2 = np.log2(np.abs(x.astype(np.float64)))
+    far = np.abs(l2 - np.floor(l2) - 0.5) > 1e-6               # a float64 log cannot be trusted to decide a near tie
+    e = oracle.ap2_exponent(x)
+    np.testing.assert_array_equal(e[far], np.round(l2[far]).astype(np.int32))
+    # the chosen power of two is within a factor sqrt(2) of |x|, on every input
+    ratio = np.abs(x.astype(np.float64)) / np.exp2(e.astype(np.float64))
+    assert np.all(ratio > 2 ** -0.5) and np.all(ratio < 2 ** 0.5)
+    # powers of two are fixed points; sign does not matter
+    p = np.array([2.0 ** k for k in range(-30, 31)], np.float32)
+    np.testing.assert_array_equal(oracle.ap2_exponent(p), np.arange(-30, 31))
+    np.testing.assert_array_equal(oracle.ap2_exponent(-p), np.arange(-30, 31))
+    # the two floats around sqrt(2): the one below rounds down, the one above rounds up (at every scale)
+    lo = np.float32(1.41421353816986083984375)
+    hi = np.nextafter(lo, np.float32(2.0))
+    assert float(lo) ** 2 < 2.0 < float(hi) ** 2
+    for k in (-5, 0, 9):
+        s = np.float32(2.0 ** k)
+        np.testing.assert_array_equal(oracle.ap2_exponent(np.array([lo * s, hi * s], np.float32)), [k, k + 1])
+    # 1.5 has log2 = 0.585 -> 1;  1.25 -> 0;  3 -> 2 (log2 3 = 1.585);  denormals have exponents below -126
+    np.testing.assert_array_equal(oracle.ap2_exponent(np.array([1.5, 1.25, 3.0, 0.75], np.float32)), [1, 0, 2, 0])
+    assert oracle.ap2_exponent(np.array([1e-40], np.float32))[0] < -126
+    # monotone in |x|
+    xs = np.sort(np.abs(x))
+    assert np.all(np.diff(oracle.ap2_exponent(xs)) >= 0)
+    sp = oracle.ap2_exponent(np.array([0.0, -0.0, np.inf, -np.inf, np.nan], np.float32))
+    assert sp[0] == sp[1] == np.iinfo(np.int32).min and sp[2] == sp[3] == sp[4] == np.iinfo(np.int32).max
+
+
+def test_log_quant_pins():
+    """Eq. 10: magnitudes clip to [2^emin, 2^emax]; result in units of 2^emin, sign of Eq. 1."""
+    x = np.array([0.0, -0.0, 1e-9, -1e-9, 0.24, 0.26, -0.7, 0.71, 1.0, -1.4, 1.42, 3.0, 100.0, -100.0, np.inf, -np.inf, np.nan],
+                 np.float32)
+    v = oracle.log_quant(x, -2, 1)               # levels 1/4, 1/2, 1, 2  ->  1, 2, 4, 8
+    np.testing.assert_array_equal(v, [1, 1, 1, -1, 1, 1, -2, 4, 4, -4, 8, 8, 8, -8, 8, -8, -8])
+    # agreement with the literal formula in float64 on random data away from ties
+    rng = np.random.default_rng(3)
+    y = (rng.standard_normal(5000) * 2.0).astype(np.float32)
+    y = y[y != 0]
+    l2 = np.log2(np.abs(y.astype(np.float64)))
+    far = np.abs(l2 - np.floor(l2) - 0.5) > 1e-6
+    want = np.where(y >= 0, 1, -1) * np.exp2(np.clip(np.round(l2), -3, 3) + 3)
+    np.testing.assert_array_equal(oracle.log_quant(y, -3, 3)[far], want[far].astype(np.int32))
+    # at most (emax - emin + 1) magnitudes, all powers of two
+    mags = np.unique(np.abs(oracle.log_quant(y, -3, 3)))
+    assert set(mags.tolist()) <= {1, 2, 4, 8, 16, 32, 64}
+    with pytest.raises(ValueError):
+        oracle.log_quant(y, 2, 1)
