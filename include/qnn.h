@@ -55,7 +55,7 @@
 extern "C" {
 #endif
 
-#define QNN_VERSION 210
+#define QNN_VERSION 220
 
 /* status codes */
 #define QNN_OK 0
@@ -401,6 +401,25 @@ QNN_API int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, 
 
 QNN_API size_t qnn_mlp_workspace_bytes(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int algo,
                                int host_io);
+
+/* Logarithmic quantiser, Eq. 10: LogQuant(x) = Clip(AP2(x), minV, maxV) with
+ * AP2(x) = sign(x) * 2^round(log2|x|) (caption of Algorithm 2), the magnitude
+ * clipped to minV = 2^emin ... maxV = 2^emax.  Each element is written as the
+ * int8 value sign * 2^(e - emin), e = clamp(round(log2|x|), emin, emax): the
+ * quantised value in units of minV, which is an operand of the int8 tensor-core
+ * form as it stands (qnn_tc_gemm with form QNN_FORM_I8, mode QNN_MODE_PM1 and
+ * planes = emax - emin + 1, so that |value| <= 2^planes - 1); the product of two such
+ * matrices is the exact integer sum in units of minV_a * minV_b.
+ * Rounding: log2|x| has no ties on floats (sqrt(2) is not a float); zero and
+ * denormals clip to emin, infinities and NaN to emax; sign as in Eq. 1.
+ *   x    device, float [rows, ldx]
+ *   out  device, int8 [rows, ld_bytes], ld_bytes >= K rounded up to 32 and a
+ *        multiple of 4 (of 16 to serve as a tensor-core operand); bytes K ...
+ *        roundup(K, 32) of every row are written as zero
+ * Errors: INVALID_ARG, UNSUPPORTED (emax - emin > 6: 2^7 does not fit int8),
+ * ALIGNMENT, CUDA. */
+QNN_API int qnn_logquant_pack_i8(const float *x, int64_t rows, int64_t K, int64_t ldx, int emin, int emax, void *out,
+                                 int64_t ld_bytes, void *stream);
 
 /* ------------------------------------------------------------------------- */
 /* The ConvNet of Table 7                                                     */

@@ -99,6 +99,7 @@ _SIGS = {
     "qnn_conv_prepared_bytes": (sz, [i32, i32, i32, i32, i32]),
     "qnn_conv_prepare": (i32, [vp, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
     "qnn_binary_conv2d_prepared": (i32, [ctypes.POINTER(qnn_conv_io), i32, i32, i32, i32, vp, i32, i32, i32, i32, vp, sz, vp]),
+    "qnn_logquant_pack_i8": (i32, [vp, i64, i64, i64, i32, i32, vp, i64, vp]),
     "qnn_conv2d_u8_workspace_bytes": (sz, [i32, i32, i32, i32, i32, i32, i32, i32]),
     "qnn_conv2d_u8": (i32, [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]),
     "qnn_maxpool2x2_bits": (i32, [vp, i32, i32, i32, i32, vp, vp, vp, i32, vp]),
@@ -337,6 +338,10 @@ def qnn_mlp_forward_host(x_host, M, in_bits, layers, scores_host, algo=QNN_ALGO_
     wp, wb = _ws(ws)
     _ck(_lib.qnn_mlp_forward_host(_p(x_host), M, in_bits, layers, len(layers), _p(scores_host), algo, wp, wb,
                                   _stream()), "qnn_mlp_forward_host")
+
+
+def qnn_logquant_pack_i8(x, rows, K, ldx, emin, emax, out, ld_bytes):
+    _ck(_lib.qnn_logquant_pack_i8(_p(x), rows, K, ldx, emin, emax, _p(out), ld_bytes, _stream()), "qnn_logquant_pack_i8")
 
 
 def qnn_conv2d_u8_workspace_bytes(B, C, H, W, Cout, KH, KW, pad) -> int:

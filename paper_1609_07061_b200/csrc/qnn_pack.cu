@@ -395,6 +395,52 @@ static int launch_trans_pack_nb(const float *w, int64_t K, int64_t N, int64_t ld
     return check_launch(what);
 }
 
+// --------------------------------------------------------------------------
+// Logarithmic quantiser (Eq. 10): AP2(x) = sign(x) * 2^round(log2|x|) with the
+// magnitude clipped to [2^emin, 2^emax], written as the int8 value
+// sign * 2^(e - emin) -- directly an operand of the int8 tensor-core form.
+// round(log2|x|) comes from the float's own fields: the exponent, plus one when
+// the mantissa is above the largest float below sqrt(2) (sqrt(2) is not a
+// float, so there are no ties).  Zero and denormals clip to emin, infinities
+// and NaN to emax; the sign is Eq. 1's (x >= 0 gives +1, NaN gives -1).
+// --------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t logquant_byte(float x, int emin, int emax)
+{
+    const uint32_t a = __float_as_uint(x) & 0x7fffffffu;
+    int e;
+    if (a >= 0x7f800000u) e = emax;
+    else if (a < 0x00800000u) e = emin;
+    else {
+        e = (int)(a >> 23) - 127 + (int)((a & 0x7fffffu) > 0x3504f3u);
+        e = e < emin ? emin : (e > emax ? emax : e);
+    }
+    const int v = 1 << (e - emin);
+    return (uint32_t)(x >= 0.0f ? v : -v) & 0xffu;
+}
+
+// One thread per 4 consecutive elements of a row (kq = ceil(Kz / 4) groups per row, Kz = K rounded up to 32: the
+// bytes between K and Kz are written as zero so that the row is a valid tensor-core operand).
+__global__ void __launch_bounds__(256) logquant_i8_kernel(const float *__restrict__ x, int64_t rows, int64_t K, int64_t ldx,
+                                                          int emin, int emax, uint8_t *__restrict__ out, int64_t ld_bytes,
+                                                          int64_t kq, bool vec)
+{
+    const int64_t total = rows * kq;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / kq, k = (i - r * kq) * 4;
+        uint32_t w = 0;
+        if (vec && k + 4 <= K) {
+            const float4 v = __ldcs(reinterpret_cast<const float4 *>(x + r * ldx + k));
+            w = logquant_byte(v.x, emin, emax) | (logquant_byte(v.y, emin, emax) << 8) | (logquant_byte(v.z, emin, emax) << 16) |
+                (logquant_byte(v.w, emin, emax) << 24);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (k + j < K) w |= logquant_byte(x[r * ldx + k + j], emin, emax) << (8 * j);
+        }
+        *reinterpret_cast<uint32_t *>(out + r * ld_bytes + k) = w;
+    }
+}
+
 }  // namespace qnn
 
 using namespace qnn;
@@ -524,6 +570,28 @@ int qnn_quantize_pack_kbit_t(const float *w, int64_t K, int64_t N, int64_t ldw, 
         case 7: return launch_trans_pack_nb<KbitCode, 7>(w, K, N, ldw, 1, 0, code, planes, ld_words, plane_stride_words, 0, row_sum_q, st, what);
         default: return launch_trans_pack_nb<KbitCode, 8>(w, K, N, ldw, 1, 0, code, planes, ld_words, plane_stride_words, 0, row_sum_q, st, what);
     }
+}
+
+int qnn_logquant_pack_i8(const float *x, int64_t rows, int64_t K, int64_t ldx, int emin, int emax, void *out, int64_t ld_bytes,
+                         void *stream)
+{
+    QNN_REQUIRE(rows >= 0 && K >= 0, QNN_ERR_INVALID_ARG, "qnn_logquant_pack_i8: negative size");
+    QNN_REQUIRE(emax >= emin && emin >= -126 && emax <= 127, QNN_ERR_INVALID_ARG,
+                "qnn_logquant_pack_i8: need -126 <= emin <= emax <= 127");
+    QNN_REQUIRE(emax - emin <= 6, QNN_ERR_UNSUPPORTED, "qnn_logquant_pack_i8: at most 7 levels (2^6 = 64) fit an int8 value");
+    if (rows == 0 || K == 0) return QNN_OK;
+    QNN_REQUIRE(x && out, QNN_ERR_INVALID_ARG, "qnn_logquant_pack_i8: NULL pointer");
+    const int64_t kz = (int64_t)round_up((size_t)K, 32);
+    QNN_REQUIRE(ldx >= K && ld_bytes >= kz, QNN_ERR_INVALID_ARG,
+                "qnn_logquant_pack_i8: ldx below K, or ld_bytes below K rounded up to 32");
+    QNN_REQUIRE(aligned(x, 4) && aligned(out, 4) && ld_bytes % 4 == 0, QNN_ERR_ALIGNMENT,
+                "qnn_logquant_pack_i8: pointers and the output row stride must be multiples of 4 bytes");
+    const int64_t kq = kz / 4;
+    const bool vec = (ldx % 4 == 0) && aligned(x, 16);
+    const int64_t need = ceil_div(rows * kq, 256), cap = (int64_t)sm_count() * 8;
+    logquant_i8_kernel<<<(int)(need < cap ? need : cap), 256, 0, as_stream(stream)>>>(x, rows, K, ldx, emin, emax,
+                                                                                     static_cast<uint8_t *>(out), ld_bytes, kq, vec);
+    return check_launch("qnn_logquant_pack_i8");
 }
 
 }  // extern "C"

@@ -193,3 +193,41 @@ def test_rescale_f32(q):
     scale = np.abs(np.float32(0.0123) * p) + np.abs(r)[:, None] + np.abs(c)[None, :] + 0.5
     assert np.max(np.abs(got - want) / scale) <= 1e-6
     y.check()
+
+
+@pytest.mark.parametrize("rows,K,ldx,emin,emax", [(7, 100, 100, -3, 3), (64, 4096, 4096, -2, 1), (3, 33, 40, 0, 0), (129, 784, 784, -6, 0),
+                                                   (5, 1, 4, -1, 2)])
+def test_logquant_pack_i8(q, rows, K, ldx, emin, emax):
+    """Eq. 10 / AP2: int8 values sign * 2^(e - emin) against the oracle, bit-exact; pad bytes up to 32-multiples zero."""
+    rng = np.random.default_rng(rows * 7 + K)
+    x = (rng.standard_normal((rows, ldx)) * np.exp(rng.uniform(-4, 4, (rows, ldx)))).astype(np.float32)
+    lo = np.float32(1.41421353816986083984375)
+    specials = [0.0, -0.0, np.inf, -np.inf, np.nan, 1e-40, -1e-40, lo, np.nextafter(lo, np.float32(2)), -lo, 0.5 * lo, 1.0, -1.0, 1.5, 3.0]
+    flat = x.reshape(-1)
+    n = min(len(specials), flat.size)
+    flat[:n] = np.array(specials[:n], np.float32)
+    kz = (K + 31) // 32 * 32
+    ld_bytes = kz + 16
+    out = Guarded((rows, ld_bytes), torch.uint8, fill=0x5C)
+    q.qnn_logquant_pack_i8(dev(x), rows, K, ldx, emin, emax, out.t, ld_bytes)
+    torch.cuda.synchronize()
+    got = out.t.cpu().numpy()
+    want = oracle.log_quant(x[:, :K], emin, emax)
+    np.testing.assert_array_equal(got[:, :K].view(np.int8).astype(np.int32), want)
+    assert not got[:, K:kz].any(), "bytes between K and the next multiple of 32 must be zero"
+    assert (got[:, kz:] == 0x5C).all(), "bytes past the written part of a row must stay untouched"
+    out.check()
+
+
+def test_logquant_argument_errors(q):
+    x = torch.zeros(4, 32, device="cuda")
+    out = torch.zeros(4, 32, dtype=torch.uint8, device="cuda")
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_pack_i8(x, 4, 32, 32, -4, 3, out, 32)          # 8 levels: 2^7 does not fit int8
+    assert e.value.status == q.QNN_ERR_UNSUPPORTED
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_pack_i8(x, 4, 32, 32, 2, 1, out, 32)
+    assert e.value.status == q.QNN_ERR_INVALID_ARG
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_pack_i8(x, 4, 20, 32, 0, 1, out, 20)           # row stride below K rounded up to 32
+    assert e.value.status == q.QNN_ERR_INVALID_ARG

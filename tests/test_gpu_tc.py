@@ -247,3 +247,38 @@ def test_tc_gemm_cta_pair_shapes(q, form_name, M, N, K, outputs):
         onb = words_per_row(N) * 16
         np.testing.assert_array_equal(of.t.cpu().numpy()[rows][:, :onb], form_ref(2 * wb.astype(np.int32) - 1, N, q.QNN_FORM_FP4, q))
         bits.check(); of.check()
+
+
+@pytest.mark.parametrize("M,N,K,la,lb", [(70, 40, 96, (-3, 3), None), (300, 130, 1000, (-2, 1), (-1, 2)), (129, 257, 4096, (-6, 0), (-3, 3)),
+                                          (5, 3, 31, (0, 0), (0, 2))])
+def test_logquant_products(q, M, N, K, la, lb):
+    """Logarithmically quantised activations (Eq. 10) times +-1 or logarithmically quantised weights on the int8
+    tensor-core form: exact integer sums in units of the two smallest levels."""
+    rng = np.random.default_rng(M + N + K)
+    X = (rng.standard_normal((M, K)) * 2.0).astype(np.float32)
+    Wt = (rng.standard_normal((N, K)) * 0.7).astype(np.float32)          # weights, one row per unit
+    va = oracle.log_quant(X, *la)
+    kz = (K + 31) // 32 * 32
+    ld = (kz + 15) // 16 * 16
+    a8 = torch.zeros(M, ld, dtype=torch.uint8, device="cuda")
+    q.qnn_logquant_pack_i8(dev(X), M, K, K, la[0], la[1], a8, ld)
+    b8 = torch.zeros(N, ld, dtype=torch.uint8, device="cuda")
+    if lb is None:
+        vb = oracle.sign(Wt)
+        bits = torch.zeros(N, (K + 31) // 32, dtype=torch.int32, device="cuda")
+        q.qnn_quantize_pack_sign(dev(Wt), N, K, K, bits, (K + 31) // 32)
+        q.qnn_tc_prepack(bits, 1, q.QNN_MODE_PM1, (K + 31) // 32, 0, N, K, q.QNN_FORM_I8, b8, ld)
+        pb = 1
+    else:
+        vb = oracle.log_quant(Wt, *lb)
+        q.qnn_logquant_pack_i8(dev(Wt), N, K, K, lb[0], lb[1], b8, ld)
+        pb = lb[1] - lb[0] + 1
+    want = oracle.int_gemm(va, vb.T)
+    out = Guarded((M, N), torch.int32, fill=-7)
+    A = q.tc_operand(a8, ld, q.QNN_FORM_I8, planes=la[1] - la[0] + 1, mode=q.QNN_MODE_PM1)
+    Bo = q.tc_operand(b8, ld, q.QNN_FORM_I8, planes=pb, mode=q.QNN_MODE_PM1)
+    q.qnn_tc_gemm(A, Bo, M, N, K, out=out.t, ldo=N)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    np.testing.assert_array_equal(out.t.cpu().numpy(), want)
+    out.check()
