@@ -198,3 +198,22 @@ def test_network_runners_replay_from_a_cuda_graph(q):
         torch.cuda.synchronize()
         assert q.qnn_device_status() == 0, q.qnn_last_error()
         np.testing.assert_array_equal(scores.cpu().numpy(), want)
+
+
+def test_degenerate_sizes(q):
+    """Empty batches and images without a 2 x 2 window are valid no-ops; nothing is written."""
+    wl = workloads.cifar_convnet(B=1, H=8, W=8, widths=(8, 8), fc=(10,), seed=5, thr=3)
+    net = q.ConvNet(3, 8, 8, wl.conv_W, wl.conv_pool, wl.fc_W, wl.Ts, wl.flips)
+    scores = Guarded((1, 10), torch.int32, fill=-7)
+    q.qnn_convnet_forward(wl.X.cuda(), 0, 8, 8, net.layers, net.prepared, scores.t, None)       # B = 0: no workspace needed
+    bits = torch.zeros(2, 1, 5, 1, dtype=torch.int32, device="cuda")
+    ob = Guarded((2, 0, 2, 1), torch.int32, fill=0)
+    q.qnn_maxpool2x2_bits(bits, 2, 1, 5, 8, None, ob.t, None, 0)                                 # a single row: no window
+    q.qnn_maxpool2x2_bits(bits, 0, 4, 4, 8, None, ob.t, None, 0)
+    out = Guarded((4, 32), torch.uint8, fill=0x5C)
+    q.qnn_logquant_pack_i8(torch.zeros(4, 8, device="cuda"), 0, 8, 8, -1, 1, out.t, 32)
+    q.qnn_logquant_pack_i8(torch.zeros(4, 8, device="cuda"), 4, 0, 8, -1, 1, out.t, 32)
+    torch.cuda.synchronize()
+    assert (scores.t.cpu().numpy() == -7).all() and (out.t.cpu().numpy() == 0x5C).all()
+    for g in (scores, ob, out):
+        g.check()
