@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <atomic>
 #include <climits>
+#include <cstdlib>
 #include "qnn_internal.cuh"
 
 namespace qnn {
@@ -22,6 +23,12 @@ int fail(int code, const char *fmt, ...)
 }
 
 void clear_error() { g_err[0] = 0; }
+
+bool pdl_enabled()
+{
+    static const bool on = [] { const char *e = getenv("QNN_PDL"); return !(e && e[0] == '0'); }();
+    return on;
+}
 void profile_arm(cudaEvent_t a, cudaEvent_t b, int skip);
 
 int check_launch(const char *what)

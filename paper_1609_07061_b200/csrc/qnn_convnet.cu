@@ -21,6 +21,8 @@ __global__ void __launch_bounds__(256) im2col_u8_kernel(const uint8_t *__restric
                                                         int pad, int pad_code, int Ho, int Wo, uint8_t *__restrict__ dst, int P,
                                                         int64_t total)
 {
+    griddep_launch_dependents();
+    griddep_wait();
     const int K = KH * KW * C;
     const int pieces = P >> 4;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -86,6 +88,7 @@ __global__ void __launch_bounds__(256) maxpool2x2_bits_kernel(const uint32_t *__
                                                               uint8_t *__restrict__ out_form, int kind, int64_t total)
 {
     __shared__ uint32_t fmask[64];
+    griddep_launch_dependents();
     for (int cw = threadIdx.x; cw < Cw; cw += blockDim.x) {
         uint32_t m = 0;
         if (flip != nullptr)
@@ -96,6 +99,7 @@ __global__ void __launch_bounds__(256) maxpool2x2_bits_kernel(const uint32_t *__
         fmask[cw] = m;
     }
     __syncthreads();
+    griddep_wait();                                  // the flips above are constants; the bits below are the previous kernel's
     const int Ho = H >> 1, Wo = W >> 1;
     const uint32_t tail = (C & 31) ? ((1u << (C & 31)) - 1u) : 0xffffffffu;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -170,7 +174,7 @@ int conv_u8_run(const uint8_t *x, int B, int C, int H, int W, const uint8_t *wf,
 {
     if (l.M == 0) return QNN_OK;
     const int64_t total = l.M * (l.Pa / 16);
-    im2col_u8_kernel<<<grid_for(total), 256, 0, st>>>(x, C, H, W, KH, KW, pad, pad_code, l.Ho, l.Wo, col, l.Pa, total);
+    QNN_CUDA(launch_pdl(im2col_u8_kernel, dim3(grid_for(total)), dim3(256), 0, st, x, C, H, W, KH, KW, pad, pad_code, l.Ho, l.Wo, col, l.Pa, total));
     if (int rc = check_launch("first-layer im2col")) return rc;
     GemmArgs g{};
     g.ka = 8; g.a_mode = QNN_MODE_U01; g.kb = 1; g.b_mode = QNN_MODE_PM1;
@@ -193,8 +197,8 @@ int maxpool_run(const uint32_t *bits, int B, int H, int W, int C, const uint8_t 
     const int Cw = (int)ceil_div(C, 32);
     const int64_t total = (int64_t)B * (H / 2) * (W / 2) * Cw;
     if (total == 0) return QNN_OK;
-    maxpool2x2_bits_kernel<<<grid_for(total), 256, 0, st>>>(bits, H, W, Cw, C, flip, out_bits, static_cast<uint8_t *>(out_form),
-                                                          out_form_kind, total);
+    QNN_CUDA(launch_pdl(maxpool2x2_bits_kernel, dim3(grid_for(total)), dim3(256), 0, st, bits, H, W, Cw, C, flip, out_bits,
+                        static_cast<uint8_t *>(out_form), out_form_kind, total));
     return check_launch("qnn_maxpool2x2_bits");
 }
 

@@ -227,6 +227,8 @@ __global__ void __launch_bounds__(256) gemm_popc_skinny_kernel(const uint32_t *_
 {
     extern __shared__ __align__(16) uint32_t bs[];               // [N][kw4], kw4 = kwords rounded up to 4, zero padded
     const int kw4 = (int)((kwords + 3) & ~(int64_t)3);
+    griddep_launch_dependents();
+    griddep_wait();                                              // (the weights could be read before this; the activations not)
     for (int e = threadIdx.x; e < N * kw4; e += blockDim.x) {
         const int n = e / kw4, k = e - n * kw4;
         bs[e] = k < kwords ? __ldg(b + (int64_t)n * ldb + k) : 0u;
@@ -305,7 +307,7 @@ int launch_skinny(const PopcParams &P, cudaStream_t st)
     const int64_t cap = (int64_t)sm_count() * 4;
     const int blocks = (int)(need < cap ? need : cap);
     profile_before(st);
-    kern<<<blocks, 256, smem, st>>>(g.a, g.lda, g.b, g.ldb, g.M, (int)g.N, P.kwords, P.kll, g.out, g.ldo);
+    QNN_CUDA(launch_pdl(kern, dim3(blocks), dim3(256), smem, st, g.a, g.lda, g.b, g.ldb, g.M, (int)g.N, P.kwords, P.kll, g.out, g.ldo));
     profile_after(st);
     return check_launch("popc gemm (few units)");
 }

@@ -389,12 +389,6 @@ __device__ __forceinline__ uint32_t tma_stage_conv(uint32_t next_empty_bar, uint
     return ready;
 }
 
-// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start while the kernel
-// before it is still draining; it must not touch that kernel's results (or buffers that kernel still reads) before
-// griddep_wait() returns, which is when every earlier kernel has completed and its writes are visible.
-__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -926,6 +920,8 @@ __global__ void __launch_bounds__(256) expand_i8_kernel(const uint32_t *__restri
                                                         int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
                                                         int64_t period64, int tail, uint8_t *__restrict__ out, int64_t out_ld)
 {
+    griddep_launch_dependents();
+    griddep_wait();
     const IDX chunks = (IDX)(kwords * 2);
     const IDX total = (IDX)rows * chunks;
     const IDX period = (IDX)period64;
@@ -966,6 +962,8 @@ __global__ void __launch_bounds__(256) expand_fp4_kernel(const uint32_t *__restr
                                                          int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords64,
                                                          int64_t period64, int tail, uint8_t *__restrict__ out, int64_t out_ld)
 {
+    griddep_launch_dependents();
+    griddep_wait();
     const IDX kwords = (IDX)kwords64;
     const IDX total = (IDX)rows * kwords;
     const IDX period = (IDX)period64;
@@ -1110,7 +1108,7 @@ int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMa
     {
         // programmatic stream serialisation: the grid may be scheduled while the previous kernel drains (the kernel
         // calls griddepcontrol.wait before it touches global memory); QNN_PDL=0 in the environment turns it off
-        static const bool pdl = [] { const char *e = getenv("QNN_PDL"); return !(e && e[0] == '0'); }();
+        const bool pdl = pdl_enabled();
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(CTAS * nw));
         cfg.blockDim = dim3(TC_THREADS);
@@ -1227,14 +1225,18 @@ int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t pla
     const int pm1 = mode == QNN_MODE_PM1;
     if (form == QNN_FORM_FP4) {
         if (narrow)
-            expand_fp4_kernel<uint32_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
+            QNN_CUDA(launch_pdl(expand_fp4_kernel<uint32_t>, dim3(grid), dim3(256), 0, st, src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst,
+                                dst_ld));
         else
-            expand_fp4_kernel<int64_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
+            QNN_CUDA(launch_pdl(expand_fp4_kernel<int64_t>, dim3(grid), dim3(256), 0, st, src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst,
+                                dst_ld));
     } else {
         if (narrow)
-            expand_i8_kernel<uint32_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
+            QNN_CUDA(launch_pdl(expand_i8_kernel<uint32_t>, dim3(grid), dim3(256), 0, st, src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst,
+                                dst_ld));
         else
-            expand_i8_kernel<int64_t><<<grid, 256, 0, st>>>(src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst, dst_ld);
+            QNN_CUDA(launch_pdl(expand_i8_kernel<int64_t>, dim3(grid), dim3(256), 0, st, src, planes, pm1, ld, plane_stride, rows, kwords, pad_period, pad_tail, dst,
+                                dst_ld));
     }
     return check_launch("tc expand");
 }

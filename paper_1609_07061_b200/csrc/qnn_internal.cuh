@@ -111,6 +111,28 @@ int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t pla
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st);
 
 #ifdef __CUDACC__
+// Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the kernel before it in the
+// stream is still draining; it must not touch that kernel's results (or buffers that kernel still reads) before
+// griddep_wait() returns, which is when every earlier kernel has completed and its writes are visible.
+// griddep_launch_dependents() lets the kernel after this one be scheduled early in the same way.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// QNN_PDL=0 in the environment launches everything with plain stream ordering.
+bool pdl_enabled();
+
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // bit i of the low byte of x -> bit 4*i (one bit per nibble)
 __device__ __forceinline__ uint32_t spread_bits_to_nibbles(uint32_t x)
 {

@@ -27,6 +27,8 @@ inline bool is_tc(int algo) { return algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_
 __global__ void __launch_bounds__(256) repitch_rows_kernel(const uint4 *__restrict__ src, int64_t rows, int64_t k16,
                                                            uint4 *__restrict__ dst, int64_t pitch16)
 {
+    griddep_launch_dependents();
+    griddep_wait();
     const int64_t total = rows * k16;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
         const int64_t r = e / k16, c = e - r * k16;
@@ -142,8 +144,8 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
                     const int64_t pitch = p.kw0 * 32;
                     const int64_t total = M * (ly.K / 16);
                     const int64_t need = ceil_div(total, 256), cap = (int64_t)sm_count() * 16;
-                    repitch_rows_kernel<<<(int)(need < cap ? need : cap), 256, 0, st>>>(
-                        reinterpret_cast<const uint4 *>(x_dev), M, ly.K / 16, reinterpret_cast<uint4 *>(planes), pitch / 16);
+                    QNN_CUDA(launch_pdl(repitch_rows_kernel, dim3((unsigned)(need < cap ? need : cap)), dim3(256), 0, st,
+                                        reinterpret_cast<const uint4 *>(x_dev), M, ly.K / 16, reinterpret_cast<uint4 *>(planes), pitch / 16));
                     if (int rc = check_launch("mlp input re-spacing")) return rc;
                     g.a_tc = planes; g.a_tc_ld = pitch;
                 }
