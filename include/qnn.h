@@ -55,7 +55,7 @@
 extern "C" {
 #endif
 
-#define QNN_VERSION 220
+#define QNN_VERSION 230
 
 /* status codes */
 #define QNN_OK 0
@@ -345,7 +345,16 @@ typedef struct qnn_conv_io {
     void *out_form;       /* the same signs as NHWC values in out_form_kind (dense), the
                              next convolution's x, or NULL                               */
     int out_form_kind;
+    int pool2x2;          /* 1: 2 x 2 max-pooling between the convolution and the threshold
+                             (Table 7), done inside the call on the thresholded signs:
+                             out_bits / out_form are then [B, H/2, W/2, ...]; needs
+                             qnn_conv_can_pool(H, W) and out_nchw == NULL                */
 } qnn_conv_io;
+
+/* 1 when qnn_binary_conv2d_prepared can pool inside the call: W in {2,4,8,16} and H even
+ * (a window's four pixels then sit in one warp of the epilogue); other sizes pool with
+ * qnn_maxpool2x2_bits. */
+QNN_API int qnn_conv_can_pool(int H, int W);
 
 /* Section 5 with a prepared filter bank: same result as qnn_binary_conv2d
  * (stride 1, the pad and pad_bit given to qnn_conv_prepare).  A workspace of

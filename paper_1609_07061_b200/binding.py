@@ -55,7 +55,7 @@ class qnn_tc_output(ctypes.Structure):
 
 class qnn_conv_io(ctypes.Structure):
     _fields_ = [("x", vp), ("x_form", i32), ("out_nchw", vp), ("thr", vp), ("flip", vp), ("out_bits", vp),
-                ("out_form", vp), ("out_form_kind", i32)]
+                ("out_form", vp), ("out_form_kind", i32), ("pool2x2", i32)]
 
 
 class qnn_mlp_layer(ctypes.Structure):
@@ -96,6 +96,7 @@ _SIGS = {
     "qnn_rescale_f32": (i32, [vp, i64, i64, i64, f32, vp, vp, f32, vp, i64, vp]),
     "qnn_binary_conv2d": (i32, [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32, vp, sz, vp]),
     "qnn_conv_form": (i32, [i32]),
+    "qnn_conv_can_pool": (i32, [i32, i32]),
     "qnn_conv_prepared_bytes": (sz, [i32, i32, i32, i32, i32]),
     "qnn_conv_prepare": (i32, [vp, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
     "qnn_binary_conv2d_prepared": (i32, [ctypes.POINTER(qnn_conv_io), i32, i32, i32, i32, vp, i32, i32, i32, i32, vp, sz, vp]),
@@ -281,8 +282,8 @@ def qnn_conv_prepare(w, Cout, C, KH, KW, pad, pad_bit, prepared):
 
 
 def qnn_binary_conv2d_prepared(x, x_form, B, C, H, W, prepared, Cout, KH, KW, pad, out_nchw=None, thr=None, flip=None,
-                               out_bits=None, out_form=None, out_form_kind=0, ws=None):
-    io = qnn_conv_io(_p(x), x_form, _p(out_nchw), _p(thr), _p(flip), _p(out_bits), _p(out_form), out_form_kind)
+                               out_bits=None, out_form=None, out_form_kind=0, ws=None, pool2x2=0):
+    io = qnn_conv_io(_p(x), x_form, _p(out_nchw), _p(thr), _p(flip), _p(out_bits), _p(out_form), out_form_kind, pool2x2)
     wp, wb = _ws(ws)
     _ck(_lib.qnn_binary_conv2d_prepared(ctypes.byref(io), B, C, H, W, _p(prepared), Cout, KH, KW, pad, wp, wb, _stream()),
         "qnn_binary_conv2d_prepared")
@@ -342,6 +343,10 @@ def qnn_mlp_forward_host(x_host, M, in_bits, layers, scores_host, algo=QNN_ALGO_
 
 def qnn_logquant_pack_i8(x, rows, K, ldx, emin, emax, out, ld_bytes):
     _ck(_lib.qnn_logquant_pack_i8(_p(x), rows, K, ldx, emin, emax, _p(out), ld_bytes, _stream()), "qnn_logquant_pack_i8")
+
+
+def qnn_conv_can_pool(H, W) -> bool:
+    return bool(_lib.qnn_conv_can_pool(H, W))
 
 
 def qnn_conv2d_u8_workspace_bytes(B, C, H, W, Cout, KH, KW, pad) -> int:

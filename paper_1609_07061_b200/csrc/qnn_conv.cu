@@ -264,6 +264,11 @@ int qnn_conv_prepare(const uint32_t *w, int Cout, int C, int KH, int KW, int pad
     return conv_prepare_into(w, Cout, C, KH, KW, pad, pad_bit, l, wf, reinterpret_cast<int32_t *>(wf + l.w_bytes), as_stream(stream));
 }
 
+int qnn_conv_can_pool(int H, int W)
+{
+    return (W == 2 || W == 4 || W == 8 || W == 16) && H >= 2 && H % 2 == 0;
+}
+
 int qnn_conv_form(int C)
 {
     return C > 0 && C % 128 == 0 ? QNN_FORM_FP4 : 0;
@@ -283,6 +288,9 @@ int qnn_binary_conv2d_prepared(const qnn_conv_io *io, int B, int C, int H, int W
                 "qnn_binary_conv2d_prepared: input form %d, but this filter bank multiplies in form %d", io->x_form, l.form);
     QNN_REQUIRE(io->out_nchw || io->out_bits || io->out_form, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: no output buffer");
     QNN_REQUIRE(!(io->out_bits || io->out_form) || io->thr, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d_prepared: thresholds required");
+    QNN_REQUIRE(!io->pool2x2 || (qnn_conv_can_pool(H, W) && io->out_nchw == nullptr), QNN_ERR_UNSUPPORTED,
+                "qnn_binary_conv2d_prepared: pooling in the same call needs W in {2,4,8,16}, an even H and no int32 output; "
+                "use qnn_maxpool2x2_bits");
     cudaStream_t st = as_stream(stream);
     const int64_t Cw = ceil_div(C, 32);
     const int64_t M = (int64_t)B * H * W;
@@ -317,6 +325,7 @@ int qnn_binary_conv2d_prepared(const qnn_conv_io *io, int B, int C, int H, int W
     ConvImplicit ci{};
     ci.B = B; ci.H = H; ci.W = W; ci.KH = KH; ci.KW = KW; ci.pad = pad;
     ci.cblocks = (int32_t)(cbytes / l.kblk); ci.kblk = l.kblk;
+    ci.pool = io->pool2x2 ? 1 : 0;
     ci.corr = reinterpret_cast<const int32_t *>(wf + l.w_bytes);
     g.conv = &ci;
     return launch_gemm_tc(g, l.form, nullptr, 0, st);

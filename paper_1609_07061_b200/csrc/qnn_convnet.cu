@@ -2,6 +2,7 @@
 // them on one stream: the first convolution on 8-bit pixel codes (Eq. 8 recomposed: codes x +-1 filters on the
 // int8 tensor-core path), 2 x 2 max-pooling between a convolution and its folded batch-norm threshold, and the
 // fully connected head of Algorithm 4.
+#include <cstdlib>
 #include "qnn_internal.cuh"
 
 namespace qnn {
@@ -503,8 +504,13 @@ int qnn_convnet_forward(const uint8_t *x, int B, int H, int W, const qnn_net_lay
         // a convolution: threshold straight to what the next layer reads, or to bits that the pooling step turns into it
         ConvOut o{};
         o.thr = ly.thr; o.flip = ly.flip;
-        const bool direct_form = want_form != 0 && !ly.pool;
-        if (ly.pool) o.out_bits = pre;
+        // narrow images pool inside the convolution's own epilogue; wider ones through packed bits and the pooling kernel
+        // (QNN_FUSED_POOL=0 in the environment keeps the pooling kernel everywhere)
+        static const bool fuse_ok = [] { const char *e = getenv("QNN_FUSED_POOL"); return !(e && e[0] == '0'); }();
+        const bool fused_pool = fuse_ok && ly.pool && ly.kind == QNN_LAYER_CONV && lp.fast && qnn_conv_can_pool(lp.H, lp.W);
+        const bool separate_pool = ly.pool && !fused_pool;
+        const bool direct_form = want_form != 0 && !separate_pool;
+        if (separate_pool) o.out_bits = pre;
         else if (direct_form) { o.out_form = act_form; o.out_form_kind = want_form; }
         else o.out_bits = act_bits;
 
@@ -517,13 +523,14 @@ int qnn_convnet_forward(const uint8_t *x, int B, int H, int W, const qnn_net_lay
             io.x = cur_form && cur_kind == lp.prep.form ? cur_form : static_cast<const void *>(cur_bits);
             io.x_form = cur_form && cur_kind == lp.prep.form ? cur_kind : 0;
             io.thr = o.thr; io.flip = o.flip; io.out_bits = o.out_bits; io.out_form = o.out_form; io.out_form_kind = o.out_form_kind;
+            io.pool2x2 = fused_pool ? 1 : 0;
             QNN_REQUIRE(io.x != nullptr, QNN_ERR_INVALID_ARG, "convnet: layer %d has no input", i);
             if (int rc = qnn_binary_conv2d_prepared(&io, B, ly.C, lp.H, lp.W, prep + lp.prep_off, ly.Cout, ly.ksize, ly.ksize, ly.pad, gen,
                                                     p.gen_bytes, stream))
                 return rc;
         } else {
             // any other geometry: packed im2col and the matrix product the library picks; it writes bits only
-            uint32_t *dst = ly.pool ? pre : act_bits;
+            uint32_t *dst = separate_pool ? pre : act_bits;
             if (int rc = qnn_binary_conv2d(cur_bits, B, ly.C, lp.H, lp.W, ly.w, ly.Cout, ly.ksize, ly.ksize, 1, ly.pad, 1, nullptr, ly.thr,
                                            ly.flip, dst, QNN_ALGO_AUTO, gen, p.gen_bytes, stream))
                 return rc;
@@ -534,7 +541,7 @@ int qnn_convnet_forward(const uint8_t *x, int B, int H, int W, const qnn_net_lay
                     return rc;
             }
         }
-        if (ly.pool) {
+        if (separate_pool) {
             if (int rc = maxpool_run(pre, B, lp.H, lp.W, ly.Cout, ly.flip, want_form ? nullptr : act_bits, want_form ? act_form : nullptr,
                                      want_form, st))
                 return rc;

@@ -55,6 +55,7 @@ struct TcParams {
     int conv;
     int32_t cH, cW, cR, tiles_per_img, cKW, cpad, cblocks;
     int32_t cG, cB;             // images per tile (> 1 only when a whole image is at most half a tile), images in all
+    int32_t pool;               // conv: 2 x 2 max-pooling of the thresholded signs inside the epilogue
     const int32_t *corr;
     int64_t corr_ld;                 // row length of the correction table: N rounded up to 32, pad zero
 };
@@ -694,6 +695,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int r = q * 32 + lane;
             int64_t m, m_warp0;                                  // this thread's row, and the row of the warp's lane 0
             bool mrow;
+            int64_t m_st = 0;                                    // row and predicate of the sign outputs (differ when pooling)
+            bool st_ok = false;
             int32_t cls = 0, c_img = 0, c_pix0 = 0;
             if (p.conv) {
                 // a tile is cR rows of one image, or cG whole images one after the other
@@ -707,6 +710,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 m = ((int64_t)c_img * p.cH + y) * p.cW + x;
                 c_pix0 = y0 * p.cW + q * 32;
                 m_warp0 = (int64_t)tile_img * p.cG * p.cH * p.cW + c_pix0;
+                if (p.pool) {
+                    // the even-row, even-column pixel of every 2 x 2 window writes the pooled pixel
+                    st_ok = mrow && ((x & 1) == 0) && ((y & 1) == 0);
+                    m_st = ((int64_t)c_img * (p.cH >> 1) + (y >> 1)) * (p.cW >> 1) + (x >> 1);
+                }
                 const int32_t pd = p.cpad, pc = pd + 1;
                 const int32_t ty = max(pd - y, 0), by = max(y + pd - (p.cH - 1), 0);
                 const int32_t tx = max(pd - x, 0), bx = max(x + pd - (p.cW - 1), 0);
@@ -716,6 +724,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 m_warp0 = ((int64_t)tm * CTAS + rank) * BM + q * 32;
                 mrow = m < p.M;
             }
+            if (!p.pool) { m_st = m; st_ok = mrow; }
             const bool any_border = p.conv ? (__any_sync(0xffffffffu, cls != 0) != 0) : false;
             int64_t img = 0, pix = 0;                            // where an int32 NCHW result of this row goes
             if (p.epilogue == EPI_NCHW && mrow && p.out != nullptr) {
@@ -849,7 +858,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     const int64_t left = p.N - n0;
                     const uint32_t nmask = left >= 32 ? 0xffffffffu : ((1u << (int)left) - 1u);
                     w = (w ^ flip_w[lc]) & nmask;
-                    if (want_bits && mrow) p.out_bits[m * p.ld_bits + (n0 >> 5)] = w;
+                    if (p.pool) {
+                        // Max-pooling sits between the convolution and the threshold (Table 7); the threshold is monotone
+                        // in the sum, so the pooled sign is the OR of the window's four signs, the AND where the
+                        // comparison is flipped.  The window's pixels are lanes l, l^1 (next column), l^W, l^W^1 (next row).
+                        const uint32_t f = flip_w[lc];
+                        uint32_t wo = w, wa = w;
+                        wo |= __shfl_xor_sync(0xffffffffu, wo, 1);
+                        wa &= __shfl_xor_sync(0xffffffffu, wa, 1);
+                        wo |= __shfl_xor_sync(0xffffffffu, wo, p.cW);
+                        wa &= __shfl_xor_sync(0xffffffffu, wa, p.cW);
+                        w = ((wo & ~f) | (wa & f)) & nmask;
+                    }
+                    if (want_bits && st_ok) p.out_bits[m_st * p.ld_bits + (n0 >> 5)] = w;
                     if (want_form) {
                         if (form_fp4) {
                             // +1 -> e2m1 0x2, -1 -> 0xA, columns past N -> 0
@@ -861,7 +882,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                                 for (int b = 0; b < 4; ++b) o[b] &= spread_bits_to_nibbles((nmask >> (8 * b)) & 0xffu) * 0xfu;
                             }
                             const uint4 o4 = make_uint4(o[0], o[1], o[2], o[3]);
-                            if (mrow) *reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + (n0 >> 1)) = o4;
+                            if (st_ok) *reinterpret_cast<uint4 *>(p.out_form + m_st * p.ld_form + (n0 >> 1)) = o4;
                         } else {
                             // +1 -> 0x01, -1 -> 0xFF, columns past N -> 0
                             uint32_t o[8];
@@ -871,8 +892,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                                 const uint32_t vm = spread_bits_to_bytes((nmask >> (4 * b)) & 0xfu) * 0xffu;
                                 o[b] = (0xFFFFFFFFu ^ (sb * 0xfeu)) & vm;
                             }
-                            uint4 *dst = reinterpret_cast<uint4 *>(p.out_form + m * p.ld_form + n0);
-                            if (mrow) {
+                            uint4 *dst = reinterpret_cast<uint4 *>(p.out_form + m_st * p.ld_form + n0);
+                            if (st_ok) {
                                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
                             }
@@ -1358,6 +1379,11 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
         const int G = (R == c.H && BM / (c.H * c.W) >= 2) ? BM / (c.H * c.W) : 1;
         p.conv = 1; p.cH = c.H; p.cW = c.W; p.cR = R; p.tiles_per_img = (int32_t)ceil_div(c.H, R);
         p.cG = G; p.cB = c.B;
+        if (c.pool) {
+            QNN_REQUIRE((c.W == 2 || c.W == 4 || c.W == 8 || c.W == 16) && c.H % 2 == 0 && (R % 2 == 0) && g.out == nullptr,
+                        QNN_ERR_UNSUPPORTED, "tc conv: pooling inside the epilogue needs W in {2,4,8,16}, an even H and no int32 output");
+            p.pool = 1;
+        }
         p.cKW = c.KW; p.cpad = c.pad; p.cblocks = c.cblocks; p.corr = c.corr; p.corr_ld = (int64_t)round_up((size_t)g.N, 32);
         QNN_REQUIRE(aligned(c.corr, 16), QNN_ERR_ALIGNMENT, "tc conv: correction table must be 16-byte aligned");
         p.tiles_m = (int32_t)ceil_div(c.B, G) * p.tiles_per_img;

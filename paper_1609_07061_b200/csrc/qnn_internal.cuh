@@ -49,6 +49,7 @@ struct ConvImplicit {
     int32_t B, H, W, KH, KW, pad;
     int32_t cblocks;            // channel blocks per pixel
     int32_t kblk;               // bytes per channel block: 128 (0 means 128), or 64 for 128 e2m1 channels
+    int32_t pool;               // 1: the epilogue max-pools the thresholded signs 2 x 2 (outputs are [B, H/2, W/2, ...])
     const int32_t *corr;        // [(pad+1)^4][N rounded up to 32] border corrections (pad columns and class 0 zero)
 };
 

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(q):
 
 
 def test_version_and_strings(q):
-    assert q.qnn_version() == 220
+    assert q.qnn_version() == 230
     assert q.qnn_status_string(0) == "ok"
     assert "overflow" in q.qnn_status_string(q.QNN_ERR_OVERFLOW)
 

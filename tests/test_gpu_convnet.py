@@ -217,3 +217,52 @@ def test_degenerate_sizes(q):
     assert (scores.t.cpu().numpy() == -7).all() and (out.t.cpu().numpy() == 0x5C).all()
     for g in (scores, ob, out):
         g.check()
+
+
+@pytest.mark.parametrize("B,C,H,W,Co", [(3, 256, 16, 16, 256), (5, 128, 8, 8, 70), (2, 128, 4, 4, 32), (2, 256, 6, 16, 40), (1, 512, 2, 2, 33),
+                                         (9, 256, 8, 8, 64)])
+def test_conv_with_pooling_inside_the_call(q, B, C, H, W, Co):
+    """conv -> 2x2 max-pool -> threshold (Table 7's order) in one call: the epilogue pools the thresholded signs."""
+    rng = np.random.default_rng(B + C + H + W + Co)
+    X = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    Wt = rng.uniform(-1, 1, (Co, C, 3, 3)).astype(np.float32)
+    T = (rng.integers(-24, 25, Co) + int(round((9 * C) ** 0.5))).astype(np.int32)
+    flip = rng.integers(0, 2, Co).astype(np.uint8)
+    s = oracle.conv2d(oracle.sign(X), oracle.sign(Wt), 1, 1, 1)
+    pooled = oracle.maxpool2x2(s)
+    want = oracle.threshold(pooled.transpose(0, 2, 3, 1).reshape(-1, Co), T, flip)
+    assert 0.02 < want.mean() < 0.98                       # both outcomes occur, so the comparison means something
+    cw, cwo = words_per_row(C), words_per_row(Co)
+    xb = torch.zeros(B, H, W, cw, dtype=torch.int32, device="cuda")
+    wb = torch.zeros(Co, 9 * cw, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_sign_nchw(dev(X), B, C, H, W, xb)
+    q.qnn_pack_conv_weights(dev(Wt), Co, C, 3, 3, wb)
+    prep = torch.empty(q.qnn_conv_prepared_bytes(Co, C, 3, 3, 1), dtype=torch.uint8, device="cuda")
+    q.qnn_conv_prepare(wb, Co, C, 3, 3, 1, 1, prep)
+    assert q.qnn_conv_can_pool(H, W)
+    ws = torch.empty(B * H * W * cw * 32 + 256, dtype=torch.uint8, device="cuda")
+    Hp, Wp = H // 2, W // 2
+    for fk, per_word in ((q.QNN_FORM_FP4, 16), (q.QNN_FORM_I8, 32)):
+        bits = Guarded((B, Hp, Wp, cwo), torch.int32, fill=0)
+        of = Guarded((B * Hp * Wp, cwo * per_word), torch.uint8, fill=0x5C)
+        q.qnn_binary_conv2d_prepared(xb, 0, B, C, H, W, prep, Co, 3, 3, 1, thr=dev(T), flip=dev(flip), out_bits=bits.t, out_form=of.t,
+                                     out_form_kind=fk, ws=ws, pool2x2=1)
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        np.testing.assert_array_equal(unpack_words(words_np(bits.t).reshape(-1, cwo), Co), want)
+        np.testing.assert_array_equal(of.t.cpu().numpy(), _form_bytes(want, Co, fk, q))
+        bits.check()
+        of.check()
+
+
+def test_pooling_inside_the_call_is_refused_for_wide_images(q):
+    assert not q.qnn_conv_can_pool(32, 32) and not q.qnn_conv_can_pool(7, 8)
+    xb = torch.zeros(1, 32, 32, 4, dtype=torch.int32, device="cuda")
+    wb = torch.zeros(32, 36, dtype=torch.int32, device="cuda")
+    prep = torch.empty(q.qnn_conv_prepared_bytes(32, 128, 3, 3, 1), dtype=torch.uint8, device="cuda")
+    q.qnn_conv_prepare(wb, 32, 128, 3, 3, 1, 1, prep)
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_binary_conv2d_prepared(xb, 0, 1, 128, 32, 32, prep, 32, 3, 3, 1, thr=torch.zeros(32, dtype=torch.int32, device="cuda"),
+                                     out_bits=torch.zeros(256, dtype=torch.int32, device="cuda"), ws=ws, pool2x2=1)
+    assert e.value.status == q.QNN_ERR_UNSUPPORTED
