@@ -658,16 +658,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 else flip_raw[lc] = 0;
             }
         };
-        if (want_sign && blockIdx.x / CTAS < num_tiles) fetch_thresholds((int64_t)((blockIdx.x / CTAS) / tiles_m) * BN);
+        // Consecutive tiles of a CTA mostly share their column block, so thresholds are fetched and parked only when
+        // the column block changes: tn_fetched is the block whose values the registers hold, tn_parked the one in
+        // shared memory.
+        int32_t tn_fetched = -1, tn_parked = -1;
+        if (want_sign && blockIdx.x / CTAS < num_tiles) {
+            tn_fetched = (int32_t)((blockIdx.x / CTAS) / tiles_m);
+            fetch_thresholds((int64_t)tn_fetched * BN);
+        }
         for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS, ++iter) {
             const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
             const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
             const int64_t ntile = (int64_t)tn * BN;
 
-            // Thresholds and flip bytes of this tile were fetched into registers one tile ago (or just before
-            // the loop): park them in this warp's shared rows, then start fetching the next tile's, so that
+            // Thresholds and flip bytes of this tile's column block were fetched into registers a tile ago (or just
+            // before the loop): park them in this warp's shared rows, then start fetching the next block's, so that
             // their global-memory latency never sits between two tiles.
-            if (want_sign) {
+            if (want_sign && tn != tn_parked) {                  // (warp-uniform)
+                tn_parked = tn;
                 __syncwarp();
 #pragma unroll
                 for (int lc = 0; lc < CPW; ++lc) {
@@ -687,8 +695,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     if (lane == lc) flip_w[lc] = fw;
                 }
                 __syncwarp();
+            }
+            if (want_sign) {
                 const uint32_t tnext = t + gridDim.x / CTAS;
-                if (tnext < num_tiles) fetch_thresholds((int64_t)(tnext / tiles_m) * BN);
+                if (tnext < num_tiles) {
+                    const int32_t tn_next = (int32_t)(tnext / tiles_m);
+                    if (tn_next != tn_fetched) { tn_fetched = tn_next; fetch_thresholds((int64_t)tn_next * BN); }
+                }
             }
 
             // which output row this thread owns
