@@ -662,6 +662,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // the column block changes: tn_fetched is the block whose values the registers hold, tn_parked the one in
         // shared memory.
         int32_t tn_fetched = -1, tn_parked = -1;
+        // convolution: where this thread's row sits inside a tile never changes (image of the tile, row, column)
+        int32_t r_gi = 0, r_y = 0, r_x = 0;
+        if (p.conv) {
+            const int32_t r = q * 32 + lane;
+            r_gi = r / (p.cR * p.cW);
+            const int32_t rem = r - r_gi * (p.cR * p.cW);
+            r_y = rem / p.cW;
+            r_x = rem - r_y * p.cW;
+        }
         if (want_sign && blockIdx.x / CTAS < num_tiles) {
             tn_fetched = (int32_t)((blockIdx.x / CTAS) / tiles_m);
             fetch_thresholds((int64_t)tn_fetched * BN);
@@ -715,9 +724,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 // a tile is cR rows of one image, or cG whole images one after the other
                 const int32_t tile_img = tm / p.tiles_per_img;
                 const int32_t y0 = (tm - tile_img * p.tiles_per_img) * p.cR;
-                const int32_t gi = r / (p.cR * p.cW), rem = r - gi * (p.cR * p.cW);
-                const int32_t y = y0 + rem / p.cW;
-                const int32_t x = rem % p.cW;
+                const int32_t gi = r_gi;
+                const int32_t y = y0 + r_y;
+                const int32_t x = r_x;
                 c_img = tile_img * p.cG + gi;
                 mrow = (gi < p.cG) && (y < p.cH) && (c_img < p.cB);
                 m = ((int64_t)c_img * p.cH + y) * p.cW + x;
