@@ -1,0 +1,87 @@
+"""Times single library calls on seeded paper-shaped inputs (device time, L2 flushed before every timed call).
+
+    python -m paper_1609_07061_b200.microbench pack_sign 8192          # fp32 [n, n] -> packed bits, row-major
+    python -m paper_1609_07061_b200.microbench pack_sign_t 8192        # the transposed (weight) packer
+    python -m paper_1609_07061_b200.microbench threshold_pack 10000 4096
+    python -m paper_1609_07061_b200.microbench conv_c4                 # 128 x 256 x 16 x 16, 3x3, prepared bank, form in / form out
+    python -m paper_1609_07061_b200.microbench conv_c4 pool            # the same with 2x2 pooling inside the call
+
+Prints one JSON line.  Small enough to put under a profiler: one warm-up call and `--reps` timed ones.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+
+import torch
+
+from . import binding as q
+from . import workloads
+
+
+def _time(fn, reps):
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    fn()
+    ts = []
+    for _ in range(reps):
+        flush.fill_(1)
+        flush.sum()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b))
+    return statistics.median(ts)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("op", choices=["pack_sign", "pack_sign_t", "threshold_pack", "conv_c4"])
+    ap.add_argument("args", nargs="*")
+    ap.add_argument("--reps", type=int, default=5)
+    a = ap.parse_args()
+    rec = {"op": a.op}
+    if a.op in ("pack_sign", "pack_sign_t"):
+        n = int(a.args[0]) if a.args else 8192
+        g = torch.Generator(device="cuda").manual_seed(0)
+        x = torch.randn(n, n, device="cuda", generator=g)
+        out = torch.zeros(n, n // 32, dtype=torch.int32, device="cuda")
+        if a.op == "pack_sign":
+            ms = _time(lambda: q.qnn_quantize_pack_sign(x, n, n, n, out, n // 32), a.reps)
+        else:
+            ms = _time(lambda: q.qnn_quantize_pack_sign_t(x, n, n, n, out, n // 32), a.reps)
+        rec.update(shape=[n, n], ms=ms, GBps=n * n * 4.125 / ms / 1e6)
+    elif a.op == "threshold_pack":
+        M = int(a.args[0]) if a.args else 10000
+        N = int(a.args[1]) if len(a.args) > 1 else 4096
+        g = torch.Generator(device="cuda").manual_seed(0)
+        s = torch.randint(-100, 100, (M, N), dtype=torch.int32, device="cuda", generator=g)
+        thr = torch.randint(-64, 65, (N,), dtype=torch.int32, device="cuda", generator=g)
+        out = torch.zeros(M, N // 32, dtype=torch.int32, device="cuda")
+        ms = _time(lambda: q.qnn_threshold_pack(s, M, N, N, thr, None, out, N // 32), a.reps)
+        rec.update(shape=[M, N], ms=ms, GBps=M * N * 4.125 / ms / 1e6)
+    else:
+        pool = 1 if (a.args and a.args[0] == "pool") else 0
+        wl = workloads.cifar_conv()
+        B, C, H, W = wl.X.shape
+        Co = wl.W.shape[0]
+        xb = torch.zeros(B, H, W, C // 32, dtype=torch.int32, device="cuda")
+        wb = torch.zeros(Co, 9 * C // 32, dtype=torch.int32, device="cuda")
+        q.qnn_quantize_pack_sign_nchw(wl.X.cuda(), B, C, H, W, xb)
+        q.qnn_pack_conv_weights(wl.W.cuda(), Co, C, 3, 3, wb)
+        prep = torch.empty(q.qnn_conv_prepared_bytes(Co, C, 3, 3, 1), dtype=torch.uint8, device="cuda")
+        q.qnn_conv_prepare(wb, Co, C, 3, 3, 1, 1, prep)
+        form = q.qnn_conv_form(C)
+        xf = torch.empty(B * H * W, q.qnn_tc_row_bytes(C, form), dtype=torch.uint8, device="cuda")
+        q.qnn_tc_prepack(xb, 1, q.QNN_MODE_PM1, C // 32, 0, B * H * W, C, form, xf, xf.shape[1])
+        rows = B * (H // 2) * (W // 2) if pool else B * H * W
+        of = torch.empty(rows, q.qnn_tc_row_bytes(Co, form), dtype=torch.uint8, device="cuda")
+        thr = wl.T.cuda()
+        ms = _time(lambda: q.qnn_binary_conv2d_prepared(xf, form, B, C, H, W, prep, Co, 3, 3, 1, thr=thr, out_form=of, out_form_kind=form,
+                                                        pool2x2=pool), a.reps)
+        rec.update(shape=[B, C, H, W, Co], pool=pool, ms=ms, binary_Tops=2.0 * B * H * W * Co * 9 * C / ms / 1e9)
+    print(json.dumps(rec))
+
+
+if __name__ == "__main__":
+    main()
