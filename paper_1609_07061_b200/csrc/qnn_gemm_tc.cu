@@ -1447,7 +1447,12 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
         }
     }
 
-    const int bn = pick_bn(p.tiles_m, g.N, sm_count(), 32);
+    // (int8 has no scale columns in tensor memory, so two 256-column accumulator stages fit: tried for wide single-CTA products)
+    int bn = pick_bn(p.tiles_m, g.N, sm_count(), 32);
+    if (form == QNN_FORM_I8 && !g.conv && kblk == BKB && bn == 224) {
+        const int64_t w224 = ceil_div(p.tiles_m * ceil_div(g.N, 224), sm_count()), w256 = ceil_div(p.tiles_m * ceil_div(g.N, 256), sm_count());
+        if (w256 * (256 + 900) < w224 * (224 + 900)) bn = 256;
+    }
     if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn, kblk)) return rc;
     if (kblk == 64) {
         switch (bn) {
@@ -1468,6 +1473,7 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
         }
     }
     switch (bn) {
+        case 256: return launch_tc_cfg<QNN_FORM_I8, 256, 1>(ma, mb, p, sm_count(), st);
         case 224: return launch_tc_cfg<QNN_FORM_I8, 224, 1>(ma, mb, p, sm_count(), st);
         case 192: return launch_tc_cfg<QNN_FORM_I8, 192, 1>(ma, mb, p, sm_count(), st);
         case 128: return launch_tc_cfg<QNN_FORM_I8, 128, 1>(ma, mb, p, sm_count(), st);
