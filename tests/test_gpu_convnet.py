@@ -266,3 +266,32 @@ def test_pooling_inside_the_call_is_refused_for_wide_images(q):
         q.qnn_binary_conv2d_prepared(xb, 0, 1, 128, 32, 32, prep, 32, 3, 3, 1, thr=torch.zeros(32, dtype=torch.int32, device="cuda"),
                                      out_bits=torch.zeros(256, dtype=torch.int32, device="cuda"), ws=ws, pool2x2=1)
     assert e.value.status == q.QNN_ERR_UNSUPPORTED
+
+
+def test_back_to_back_passes_do_not_interfere(q):
+    """Kernels of consecutive passes overlap their starts with the previous kernel's tail (programmatic stream
+    serialisation) and share one workspace: many passes queued without synchronisation, on alternating inputs, must each
+    give the result of a lone pass."""
+    B = 32
+    wl = workloads.cifar_convnet(B=B, H=16, W=16, widths=(128, 128, 256, 256), fc=(256, 10), seed=5, thr=24)
+    net = q.ConvNet(3, 16, 16, wl.conv_W, wl.conv_pool, wl.fc_W, wl.Ts, wl.flips)
+    ws = net.workspace(B)
+    xs = [wl.X.cuda(), workloads.cifar_convnet(B=B, H=16, W=16, widths=(128, 128, 256, 256), fc=(256, 10), seed=5, thr=24,
+                                               stream=1).X.cuda()]
+    ref = []
+    for x in xs:
+        s = torch.zeros(B, 10, dtype=torch.int32, device="cuda")
+        net.forward(x, s, ws)
+        torch.cuda.synchronize()
+        ref.append(s.clone())
+    np.testing.assert_array_equal(ref[0].cpu().numpy(), oracle.convnet_forward(wl.X.numpy().astype(np.int32), _oracle_layers(wl)))
+    assert not torch.equal(ref[0], ref[1])
+    outs = [torch.zeros(B, 10, dtype=torch.int32, device="cuda") for _ in range(48)]
+    for _ in range(3):
+        for i, o in enumerate(outs):
+            net.forward(xs[i & 1], o, ws)
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        for i, o in enumerate(outs):
+            assert torch.equal(o, ref[i & 1]), f"pass {i} differs"
+            o.zero_()
