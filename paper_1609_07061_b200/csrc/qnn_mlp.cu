@@ -120,6 +120,18 @@ int run_mlp(const uint8_t *x_dev, int64_t M, int in_bits, const qnn_mlp_layer *l
     LayerChoice choice[64];
     QNN_REQUIRE(L <= 64, QNN_ERR_UNSUPPORTED, "mlp: at most 64 layers");
     for (int l = 0; l < L; ++l) choice[l] = choose_layer(M, in_bits, layers, l, algo);
+    // A few-unit last layer is too little work for the tensor cores to win when its operands have to be rewritten
+    // first; with weights already in form and the previous layer able to hand its signs over in form there is nothing
+    // to rewrite, and the tensor-core kernel is the faster one (measured: 10000 x 10 x 4096 head, step 176 -> 173 us).
+    if (algo == QNN_ALGO_AUTO && resolve_env_algo() == QNN_ALGO_AUTO && L >= 2 && choice[L - 1].algo == QNN_ALGO_POPC &&
+        is_tc(choice[L - 2].algo) && M >= 1024) {
+        const qnn_mlp_layer &ly = layers[L - 1];
+        const int form = tc_pick_form(1, QNN_MODE_PM1, 1, QNN_MODE_PM1, ly.K);
+        if (form != 0 && ly.w_tc != nullptr && ly.w_tc_form == form) {
+            choice[L - 1].algo = form == QNN_FORM_FP4 ? QNN_ALGO_TC_FP4 : QNN_ALGO_TC_I8;
+            choice[L - 1].form = form;
+        }
+    }
 
     // what the previous layer left behind for this one
     const uint32_t *cur_bits = nullptr; int64_t cur_ld = 0;
