@@ -194,7 +194,7 @@ class MlpBench:
     def step_forward(self, ev=None):
         """qnn_mlp_forward with prepacked weights: the uint8 input is the int8-form operand of layer 1 (Eq. 8
         recomposed), hidden activations travel as e2m1 values written by the previous product's threshold
-        epilogue, the last hidden layer emits packed bits for the 10-unit xor/popc head."""
+        epilogue, down to the 10-unit head, which runs on the tensor cores too since its weights are prepacked."""
         q = self.q
         if ev is not None:
             q.qnn_set_kernel_events_nth(ev[0], ev[1], 1)  # second product kernel = hidden layer 2 (10000 x 4096 x 4096)
