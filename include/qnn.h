@@ -323,8 +323,9 @@ QNN_API int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, con
 /* Filter banks prepared once (static weights) for the tensor-core convolution.
  * Applies to stride-1 "same" filters (KH = KW = 2 * pad + 1, at most 7 x 7) with
  * C a multiple of 128 and images at most 128 pixels wide; qnn_conv_form(C) is the
- * form such a layer multiplies in (QNN_FORM_FP4 for C % 256 == 0, else
- * QNN_FORM_I8; 0 = not available: use qnn_binary_conv2d).
+ * form such a layer multiplies in (QNN_FORM_FP4: a pixel is 128-byte channel
+ * blocks when C % 256 == 0, else 64-byte ones; 0 = not available: use
+ * qnn_binary_conv2d).
  * qnn_conv_prepare rewrites w (qnn_pack_conv_weights layout) in that form and
  * appends the table of what the padding value contributes per border position;
  * `prepared` is a 256-byte aligned device buffer of qnn_conv_prepared_bytes. */
