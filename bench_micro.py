@@ -1,10 +1,10 @@
 """Times single library calls on seeded paper-shaped inputs (device time, L2 flushed before every timed call).
 
-    python -m paper_1609_07061_b200.microbench pack_sign 8192          # fp32 [n, n] -> packed bits, row-major
-    python -m paper_1609_07061_b200.microbench pack_sign_t 8192        # the transposed (weight) packer
-    python -m paper_1609_07061_b200.microbench threshold_pack 10000 4096
-    python -m paper_1609_07061_b200.microbench conv_c4                 # 128 x 256 x 16 x 16, 3x3, prepared bank, form in / form out
-    python -m paper_1609_07061_b200.microbench conv_c4 pool            # the same with 2x2 pooling inside the call
+    python bench_micro.py pack_sign 8192          # fp32 [n, n] -> packed bits, row-major
+    python bench_micro.py pack_sign_t 8192        # the transposed (weight) packer
+    python bench_micro.py threshold_pack 10000 4096
+    python bench_micro.py conv_c4                 # 128 x 256 x 16 x 16, 3x3, prepared bank, form in / form out
+    python bench_micro.py conv_c4 pool            # the same with 2x2 pooling inside the call
 
 Prints one JSON line.  Small enough to put under a profiler: one warm-up call and `--reps` timed ones.
 """
@@ -14,10 +14,17 @@ import argparse
 import json
 import statistics
 
+import os
+import sys
+
 import torch
 
-from . import binding as q
-from . import workloads
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1609_07061_b200 import binding as q          # noqa: E402
+from paper_1609_07061_b200 import workloads             # noqa: E402
 
 
 def _time(fn, reps):

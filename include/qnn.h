@@ -12,8 +12,14 @@
  * Conventions (all entry points):
  *  - Every function returns an int status (QNN_OK = 0 or a QNN_ERR_* code),
  *    never throws, aborts or traps.  qnn_last_error() returns a thread-local
- *    text for the last failure.  Arguments are validated on the host BEFORE
- *    anything is launched: a call that returns an error launched nothing.
+ *    text for the last failure.  Arguments (pointers, sizes, alignment,
+ *    workspace) are validated on the host BEFORE anything is launched: a call
+ *    that returns an argument error launched nothing.  QNN_ERR_CUDA is the one
+ *    exception: a runtime or driver call that fails part-way through a call
+ *    made of several kernels may leave the earlier ones queued.
+ *    When QNN_ALGO_AUTO has to leave its preferred algorithm (no workspace, a
+ *    misaligned one), the call still returns QNN_OK and qnn_last_error() holds
+ *    a note saying which algorithm ran instead and why.
  *  - Unless a parameter says "host", every data pointer is a DEVICE pointer
  *    owned by the caller; the library keeps no reference after the call.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
@@ -145,6 +151,13 @@ QNN_API int qnn_pack_planes_u8(const uint8_t *x, int64_t rows, int64_t K, int64_
  * reduction ordered (kh, kw, channel word) to match the packed im2col rows. */
 QNN_API int qnn_pack_conv_weights(const float *w, int Cout, int C, int KH, int KW, uint32_t *out, void *stream);
 
+/* Table 7, the first fully-connected layer after the last convolution: its
+ * inputs are the H x W x C feature map in (h, w, c) order, i.e. the packed NHWC
+ * bits of that map read as one row in which every pixel is padded to whole
+ * words.  w fp32 [H*W*C, N] row-major (input index (h*W + w)*C + c) is
+ * binarised with Eq. 1 and laid out as out[N, H*W*ceil(C/32)] words to match. */
+QNN_API int qnn_pack_fc_after_conv_weights(const float *w, int N, int C, int H, int W, uint32_t *out, void *stream);
+
 /* ------------------------------------------------------------------------- */
 /* Matrix products                                                            */
 /* ------------------------------------------------------------------------- */
@@ -270,7 +283,10 @@ QNN_API int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_
  * array, which keeps the previous call's contents: the call rewrites every
  * byte it later reads, so no clearing is needed, but two calls that overlap on
  * the GPU (different streams, or several host threads) race on it -- keep
- * calls to this entry point on one stream or serialise them yourself. */
+ * calls to this entry point on one stream or serialise them yourself.
+ * K = 0 gives all zeros like qnn_xnor_gemm.  The looked-up address is kept for
+ * the life of the process and does not survive cudaDeviceReset: do not call
+ * this entry point on a device after resetting it. */
 QNN_API int qnn_xnor_gemm_noalloc(const uint32_t *a, int64_t lda, const uint32_t *b, int64_t ldb, int64_t M,
                                   int64_t N, int64_t K, int32_t *out, int64_t ldo, void *stream);
 
@@ -523,6 +539,15 @@ QNN_API int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int
  * This call synchronises `stream`, reads and clears that word and returns
  * QNN_OK or QNN_ERR_TIMEOUT. */
 QNN_API int qnn_device_status(void *stream);
+
+/* Diagnostic (the paper has no counterpart): launches one tiny kernel whose
+ * only action is a bounded wait, with a limit of a few thousand polls, on a
+ * barrier that nothing arrives on -- no copy and no tensor-core work is in
+ * flight.  The wait runs out through the same code the product kernels use,
+ * so the next qnn_device_status() returns QNN_ERR_TIMEOUT once and QNN_OK
+ * after that, and the context stays fully usable.  For checking the failure
+ * path of an installation; never needed in normal operation. */
+QNN_API int qnn_selftest_wait_timeout(void *stream);
 
 /* Measurement aid: arms two cudaEvent_t handles (passed as void*) on the calling
  * thread.  The next matrix-product call made by this thread records `start`

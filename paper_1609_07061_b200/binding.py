@@ -79,6 +79,7 @@ _SIGS = {
     "qnn_quantize_pack_kbit_t": (i32, [vp, i64, i64, i64, i32, f32, f32, vp, i64, i64, vp, vp]),
     "qnn_pack_planes_u8": (i32, [vp, i64, i64, i64, i32, vp, i64, i64, vp, vp]),
     "qnn_pack_conv_weights": (i32, [vp, i32, i32, i32, i32, vp, vp]),
+    "qnn_pack_fc_after_conv_weights": (i32, [vp, i32, i32, i32, i32, vp, vp]),
     "qnn_xnor_gemm": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
     "qnn_xnor_gemm_noalloc": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, i64, vp]),
     "qnn_xnor_gemm_threshold": (i32, [vp, i64, vp, i64, i64, i64, i64, vp, vp, vp, i64, i32, vp, sz, vp]),
@@ -115,6 +116,7 @@ _SIGS = {
     "qnn_workspace_bytes": (sz, [i32, i64, i64, i64, i32, i32, i32]),
     "qnn_select_algo": (i32, [i64, i64, i64, i32, i32, i32, i32]),
     "qnn_device_status": (i32, [vp]),
+    "qnn_selftest_wait_timeout": (i32, [vp]),
     "qnn_launch_count": (ctypes.c_uint64, []),
     "qnn_set_kernel_events": (i32, [vp, vp]),
     "qnn_set_kernel_events_nth": (i32, [vp, vp, i32]),
@@ -188,6 +190,10 @@ def qnn_pack_planes_u8(x, rows, K, ldx, bits, planes, ld_words, plane_stride_wor
 
 def qnn_pack_conv_weights(w, Cout, C, KH, KW, out):
     _ck(_lib.qnn_pack_conv_weights(_p(w), Cout, C, KH, KW, _p(out), _stream()), "qnn_pack_conv_weights")
+
+
+def qnn_pack_fc_after_conv_weights(w, N, C, H, W, out):
+    _ck(_lib.qnn_pack_fc_after_conv_weights(_p(w), N, C, H, W, _p(out), _stream()), "qnn_pack_fc_after_conv_weights")
 
 
 def qnn_xnor_gemm(a, lda, b, ldb, M, N, K, out, ldo, algo=QNN_ALGO_AUTO, ws=None):
@@ -405,10 +411,9 @@ class ConvNet:
             K, N = Wf.shape
             last = j == len(fc_W) - 1
             if first and len(conv_W) > 0:
-                # inputs in (h, w, c) order, every pixel padded to whole words: the packed layout of an h x w filter
-                w4 = Wf.reshape(h, w, c, N).permute(3, 2, 0, 1).contiguous().cuda()
+                # inputs in (h, w, c) order, every pixel padded to whole words
                 wb = torch.zeros(N, h * w * ((c + 31) // 32), dtype=torch.int32, device="cuda")
-                qnn_pack_conv_weights(w4, N, c, h, w, wb)
+                qnn_pack_fc_after_conv_weights(Wf.cuda().contiguous(), N, c, h, w, wb)
             else:
                 ld = (K + 31) // 32
                 wb = torch.zeros(N, ld, dtype=torch.int32, device="cuda")
@@ -465,6 +470,11 @@ def qnn_select_algo(M, N, K, ka=1, kb=1, a_mode=QNN_MODE_PM1, b_mode=QNN_MODE_PM
 
 def qnn_device_status() -> int:
     return int(_lib.qnn_device_status(_stream()))
+
+
+def qnn_selftest_wait_timeout():
+    """Launches the diagnostic kernel whose bounded wait runs out; the next qnn_device_status() reports it once."""
+    _ck(_lib.qnn_selftest_wait_timeout(_stream()), "qnn_selftest_wait_timeout")
 
 
 def qnn_launch_count() -> int:

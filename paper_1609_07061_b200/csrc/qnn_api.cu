@@ -24,6 +24,14 @@ int fail(int code, const char *fmt, ...)
 
 void clear_error() { g_err[0] = 0; }
 
+void note(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
 bool pdl_enabled()
 {
     static const bool on = [] { const char *e = getenv("QNN_PDL"); return !(e && e[0] == '0'); }();

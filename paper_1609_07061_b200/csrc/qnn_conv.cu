@@ -54,6 +54,26 @@ __global__ void __launch_bounds__(256) conv_weight_pack_kernel(const float *__re
     }
 }
 
+// First fully-connected layer after a convolution: w is [H*W*C, N] row-major with its inputs in (h, w, c) order.
+// One thread per output word out[n, pix*Cw + cw]; consecutive threads take consecutive n (coalesced reads).
+__global__ void __launch_bounds__(256) fc_after_conv_pack_kernel(const float *__restrict__ w, int N, int C, int HW,
+                                                                 uint32_t *__restrict__ out, int64_t total)
+{
+    const int Cw = (C + 31) >> 5;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(e % N);
+        const int64_t t = e / N;
+        const int cw = (int)(t % Cw);
+        const int pix = (int)(t / Cw);
+        uint32_t word = 0;
+        for (int j = 0; j < 32; ++j) {
+            const int c = cw * 32 + j;
+            if (c < C) word |= (uint32_t)(__ldg(w + ((int64_t)pix * C + c) * N + n) >= 0.0f) << j;
+        }
+        out[(int64_t)n * HW * Cw + (int64_t)pix * Cw + cw] = word;
+    }
+}
+
 __global__ void __launch_bounds__(256) rescale_kernel(const int32_t *__restrict__ p, int64_t M, int64_t N, int64_t ldp,
                                                       float alpha, const float *__restrict__ row_off,
                                                       const float *__restrict__ col_off, float delta,
@@ -158,6 +178,16 @@ int qnn_pack_conv_weights(const float *w, int Cout, int C, int KH, int KW, uint3
     const int64_t total = (int64_t)Cout * KH * KW * ceil_div(C, 32);
     conv_weight_pack_kernel<<<grid_for(total), 256, 0, as_stream(stream)>>>(w, Cout, C, KH, KW, out, total);
     return check_launch("qnn_pack_conv_weights");
+}
+
+int qnn_pack_fc_after_conv_weights(const float *w, int N, int C, int H, int W, uint32_t *out, void *stream)
+{
+    QNN_REQUIRE(N >= 0 && C >= 0 && H >= 1 && W >= 1, QNN_ERR_INVALID_ARG, "qnn_pack_fc_after_conv_weights: bad sizes");
+    if (N == 0 || C == 0) return QNN_OK;
+    QNN_REQUIRE(w && out, QNN_ERR_INVALID_ARG, "qnn_pack_fc_after_conv_weights: NULL pointer");
+    const int64_t total = (int64_t)N * H * W * ceil_div(C, 32);
+    fc_after_conv_pack_kernel<<<grid_for(total), 256, 0, as_stream(stream)>>>(w, N, C, H * W, out, total);
+    return check_launch("qnn_pack_fc_after_conv_weights");
 }
 
 int qnn_rescale_f32(const int32_t *p, int64_t M, int64_t N, int64_t ldp, float alpha, const float *row_off,

@@ -74,9 +74,16 @@ int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_
             const bool fits = tc_form_holds(form, g.ka, g.a_mode) && tc_form_holds(form, g.kb, g.b_mode) &&
                               (form != QNN_FORM_FP4 || tc_pick_form(g.ka, g.a_mode, g.kb, g.b_mode, g.K) == QNN_FORM_FP4);
             const int64_t kw = g.kwords > 0 ? g.kwords : ceil_div(g.K, 32);
-            const size_t need = round_up((size_t)g.M * (size_t)tc_row_pitch(kw, form), 256) +
-                                round_up((size_t)g.N * (size_t)tc_row_pitch(kw, form), 256);
-            if (!fits || kw == 0 || ws == nullptr || ws_bytes < need) algo = QNN_ALGO_POPC;
+            const size_t need = (g.a_tc ? 0 : round_up((size_t)g.M * (size_t)tc_row_pitch(kw, form), 256)) +
+                                (g.b_tc ? 0 : round_up((size_t)g.N * (size_t)tc_row_pitch(kw, form), 256));
+            if (!fits || kw == 0) {
+                algo = QNN_ALGO_POPC;
+            } else if (need > 0 && (ws == nullptr || !aligned(ws, 256) || ws_bytes < need)) {
+                // the result is the same, the speed is not: leave word of it where the caller can find it
+                note("gemm: QNN_ALGO_AUTO ran the CUDA-core kernel instead of the tensor-core one: it needs a 256-byte "
+                     "aligned workspace of %zu bytes (got %zu at %p)", need, ws_bytes, ws);
+                algo = QNN_ALGO_POPC;
+            }
         }
         if (algo == QNN_ALGO_B1_MMA && !(g.ka == 1 && g.kb == 1)) algo = QNN_ALGO_POPC;
     }

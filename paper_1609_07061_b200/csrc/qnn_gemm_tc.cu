@@ -23,6 +23,7 @@
 // code in a device status word, raises a block-wide abort flag, lets copies in
 // flight land, frees its tensor memory and returns.
 #include <cuda.h>
+#include <atomic>
 #include <cstdlib>
 #include "qnn_internal.cuh"
 
@@ -85,9 +86,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false when the block is aborting (this wait ran out, or another one did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code,
+                                          const uint32_t limit = WAIT_LIMIT)
 {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 4096) __nanosleep(64);
         if ((it & 63) == 63 && *abort_flag) return false;
@@ -428,6 +430,22 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t saddr)
     return d;
 }
 
+// Diagnostic: one CTA waits, with a short limit, on a barrier that nothing ever arrives on.  No copy and no MMA is in
+// flight, so the wait running out is all that happens: the status word is set through the same code path the product
+// kernel's waits use, and the kernel returns.
+constexpr int WAIT_PROBE_CODE = 9;
+__global__ void __launch_bounds__(32) wait_probe_kernel()
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        (void)mbar_wait(smem_u32(&bar), 0, &abort_flag, WAIT_PROBE_CODE, 1u << 13);
+    }
+}
+
 constexpr int next_pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
 template <int FORM, int BN, int STG, int CTAS, int KB = BKB>
@@ -693,7 +711,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         // accumulators are exact integers below 2^24 held as floats: compare there.  A threshold
                         // beyond +-2^24 decides the same way as +-2^24, which a float holds exactly.
                         tv = tv > (1 << 24) ? (1 << 24) : (tv < -(1 << 24) ? -(1 << 24) : tv);
-                        tv = __float_as_int((float)tv);
+                        // (a zero threshold is parked as -0.0: a sum that came out as -0.0 then gives -0.0 - (-0.0) = +0.0,
+                        // whose clear sign bit is the right answer to 0 >= 0; +0.0 would give -0.0)
+                        tv = tv == 0 ? (int32_t)0x80000000u : __float_as_int((float)tv);
                     } else if (p.thr_clamp > 0) {
                         // |sum| <= thr_clamp - 1 < 2^30: a threshold beyond +-thr_clamp decides like +-thr_clamp, and
                         // sum - threshold then cannot overflow, so its sign bit is the comparison
@@ -1131,18 +1151,34 @@ int max_pairs()
     return n;
 }
 
+// The same, asked once per device ordinal (the answer depends on the device's SM count and shared memory) and kept;
+// two host threads racing on the first call compute the same number.
+int pairs_resident_on_current_device()
+{
+    static std::atomic<int> cached[64];                 // 0 = not asked yet; stored as pairs + 1
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    int v = cached[dev].load(std::memory_order_acquire);
+    if (v == 0) {
+        v = max_pairs<QNN_FORM_FP4, 224, 0>() + 1;
+        cached[dev].store(v, std::memory_order_release);
+    }
+    return v - 1;
+}
+
 template <int FORM, int BN, int STG, int CTAS, int KB = BKB>
 int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mo, TcParams p, int workers, cudaStream_t st)
 {
     using S = TcCfg<FORM, BN, STG, CTAS, KB>;
     auto kern = gemm_tc_kernel<FORM, BN, STG, CTAS, KB>;
     // the shared-memory opt-in is per kernel and device: asked for once, not on every launch (it costs microseconds)
-    static bool opted_in[64] = {};
+    // (per device ordinal; racing first calls of two host threads both set the same attribute, which is harmless)
+    static std::atomic<bool> opted_in[64];
     int dev = 0;
     QNN_CUDA(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+    if (dev < 0 || dev >= 64 || !opted_in[dev].load(std::memory_order_acquire)) {
         QNN_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL));
-        if (dev >= 0 && dev < 64) opted_in[dev] = true;
+        if (dev >= 0 && dev < 64) opted_in[dev].store(true, std::memory_order_release);
     }
     const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
     QNN_REQUIRE(tiles < ((int64_t)1 << 31), QNN_ERR_UNSUPPORTED, "tc gemm: too many output tiles");
@@ -1326,7 +1362,16 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     if (g.pad_period > 0) { period = g.pad_period; tail = g.pad_tail; }
     QNN_REQUIRE(tail >= 1 && tail <= 32, QNN_ERR_INVALID_ARG, "tc gemm: inconsistent K / kwords");
 
-    // operands: use prepared ones, expand the others into the workspace
+    if (g.out_form) {
+        QNN_REQUIRE(g.thr != nullptr, QNN_ERR_INVALID_ARG, "tc gemm: thresholds required for a form output");
+        QNN_REQUIRE(g.out_form_kind == QNN_FORM_I8 || g.out_form_kind == QNN_FORM_FP4, QNN_ERR_INVALID_ARG, "tc gemm: bad output form");
+        QNN_REQUIRE(aligned(g.out_form, 16) && g.ld_form % 16 == 0 &&
+                        g.ld_form >= tc_row_bytes(ceil_div(g.N, 32), g.out_form_kind),
+                    QNN_ERR_ALIGNMENT, "tc gemm: form output needs a 16-byte aligned base and a row stride covering N");
+    }
+    if (g.conv) QNN_REQUIRE(g.a_tc != nullptr, QNN_ERR_INVALID_ARG, "tc conv: the NHWC operand must be prepared");
+
+    // operands: use prepared ones, expand the others into the workspace (every argument check comes before this point)
     const uint8_t *a8 = static_cast<const uint8_t *>(g.a_tc);
     const uint8_t *b8 = static_cast<const uint8_t *>(g.b_tc);
     int64_t a_ld = g.a_tc_ld, b_ld = g.b_tc_ld;
@@ -1367,13 +1412,6 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     p.epilogue = g.epilogue; p.out = g.out; p.ldo = g.ldo; p.hw = g.hw > 0 ? g.hw : 1;
     p.thr = g.thr; p.flip = g.flip; p.out_bits = g.out_bits; p.ld_bits = g.ld_bits;
     p.out_form = static_cast<uint8_t *>(g.out_form); p.ld_form = g.ld_form; p.out_form_kind = g.out_form_kind;
-    if (g.out_form) {
-        QNN_REQUIRE(g.thr != nullptr, QNN_ERR_INVALID_ARG, "tc gemm: thresholds required for a form output");
-        QNN_REQUIRE(g.out_form_kind == QNN_FORM_I8 || g.out_form_kind == QNN_FORM_FP4, QNN_ERR_INVALID_ARG, "tc gemm: bad output form");
-        QNN_REQUIRE(aligned(g.out_form, 16) && g.ld_form % 16 == 0 &&
-                        g.ld_form >= tc_row_bytes(ceil_div(g.N, 32), g.out_form_kind),
-                    QNN_ERR_ALIGNMENT, "tc gemm: form output needs a 16-byte aligned base and a row stride covering N");
-    }
     {
         const int64_t maxsum = g.K * ((1 << g.ka) - 1) * (int64_t)((1 << g.kb) - 1);
         p.thr_clamp = maxsum + 1 < ((int64_t)1 << 30) ? (int32_t)(maxsum + 1) : 0;
@@ -1424,7 +1462,7 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     // cross-SM hand-offs cost more than the pair saves (10000 x 4096 x 784: 41 -> 47 us), so those stay on single
     // CTAs.  QNN_TC_PAIRS=0 in the environment keeps single CTAs everywhere.
     static const bool pairs_off = [] { const char *e = getenv("QNN_TC_PAIRS"); return e && e[0] == '0'; }();
-    static const int pairs_resident = pairs_off ? 0 : max_pairs<QNN_FORM_FP4, 224, 0>();
+    const int pairs_resident = pairs_off ? 0 : pairs_resident_on_current_device();
     const int64_t tiles_m2 = ceil_div(g.M, 2 * BM);
     const bool pairs = !g.conv && pairs_resident >= 8 && p.num_kb >= 12 && tiles_m2 * ceil_div(g.N, 224) >= pairs_resident;
     if (pairs) {
@@ -1483,6 +1521,13 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
 }
 
 }  // namespace qnn
+
+extern "C" int qnn_selftest_wait_timeout(void *stream)
+{
+    using namespace qnn;
+    wait_probe_kernel<<<1, 32, 0, as_stream(stream)>>>();
+    return check_launch("qnn_selftest_wait_timeout");
+}
 
 extern "C" int qnn_device_status(void *stream)
 {

@@ -11,6 +11,8 @@ namespace qnn {
 // Records a formatted message in the thread-local error slot and returns `code`.
 int fail(int code, const char *fmt, ...);
 void clear_error();
+// Leaves a text in the same slot without failing the call (e.g. when QNN_ALGO_AUTO had to take a slower algorithm).
+void note(const char *fmt, ...);
 
 inline cudaStream_t as_stream(void *s) { return reinterpret_cast<cudaStream_t>(s); }
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }

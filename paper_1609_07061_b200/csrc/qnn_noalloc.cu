@@ -17,6 +17,9 @@ void *g_scratch_addr[kMaxDevices] = {};     // device address of g_noalloc_scrat
 
 // In host code the array's name is only a handle for the runtime, not an address a
 // kernel may use: the per-device address has to be asked for, with that device current.
+// The address is kept per device ordinal for the life of the process; it does not
+// survive cudaDeviceReset (a process that resets a device must not call this entry
+// point on it again).
 int scratch_for_current_device(void **out)
 {
     int dev = 0;
@@ -48,7 +51,8 @@ extern "C" int qnn_xnor_gemm_noalloc(const uint32_t *a, int64_t lda, const uint3
     QNN_REQUIRE(out != nullptr || M == 0 || N == 0, QNN_ERR_INVALID_ARG, "qnn_xnor_gemm_noalloc: out is NULL");
     if (int rc = validate_gemm(g)) return rc;
     if (M == 0 || N == 0) return QNN_OK;
-    QNN_REQUIRE(K >= 1, QNN_ERR_UNSUPPORTED, "qnn_xnor_gemm_noalloc: K must be at least 1");
+    // An empty sum: every output is 0, as qnn_xnor_gemm gives.  The CUDA-core kernel writes it and needs no scratch.
+    if (K == 0) return run_gemm(g, QNN_ALGO_POPC, nullptr, 0, as_stream(stream));
     const size_t need = gemm_tc_workspace_bytes(M, N, K, 1, 1);
     QNN_REQUIRE(need <= (size_t)QNN_NOALLOC_SCRATCH_BYTES, QNN_ERR_WORKSPACE,
                 "qnn_xnor_gemm_noalloc: this shape needs %zu bytes of operand scratch but the built-in array holds %zu; "

@@ -148,13 +148,13 @@ def test_cifar_convnet_table7(q):
     B = 128
     wl = workloads.cifar_convnet(B=B, seed=5)
     got = _run_net(q, wl, B)
-    idx = np.random.default_rng(0).choice(B, 3, replace=False)
+    idx = np.sort(np.random.default_rng(0).choice(B, 8, replace=False))
     want = oracle.convnet_forward(wl.X.numpy().astype(np.int32)[idx], _oracle_layers(wl))
     np.testing.assert_array_equal(got[idx], want)
     # the same images in a smaller batch give the same scores (tiling does not leak between images)
     wl2 = workloads.cifar_convnet(B=B, seed=5)
     wl2.X = wl.X[torch.from_numpy(idx)]
-    np.testing.assert_array_equal(_run_net(q, wl2, 3), want)
+    np.testing.assert_array_equal(_run_net(q, wl2, len(idx)), want)
 
 
 def test_convnet_argument_errors(q):
@@ -172,25 +172,61 @@ def test_convnet_argument_errors(q):
     assert e.value.status == q.QNN_ERR_INVALID_ARG
 
 
-def test_network_runners_replay_from_a_cuda_graph(q):
-    """Both whole-network calls are allocation-free and asynchronous: captured once in a CUDA graph, a replay
-    must reproduce the oracle's scores (the tensor-core kernels inside are launched with programmatic stream
-    serialisation, which the capture has to carry over)."""
+def _capture(fn):
+    """Runs fn() once eagerly (one-time kernel attributes), then captures a second call in a CUDA graph."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn()
+    torch.cuda.synchronize()
+    return g
+
+
+def test_mlp_forward_replays_from_a_cuda_graph(q):
+    """qnn_mlp_forward (Algorithm 4 as one call) is allocation-free and asynchronous: captured once in a CUDA
+    graph, every replay must reproduce the oracle's scores, on the tensor-core chain with prepacked weights."""
+    M, dims = 2100, (784, 1024, 1024, 10)
+    wl = workloads.mnist_mlp(M=M, dims=dims, seed=1)
+    packed, ldws = [], []
+    for Wm in wl.Ws:
+        K, N = Wm.shape
+        ld = (words_per_row(K) + 3) // 4 * 4
+        o = torch.zeros(N, ld, dtype=torch.int32, device="cuda")
+        q.qnn_quantize_pack_sign_t(Wm.cuda(), K, N, N, o, ld)
+        packed.append(o); ldws.append(ld)
+    thr = [t.cuda() for t in wl.Ts]
+    layers = q.make_mlp_layers(packed, ldws, dims[:-1], dims[1:], thr, [None] * len(thr))
+    keep = q.prepack_mlp_weights(layers, packed, 8)                                   # noqa: F841
+    assert q.qnn_select_algo(M, dims[2], dims[1], 1, 1, q.QNN_MODE_PM1, q.QNN_MODE_PM1) in (q.QNN_ALGO_TC_FP4, q.QNN_ALGO_TC_I8)
+    ws = torch.empty(q.qnn_mlp_workspace_bytes(M, 8, layers, q.QNN_ALGO_AUTO, 0), dtype=torch.uint8, device="cuda")
+    x = wl.X.cuda()
+    scores = torch.zeros(M, dims[-1], dtype=torch.int32, device="cuda")
+    g = _capture(lambda: q.qnn_mlp_forward(x, M, 8, layers, scores, q.QNN_ALGO_AUTO, ws))
+    want = oracle.mlp_forward(wl.X.numpy().astype(np.int32), [oracle.sign(w.numpy()) for w in wl.Ws],
+                              [t.numpy() for t in wl.Ts])
+    for _ in range(3):
+        scores.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        np.testing.assert_array_equal(scores.cpu().numpy(), want)
+
+
+def test_convnet_forward_replays_from_a_cuda_graph(q):
+    """qnn_convnet_forward likewise: captured once in a CUDA graph, a replay must reproduce the oracle's scores
+    (the tensor-core kernels inside are launched with programmatic stream serialisation, which the capture has
+    to carry over)."""
     B = 64
     wl = workloads.cifar_convnet(B=B, H=16, W=16, widths=(128, 128, 256, 256), fc=(256, 10), seed=5, thr=24)
     net = q.ConvNet(3, 16, 16, wl.conv_W, wl.conv_pool, wl.fc_W, wl.Ts, wl.flips)
     ws = net.workspace(B)
     x = wl.X.cuda()
     scores = torch.zeros(B, net.n_out, dtype=torch.int32, device="cuda")
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        net.forward(x, scores, ws)                    # first call outside the capture (one-time kernel attributes)
-        side.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=side):
-            net.forward(x, scores, ws)
-    torch.cuda.synchronize()
+    g = _capture(lambda: net.forward(x, scores, ws))
     want = oracle.convnet_forward(wl.X.numpy().astype(np.int32), _oracle_layers(wl))
     for _ in range(3):
         scores.fill_(-7)

@@ -80,12 +80,12 @@ def test_conv2d(q, B, C, H, W, Co, KH, KW, stride, pad, pad_bit, algo):
 
 @pytest.mark.parametrize("algo", ALGOS)
 def test_cifar_conv_config_sampled(q, algo):
-    """Config 4 at full size on the GPU; the oracle checks three whole images (first, middle, last)."""
+    """Config 4 at full size on the GPU; the oracle checks sixteen whole images spread over the batch."""
     wl = workloads.cifar_conv()
     X, Wt, T = wl.X.numpy(), wl.W.numpy(), wl.T.numpy()
     got, bits = _conv_gpu(q, X, Wt, T, None, 1, 1, 1, algo)
     ws = oracle.sign(Wt)
-    for b in (0, 63, 127):
+    for b in (0, 1, 7, 8, 15, 16, 31, 32, 63, 64, 65, 95, 96, 120, 126, 127):
         want = oracle.conv2d(oracle.sign(X[b:b + 1]), ws, 1, 1, 1)
         np.testing.assert_array_equal(got[b:b + 1], want)
         rows = want.transpose(0, 2, 3, 1).reshape(-1, 256)
@@ -157,6 +157,18 @@ def test_mnist_mlp_config_auto_chain(q, prepack):
     want = oracle.mlp_forward(wl.X.numpy()[rows].astype(np.int32), [oracle.sign(w.numpy()) for w in wl.Ws],
                               [t.numpy() for t in wl.Ts])
     np.testing.assert_array_equal(got[rows], want)
+    assert q.qnn_device_status() == 0
+
+
+def test_mnist_mlp_config_every_row(q):
+    """Config 2 at full size, the launch configuration bench.py times (automatic choice, prepacked weights):
+    ALL 10000 rows of scores against the oracle's Algorithm 4, so that one wrong bit in any layer of any row shows."""
+    wl = workloads.mnist_mlp()
+    got = _mlp_gpu(q, wl, 10000, 0, prepack=True)
+    want = oracle.mlp_forward(wl.X.numpy().astype(np.int32), [oracle.sign(w.numpy()) for w in wl.Ws],
+                              [t.numpy() for t in wl.Ts])
+    np.testing.assert_array_equal(got, want)
+    np.testing.assert_array_equal(_mlp_gpu(q, wl, 10000, 0, host=True, prepack=True), want)
     assert q.qnn_device_status() == 0
 
 
@@ -258,23 +270,49 @@ def test_square_1024_full(q, algo):
     np.testing.assert_array_equal(out.cpu().numpy(), oracle.xnor_gemm(wl.X.numpy(), wl.W.numpy()))
 
 
-@pytest.mark.parametrize("algo", ALGOS)
-@pytest.mark.parametrize("n", [4096, 8192])
-def test_square_large_sampled_and_checksums(q, n, algo):
-    """Sizes where the scalar oracle cannot run whole: exact oracle on sampled full rows and full columns, plus
-    int64 row-sum and column-sum checksums that cover every output:
-      sum_n out[m,n] = a_m . (sum_n w_n)   and   sum_m out[m,n] = (sum_m a_m) . w_n ."""
-    wl, out = _square(q, n, algo)
+def _check_square_sampled_and_checksums(wl, got, n):
+    """Exact oracle on sampled full rows and full columns, plus int64 row-sum and column-sum checksums that cover
+    every output:  sum_n out[m,n] = a_m . (sum_n w_n)   and   sum_m out[m,n] = (sum_m a_m) . w_n .
+    The sign matrices are walked in row blocks so that the 16384^2 case needs no int64 copy of them."""
     X, W = wl.X.numpy(), wl.W.numpy()
-    got = out.cpu().numpy()
     rows = np.array([0, 1, 127, 128, n // 2 + 1, n - 129, n - 2, n - 1])
     cols = np.array([0, 5, 127, 128, 255, n // 2, n - 128, n - 1])
     np.testing.assert_array_equal(got[rows], oracle.xnor_gemm(X[rows], W))
     np.testing.assert_array_equal(got[:, cols], oracle.xnor_gemm(X, np.ascontiguousarray(W[:, cols])))
-    sa = oracle.sign(X).astype(np.int64)
-    sw = oracle.sign(W).astype(np.int64)
-    np.testing.assert_array_equal(got.sum(axis=1, dtype=np.int64), sa @ sw.sum(axis=1))
-    np.testing.assert_array_equal(got.sum(axis=0, dtype=np.int64), sa.sum(axis=0) @ sw)
+    blk = 1024
+    w_rowsum = np.empty(n, np.int64)                 # sum_n sign(W)[k, n]
+    a_colsum = np.zeros(n, np.int64)                 # sum_m sign(X)[m, k]
+    for r0 in range(0, n, blk):
+        w_rowsum[r0:r0 + blk] = oracle.sign(W[r0:r0 + blk]).sum(axis=1, dtype=np.int64)
+        a_colsum += oracle.sign(X[r0:r0 + blk]).sum(axis=0, dtype=np.int64)
+    want_rows = np.empty(n, np.int64)
+    want_cols = np.zeros(n, np.int64)
+    for r0 in range(0, n, blk):
+        want_rows[r0:r0 + blk] = oracle.sign(X[r0:r0 + blk]).astype(np.int64) @ w_rowsum
+        want_cols += a_colsum[r0:r0 + blk] @ oracle.sign(W[r0:r0 + blk]).astype(np.int64)
+    np.testing.assert_array_equal(got.sum(axis=1, dtype=np.int64), want_rows)
+    np.testing.assert_array_equal(got.sum(axis=0, dtype=np.int64), want_cols)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_square_large_sampled_and_checksums(q, n, algo):
+    """Sizes where the scalar oracle cannot run whole: sampled rows / columns and full-coverage checksums."""
+    wl, out = _square(q, n, algo)
+    _check_square_sampled_and_checksums(wl, out.cpu().numpy(), n)
+
+
+@pytest.mark.parametrize("algo", [0, 4])
+def test_square_16384_sampled_and_checksums(q, algo):
+    """The largest square of the scaling sweep (2^28 outputs, the CTA-pair kernel's tile arithmetic at its
+    largest), on the algorithms the automatic choice can take there."""
+    n = 16384
+    wl, out = _square(q, n, algo)
+    got = out.cpu().numpy()
+    del out
+    torch.cuda.empty_cache()
+    assert q.qnn_device_status() == 0
+    _check_square_sampled_and_checksums(wl, got, n)
 
 
 @pytest.mark.parametrize("B,C,H,W,Co,KS,pad_bit", [(2, 256, 16, 16, 256, 3, 1), (2, 128, 13, 12, 70, 3, 0), (1, 256, 7, 20, 33, 5, 1),

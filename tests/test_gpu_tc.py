@@ -282,3 +282,93 @@ def test_logquant_products(q, M, N, K, la, lb):
     assert q.qnn_device_status() == 0, q.qnn_last_error()
     np.testing.assert_array_equal(out.t.cpu().numpy(), want)
     out.check()
+
+
+@pytest.mark.parametrize("K", [256, 512, 200])
+@pytest.mark.parametrize("a_rows", ["zeros", "mixed"])
+def test_fp4_zero_sum_against_zero_threshold(q, K, a_rows):
+    """An all-zero 2-bit activation row against all -1 weights sums products 0 * (-1): in fp32 the accumulator may
+    come out as -0.0.  Eq. 1 gives sign(0) = +1, so with threshold 0 the bit must be 1 whatever the zero's sign
+    (bits and form output; the oracle decides on integers)."""
+    M, N = 130, 70
+    rng = np.random.default_rng(K)
+    codes = np.zeros((M, K), np.int32) if a_rows == "zeros" else rng.integers(0, 4, (M, K)).astype(np.int32)
+    codes[::3] = 0                                               # whole rows of zeros among the others
+    wsign = -np.ones((K, N), np.int32)
+    if a_rows == "mixed":
+        wsign[:, 1::2] = np.where(rng.random((K, (N + 0) // 2)) < 0.5, 1, -1)
+    s = oracle.int_gemm(codes, wsign)
+    T = np.zeros(N, np.int32)
+    flip = np.zeros(N, np.uint8); flip[5::7] = 1
+    ld = words_per_row(K)
+    pl = _planes_ref(codes, 2, ld)
+    a = as_i32_words(pl).cuda()
+    b = as_i32_words(pack_bits_ref((wsign.T > 0).astype(np.uint8), ld)).cuda()
+    form = q.QNN_FORM_FP4
+    rb = q.qnn_tc_row_bytes(K, form)
+    af = torch.empty(M, rb, dtype=torch.uint8, device="cuda")
+    bf = torch.empty(N, rb, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(a, 2, q.QNN_MODE_U01, ld, M * ld, M, K, form, af, rb)
+    q.qnn_tc_prepack(b, 1, q.QNN_MODE_PM1, ld, 0, N, K, form, bf, rb)
+    ldw = words_per_row(N)
+    bits = Guarded((M, ldw), torch.int32, fill=0)
+    orb = q.qnn_tc_row_bytes(N, form)
+    of = Guarded((M, orb), torch.uint8, fill=0x5C)
+    out = Guarded((M, N), torch.int32, fill=-7)
+    q.qnn_tc_gemm(q.tc_operand(af, rb, form, 2, q.QNN_MODE_U01), q.tc_operand(bf, rb, form), M, N, K, out.t, N, dev(T), dev(flip),
+                  bits.t, ldw, of.t, form, orb)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    np.testing.assert_array_equal(out.t.cpu().numpy(), s)
+    want_bits = oracle.threshold(s, T, flip)
+    assert want_bits[0, 0] == 1                                  # 0 >= 0
+    np.testing.assert_array_equal(unpack_words(words_np(bits.t), N), want_bits)
+    onb = words_per_row(N) * 16
+    np.testing.assert_array_equal(of.t.cpu().numpy()[:, :onb], form_ref(2 * want_bits.astype(np.int32) - 1, N, form, q))
+    for g in (out, bits, of):
+        g.check()
+
+
+def test_bounded_wait_that_runs_out_is_reported_once_and_leaves_the_context_usable(q):
+    """Failure path of the device-side waits, provoked in the one harmless way: a diagnostic kernel polls a barrier
+    that nothing arrives on (no copy, no tensor-core work in flight) until its short limit runs out.  The status word
+    must report QNN_ERR_TIMEOUT exactly once, and a product right after must be bit-exact."""
+    assert q.qnn_device_status() == 0
+    q.qnn_selftest_wait_timeout()
+    assert q.qnn_device_status() == q.QNN_ERR_TIMEOUT
+    assert "wait" in q.qnn_last_error()
+    assert q.qnn_device_status() == 0
+    M, N, K = 200, 300, 1000
+    rng = np.random.default_rng(3)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+    ld = words_per_row(K)
+    a = as_i32_words(pack_bits_ref((X >= 0).astype(np.uint8), ld)).cuda()
+    b = as_i32_words(pack_bits_ref((W >= 0).astype(np.uint8).T, ld)).cuda()
+    out = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    ws = torch.empty(q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, N, K, 1, 1, q.QNN_ALGO_TC_FP4), dtype=torch.uint8, device="cuda")
+    q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, out, N, q.QNN_ALGO_TC_FP4, ws)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), oracle.xnor_gemm(X, W))
+
+
+def test_auto_leaves_a_note_when_it_cannot_use_the_workspace(q):
+    """QNN_ALGO_AUTO with no (or a misaligned) workspace still gives the right integers on the CUDA-core kernel, and says so."""
+    M, N, K = 300, 4096, 4096
+    assert q.qnn_select_algo(M, N, K) in (q.QNN_ALGO_TC_FP4, q.QNN_ALGO_TC_I8)
+    g = torch.Generator(device="cuda").manual_seed(1)
+    ld = K // 32
+    a = torch.randint(-2**31, 2**31 - 1, (M, ld), dtype=torch.int32, device="cuda", generator=g)
+    b = torch.randint(-2**31, 2**31 - 1, (N, ld), dtype=torch.int32, device="cuda", generator=g)
+    want = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, want, N, q.QNN_ALGO_POPC)
+    need = q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, N, K, 1, 1, q.QNN_ALGO_AUTO)
+    raw = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
+    off = (-raw.data_ptr()) % 256
+    for ws in (None, raw[off + 16: off + 16 + need]):
+        got = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+        q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, got, N, q.QNN_ALGO_AUTO, ws)
+        assert "CUDA-core kernel instead" in q.qnn_last_error()
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
