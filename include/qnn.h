@@ -257,6 +257,30 @@ typedef struct qnn_tc_output { /* any subset; at least one of out / out_bits / o
 QNN_API int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_t M, int64_t N, int64_t K,
                         const qnn_tc_output *o, void *stream);
 
+/* Eq. 1 / Eq. 9 straight into a tensor-core form: the same values and layout
+ * qnn_quantize_pack_* followed by qnn_tc_prepack would give, in one pass over
+ * the fp32 data (4 bytes read, 1/2 or 1 byte written per element, nothing
+ * re-read).  out: rows ld_bytes apart (a multiple of 16 covering
+ * qnn_tc_row_bytes' element bytes; whole 128-byte lines recommended), 16-byte
+ * aligned; elements between K and the next multiple of 32 are written as 0,
+ * bytes beyond that are left untouched.
+ *   _sign       x [rows, K] row-major              -> +-1 per element
+ *   _sign_t     w [K, N] row-major (weights)       -> rows n = 0..N-1 along K
+ *   _sign_nchw  x [B, C, H, W]                     -> rows (b, y, x) along C
+ *   _kbit / _kbit_t  Eq. 9 codes on [lo, hi]: the code q (mode QNN_MODE_U01)
+ *               or 2q - (2^bits - 1) (QNN_MODE_PM1); bits <= 2 for
+ *               QNN_FORM_FP4, <= 8 (U01) / 7 (PM1) for QNN_FORM_I8. */
+QNN_API int qnn_quantize_form_sign(const float *x, int64_t rows, int64_t K, int64_t ldx, int form, void *out,
+                                   int64_t ld_bytes, void *stream);
+QNN_API int qnn_quantize_form_sign_t(const float *w, int64_t K, int64_t N, int64_t ldw, int form, void *out,
+                                     int64_t ld_bytes, void *stream);
+QNN_API int qnn_quantize_form_sign_nchw(const float *x, int B, int C, int H, int W, int form, void *out,
+                                        int64_t ld_bytes, void *stream);
+QNN_API int qnn_quantize_form_kbit(const float *x, int64_t rows, int64_t K, int64_t ldx, int bits, float lo, float hi,
+                                   int mode, int form, void *out, int64_t ld_bytes, void *stream);
+QNN_API int qnn_quantize_form_kbit_t(const float *w, int64_t K, int64_t N, int64_t ldw, int bits, float lo, float hi,
+                                     int mode, int form, void *out, int64_t ld_bytes, void *stream);
+
 /* Size of the scratch array built into the library for qnn_xnor_gemm_noalloc. */
 #define QNN_NOALLOC_SCRATCH_BYTES (8u << 20)
 

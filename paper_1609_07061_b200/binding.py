@@ -86,6 +86,11 @@ _SIGS = {
     "qnn_bitplane_gemm": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, i64, i32, vp, sz, vp]),
     "qnn_bitplane_gemm_threshold": (i32, [vp, i32, i32, i64, i64, vp, i32, i32, i64, i64, i64, i64, i64, vp, vp, vp,
                                           i64, i32, vp, sz, vp]),
+    "qnn_quantize_form_sign": (i32, [vp, i64, i64, i64, i32, vp, i64, vp]),
+    "qnn_quantize_form_sign_t": (i32, [vp, i64, i64, i64, i32, vp, i64, vp]),
+    "qnn_quantize_form_sign_nchw": (i32, [vp, i32, i32, i32, i32, i32, vp, i64, vp]),
+    "qnn_quantize_form_kbit": (i32, [vp, i64, i64, i64, i32, ctypes.c_float, ctypes.c_float, i32, i32, vp, i64, vp]),
+    "qnn_quantize_form_kbit_t": (i32, [vp, i64, i64, i64, i32, ctypes.c_float, ctypes.c_float, i32, i32, vp, i64, vp]),
     "qnn_tc_form": (i32, [i32, i32, i32, i32, i64]),
     "qnn_tc_row_bytes": (i64, [i64, i32]),
     "qnn_tc_operand_bytes": (sz, [i64, i64, i32]),
@@ -237,6 +242,28 @@ def qnn_tc_operand_bytes(rows, K, form) -> int:
 def qnn_tc_prepack(planes, nplanes, mode, ld, plane_stride, rows, K, form, out, ld_bytes):
     _ck(_lib.qnn_tc_prepack(_p(planes), nplanes, mode, ld, plane_stride, rows, K, form, _p(out), ld_bytes, _stream()),
         "qnn_tc_prepack")
+
+
+def qnn_quantize_form_sign(x, rows, K, ldx, form, out, ld_bytes):
+    _ck(_lib.qnn_quantize_form_sign(_p(x), rows, K, ldx, form, _p(out), ld_bytes, _stream()), "qnn_quantize_form_sign")
+
+
+def qnn_quantize_form_sign_t(w, K, N, ldw, form, out, ld_bytes):
+    _ck(_lib.qnn_quantize_form_sign_t(_p(w), K, N, ldw, form, _p(out), ld_bytes, _stream()), "qnn_quantize_form_sign_t")
+
+
+def qnn_quantize_form_sign_nchw(x, B, C, H, W, form, out, ld_bytes):
+    _ck(_lib.qnn_quantize_form_sign_nchw(_p(x), B, C, H, W, form, _p(out), ld_bytes, _stream()), "qnn_quantize_form_sign_nchw")
+
+
+def qnn_quantize_form_kbit(x, rows, K, ldx, bits, lo, hi, mode, form, out, ld_bytes):
+    _ck(_lib.qnn_quantize_form_kbit(_p(x), rows, K, ldx, bits, lo, hi, mode, form, _p(out), ld_bytes, _stream()),
+        "qnn_quantize_form_kbit")
+
+
+def qnn_quantize_form_kbit_t(w, K, N, ldw, bits, lo, hi, mode, form, out, ld_bytes):
+    _ck(_lib.qnn_quantize_form_kbit_t(_p(w), K, N, ldw, bits, lo, hi, mode, form, _p(out), ld_bytes, _stream()),
+        "qnn_quantize_form_kbit_t")
 
 
 def tc_operand(data, ld_bytes, form, planes=1, mode=QNN_MODE_PM1) -> qnn_tc_operand:

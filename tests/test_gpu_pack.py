@@ -231,3 +231,146 @@ def test_logquant_argument_errors(q):
     with pytest.raises(q.QnnError) as e:
         q.qnn_logquant_pack_i8(x, 4, 20, 32, 0, 1, out, 20)           # row stride below K rounded up to 32
     assert e.value.status == q.QNN_ERR_INVALID_ARG
+
+
+# ---- quantisers that write a tensor-core form directly ---------------------------------------------------------
+
+_E2M1 = {0: 0x0, 1: 0x2, 2: 0x4, 3: 0x5, -1: 0xA, -2: 0xC, -3: 0xD}
+
+
+def _form_bytes_of(values, K, form, q):
+    """Test-side encoding of integer values [rows, K] in a tensor-core form; elements K .. next multiple of 32 are 0."""
+    rows = values.shape[0]
+    kp = words_per_row(K) * 32
+    v = np.zeros((rows, kp), np.int32)
+    v[:, :K] = values
+    if form == q.QNN_FORM_I8:
+        return (v & 0xff).astype(np.uint8)
+    nib = np.vectorize(_E2M1.__getitem__)(v).astype(np.uint8)
+    return (nib[:, 0::2] | (nib[:, 1::2] << 4)).astype(np.uint8)
+
+
+_SPECIALS = np.array([0.0, -0.0, 1e-45, -1e-45, np.inf, -np.inf, np.nan, 1.0, -1.0, 0.5, 1.0 / 6.0, 0.49999997, 2.5 / 3.0],
+                     np.float32)
+
+
+@pytest.mark.parametrize("form_name", ["FP4", "I8"])
+@pytest.mark.parametrize("rows,K,ldx", [(1, 1, 1), (3, 31, 33), (5, 33, 36), (7, 1024, 1024), (130, 1000, 1000), (33, 4097, 4100), (100, 4096, 4096)])
+def test_quantize_form_sign_row_major(q, rows, K, ldx, form_name):
+    """Eq. 1 straight into a tensor-core form, row-major source: values +-1, pads 0, bytes past the row untouched."""
+    form = getattr(q, "QNN_FORM_" + form_name)
+    rng = np.random.default_rng(rows * 7 + K)
+    X = rng.standard_normal((rows, ldx)).astype(np.float32)
+    X.reshape(-1)[: min(X.size, _SPECIALS.size)] = _SPECIALS[: min(X.size, _SPECIALS.size)]
+    eb = words_per_row(K) * (32 if form == q.QNN_FORM_I8 else 16)
+    ldb = eb + 16
+    out = Guarded((rows, ldb), torch.uint8, fill=0x5C)
+    q.qnn_quantize_form_sign(dev(X), rows, K, ldx, form, out.t, ldb)
+    torch.cuda.synchronize()
+    got = out.t.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :eb], _form_bytes_of(oracle.sign(X[:, :K]), K, form, q))
+    assert (got[:, eb:] == 0x5C).all()
+    out.check()
+
+
+@pytest.mark.parametrize("form_name", ["FP4", "I8"])
+@pytest.mark.parametrize("K,N,ldw", [(1, 1, 1), (31, 5, 5), (33, 7, 8), (64, 130, 132), (1000, 257, 260), (4096, 512, 512), (96, 1000, 1003)])
+def test_quantize_form_sign_transposed(q, K, N, ldw, form_name):
+    """Weights [K, N] -> form rows [N, K] (one row per output unit), as qnn_tc_gemm's B operand wants them."""
+    form = getattr(q, "QNN_FORM_" + form_name)
+    rng = np.random.default_rng(K * 3 + N)
+    W = rng.uniform(-1, 1, (K, ldw)).astype(np.float32)
+    W.reshape(-1)[: min(W.size, _SPECIALS.size)] = _SPECIALS[: min(W.size, _SPECIALS.size)]
+    eb = words_per_row(K) * (32 if form == q.QNN_FORM_I8 else 16)
+    ldb = (eb + 127) // 128 * 128
+    out = Guarded((N, ldb), torch.uint8, fill=0x5C)
+    q.qnn_quantize_form_sign_t(dev(W), K, N, ldw, form, out.t, ldb)
+    torch.cuda.synchronize()
+    got = out.t.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :eb], _form_bytes_of(oracle.sign(W[:, :N]).T, K, form, q))
+    assert (got[:, eb:] == 0x5C).all()
+    out.check()
+
+
+@pytest.mark.parametrize("B,C,H,W", [(2, 256, 16, 16), (3, 128, 5, 7), (1, 40, 3, 3), (2, 512, 8, 8)])
+def test_quantize_form_sign_nchw(q, B, C, H, W):
+    """NCHW fp32 -> NHWC pixels in e2m1 form (the implicit convolution's A operand)."""
+    form = q.QNN_FORM_FP4
+    rng = np.random.default_rng(B + C + H)
+    X = rng.standard_normal((B, C, H, W)).astype(np.float32)
+    eb = words_per_row(C) * 16
+    out = Guarded((B * H * W, eb), torch.uint8, fill=0x5C)
+    q.qnn_quantize_form_sign_nchw(dev(X), B, C, H, W, form, out.t, eb)
+    torch.cuda.synchronize()
+    want = _form_bytes_of(oracle.sign(X).transpose(0, 2, 3, 1).reshape(-1, C), C, form, q)
+    np.testing.assert_array_equal(out.t.cpu().numpy(), want)
+    out.check()
+
+
+@pytest.mark.parametrize("bits,lo,hi,mode,form_name", [(2, 0.0, 1.0, 0, "FP4"), (2, -1.0, 1.0, 1, "FP4"), (1, -1.0, 1.0, 1, "FP4"),
+                                                       (4, -1.0, 1.0, 1, "I8"), (8, 0.0, 1.0, 0, "I8"), (2, 0.0, 1.0, 0, "I8"), (3, -2.0, 5.0, 0, "I8")])
+@pytest.mark.parametrize("transposed", [False, True])
+def test_quantize_form_kbit(q, bits, lo, hi, mode, form_name, transposed):
+    """Eq. 9 straight into a form: codes (or their signed-symmetric values) as the oracle's quantiser gives them,
+    including exact ties, level centres, clipping and the special values."""
+    form = getattr(q, "QNN_FORM_" + form_name)
+    rows, K = (130, 1000)
+    rng = np.random.default_rng(bits * 10 + mode)
+    X = (rng.standard_normal((rows, K)) * (hi - lo) * 0.6 + (hi + lo) / 2).astype(np.float32)
+    L = (1 << bits) - 1
+    step = (hi - lo) / L
+    ties = (lo + (np.arange(L) + 0.5) * step).astype(np.float32)
+    X[0, :ties.size] = ties
+    X[1, :L + 1] = (lo + np.arange(L + 1) * step).astype(np.float32)
+    X[2, :_SPECIALS.size] = _SPECIALS
+    codes = oracle.linear_quant_codes(X, bits, lo, hi)
+    vals = oracle.codes_to_symmetric(codes, bits) if mode == 1 else codes
+    eb = words_per_row(K if not transposed else rows) * (32 if form == q.QNN_FORM_I8 else 16)
+    if not transposed:
+        out = Guarded((rows, eb + 32), torch.uint8, fill=0x5C)
+        q.qnn_quantize_form_kbit(dev(X), rows, K, K, bits, lo, hi, mode, form, out.t, eb + 32)
+        want = _form_bytes_of(vals, K, form, q)
+    else:
+        # the same matrix read as [K' = rows, N' = K]: rows of the result run along the source's first index
+        out = Guarded((K, eb + 32), torch.uint8, fill=0x5C)
+        q.qnn_quantize_form_kbit_t(dev(X), rows, K, K, bits, lo, hi, mode, form, out.t, eb + 32)
+        want = _form_bytes_of(vals.T, rows, form, q)
+    torch.cuda.synchronize()
+    got = out.t.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :eb], want)
+    assert (got[:, eb:] == 0x5C).all()
+    out.check()
+
+
+def test_form_quantisers_feed_the_product(q):
+    """fp32 -> form -> qnn_tc_gemm with no packed planes anywhere: the config-1 layer (100 x 4096 x 4096) against the oracle."""
+    wl = workloads.fc_single()
+    X, W = wl.X.numpy(), wl.W.numpy()
+    M, K = X.shape
+    N = W.shape[1]
+    form = q.qnn_tc_form(1, q.QNN_MODE_PM1, 1, q.QNN_MODE_PM1, K)
+    rb = q.qnn_tc_row_bytes(K, form)
+    af = torch.empty(M, rb, dtype=torch.uint8, device="cuda")
+    bf = torch.empty(N, rb, dtype=torch.uint8, device="cuda")
+    q.qnn_quantize_form_sign(wl.X.cuda(), M, K, K, form, af, rb)
+    q.qnn_quantize_form_sign_t(wl.W.cuda(), K, N, N, form, bf, rb)
+    out = Guarded((M, N), torch.int32, fill=-7)
+    q.qnn_tc_gemm(q.tc_operand(af, rb, form), q.tc_operand(bf, rb, form), M, N, K, out.t, N)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0
+    np.testing.assert_array_equal(out.t.cpu().numpy(), oracle.xnor_gemm(X, W))
+    out.check()
+
+
+def test_form_quantiser_argument_errors(q):
+    x = torch.zeros(4, 64, device="cuda")
+    out = torch.zeros(4, 64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_quantize_form_kbit(x, 4, 64, 64, 4, -1.0, 1.0, 1, q.QNN_FORM_FP4, out, 64)      # 4-bit values do not fit e2m1
+    assert e.value.status == q.QNN_ERR_UNSUPPORTED
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_quantize_form_sign(x, 4, 64, 64, q.QNN_FORM_FP4, out, 24)                       # row stride not a multiple of 16
+    assert e.value.status == q.QNN_ERR_ALIGNMENT
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_quantize_form_sign(x, 4, 64, 64, 7, out, 64)
+    assert e.value.status == q.QNN_ERR_INVALID_ARG
