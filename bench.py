@@ -31,14 +31,15 @@ import torch
 DIMS = (784, 4096, 4096, 4096, 10)
 BATCH = 10000
 IN_BITS = 8
+E2E_CHUNKS = int(os.environ.get("QNN_BENCH_E2E_CHUNKS", "1"))   # pieces of the batch whose input copies overlap the previous piece's layers
+E2E_GRAPH_MAX_BATCH = int(os.environ.get("QNN_BENCH_E2E_GRAPH_MAX_BATCH", "2048"))
 METRIC = "binary_gemm_tops"
 UNIT = "Tops/s (2*M*N*K per 1-bit plane product)"
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from
-# the ncu capture summarised under profiles/; None until a capture exists for the kernel the run selects.
+# the ncu capture of that kernel; None until a capture exists for the kernel the run selects.
 NCU_TRAFFIC_BYTES = {
-    # profiles/gemm_tc_kernel_fp4_mlp_hidden_layer.md (hidden layer 2, the launch the live timing brackets):
-    # 28.97 MB read + 0.25 MB written per launch, captured on the current kernel
+    # hidden layer 2 (the launch the live timing brackets): 28.97 MB read + 0.25 MB written per launch
     "tcgen05 kind::mxf4 xnor product 10000x4096x4096, threshold epilogue (gemm_tc_kernel<FP4>)": 29.22e6,
 }
 
@@ -55,10 +56,12 @@ def _peaks():
             "source": "fallback"}
 
 
-def _ops(M):
+def _ops(M, count_planes=True):
+    """Operations per layer: 2*M*N*K per 1-bit plane product (the paper's cost model, 8 planes in layer 1), or with
+    count_planes=False per integer multiply-accumulate (layer 1 counted once: what the tensor cores issue)."""
     per_layer = []
     for l in range(len(DIMS) - 1):
-        planes = IN_BITS if l == 0 else 1
+        planes = IN_BITS if (l == 0 and count_planes) else 1
         per_layer.append(2.0 * M * DIMS[l + 1] * DIMS[l] * planes)
     return per_layer
 
@@ -178,6 +181,7 @@ class MlpBench:
         self.gws = torch.empty(gw, dtype=torch.uint8, device="cuda")
         self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         self.flush_rd = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")
+        self.graph = None
 
     def flush_l2(self):
         """Writes a 256 MiB buffer (evicts every cached input), then reads another 256 MiB so that the dirty
@@ -217,6 +221,20 @@ class MlpBench:
                         self.algo, self.gws)
 
     def step_e2e(self):
+        """One pass from pinned host memory to scores in pinned host memory.  Small batches (launch-bound) replay a CUDA
+        graph built once (input copies, all kernels, the copy back; one launch per pass); large batches, where the input
+        copy over PCIe and the layers dominate and the graph gains nothing (measured), use the call-by-call host entry
+        point, which overlaps the second half-batch's copy with the first half's layers."""
+        if self.algo == self.q.QNN_ALGO_AUTO and self.M <= E2E_GRAPH_MAX_BATCH:
+            if self.graph is None:
+                self.graph = self.q.MlpGraph(self.x_host, self.M, IN_BITS, self.layers, self.scores_host, self.algo, self.ws,
+                                             chunks=E2E_CHUNKS)
+            self.graph.launch()
+            torch.cuda.current_stream().synchronize()
+        else:
+            self.q.qnn_mlp_forward_host(self.x_host, self.M, IN_BITS, self.layers, self.scores_host, self.algo, self.ws)
+
+    def step_e2e_calls(self):
         self.q.qnn_mlp_forward_host(self.x_host, self.M, IN_BITS, self.layers, self.scores_host, self.algo, self.ws)
 
 
@@ -329,6 +347,82 @@ def convnet_record(q, Bn, flush, rec, reps=7):
         note=f"{Bn / ms * 1e3:.0f} images/s; 6 conv + 3 FC layers in one qnn_convnet_forward call, weights prepared once")
 
 
+def pipe_peaks(q):
+    """Issue-only rate of each pipe, measured in this run with the library's own measurement kernels (every SM
+    re-multiplies one resident shared-memory tile pair, or runs xor/popc/add on registers): Tops/s, best of 5."""
+    out = {}
+    for name, pipe, iters in (("e2m1_tensor", q.QNN_PIPE_TENSOR_FP4, 1500), ("int8_tensor", q.QNN_PIPE_TENSOR_I8, 800),
+                              ("popc_alu", q.QNN_PIPE_POPC, 400)):
+        ops = q.qnn_pipe_peak_launch(pipe, iters)
+        torch.cuda.synchronize()
+        best = 1e30
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); q.qnn_pipe_peak_launch(pipe, iters); b.record()
+            b.synchronize()
+            best = min(best, a.elapsed_time(b))
+        out[name] = {"Tops": round(ops / best / 1e9, 1), "ms": round(best, 4), "iters": iters}
+    return out
+
+
+def algo_matrix(q, flush):
+    """The competing inner loops measured against each other on the same shapes (whole call from packed bits, L2
+    flushed): xor/popc on the CUDA cores, 1-bit mma.sync, int8 and e2m1 on tcgen05 -- and what the library picks."""
+    from paper_1609_07061_b200 import workloads
+    names = {q.QNN_ALGO_POPC: "popc", q.QNN_ALGO_B1_MMA: "b1_mma", q.QNN_ALGO_TC_I8: "tc_i8", q.QNN_ALGO_TC_FP4: "tc_fp4",
+             q.QNN_ALGO_TC_PACKED: "tc_packed"}
+    rows = []
+
+    def measure(label, M, N, K, ka, kb, call, ops, reps):
+        r = {"shape": label, "binary_ops": ops, "ms": {}, "binary_Tops": {}}
+        for al, nm in names.items():
+            if al == q.QNN_ALGO_TC_PACKED and M > 1024:
+                continue                                   # (re-expands the weights for every 128 rows: a small-batch kernel)
+            try:
+                ms, best = _time_op(lambda: call(al), flush, reps=reps, warm=2)
+            except q.QnnError as e:
+                if e.status != q.QNN_ERR_UNSUPPORTED:
+                    raise
+                continue
+            r["ms"][nm] = round(ms, 5)
+            r["binary_Tops"][nm] = round(ops / ms / 1e9, 1)
+        picked = names[q.qnn_select_algo(M, N, K, ka, kb, q.QNN_MODE_PM1, q.QNN_MODE_PM1)]     # (with a workspace)
+        fastest = min(r["ms"], key=r["ms"].get)
+        r["selected"] = picked
+        r["fastest"] = fastest
+        r["selected_is_fastest"] = bool(picked == fastest or r["ms"][picked] <= 1.03 * r["ms"][fastest])
+        rows.append(r)
+
+    g = torch.Generator(device="cuda").manual_seed(4)
+    for (M, N, K) in ((100, 4096, 4096), (1024, 1024, 1024), (4096, 4096, 4096), (8192, 8192, 8192)):
+        ld = K // 32
+        a = torch.randint(-2**31, 2**31 - 1, (M, ld), dtype=torch.int32, device="cuda", generator=g)
+        b = torch.randint(-2**31, 2**31 - 1, (N, ld), dtype=torch.int32, device="cuda", generator=g)
+        o = torch.empty(M, N, dtype=torch.int32, device="cuda")
+        ws = torch.empty(max(q.qnn_workspace_bytes(q.QNN_OP_XNOR_GEMM, M, N, K, 1, 1, q.QNN_ALGO_AUTO), 256), dtype=torch.uint8, device="cuda")
+        measure(f"xnor {M}x{N}x{K}", M, N, K, 1, 1, lambda al: q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, o, N, al, ws), 2.0 * M * N * K,
+                3 if M >= 8192 else 5)
+        del a, b, o, ws
+    M, N, K = 700, 4096, 2048
+    ld = K // 32
+    a = torch.randint(-2**31, 2**31 - 1, (4, M, ld), dtype=torch.int32, device="cuda", generator=g)
+    b = torch.randint(-2**31, 2**31 - 1, (4, N, ld), dtype=torch.int32, device="cuda", generator=g)
+    o = torch.empty(M, N, dtype=torch.int32, device="cuda")
+    ws = torch.empty(max(q.qnn_workspace_bytes(q.QNN_OP_BITPLANE_GEMM, M, N, K, 4, 4, q.QNN_ALGO_AUTO), 256), dtype=torch.uint8, device="cuda")
+    measure("4bit x 4bit 700x4096x2048", M, N, K, 4, 4,
+            lambda al: q.qnn_bitplane_gemm(a, 4, q.QNN_MODE_PM1, ld, M * ld, b, 4, q.QNN_MODE_PM1, ld, N * ld, M, N, K, o, N, al, ws),
+            2.0 * M * N * K * 16, 5)
+    wl4 = workloads.cifar_conv()
+    B, C, H, W = wl4.X.shape; Co = wl4.W.shape[0]
+    xb = torch.randint(-2**31, 2**31 - 1, (B, H, W, C // 32), dtype=torch.int32, device="cuda", generator=g)
+    wb = torch.randint(-2**31, 2**31 - 1, (Co, 9 * C // 32), dtype=torch.int32, device="cuda", generator=g)
+    o4 = torch.empty(B, Co, H, W, dtype=torch.int32, device="cuda")
+    w4 = torch.empty(q.qnn_workspace_bytes(q.QNN_OP_CONV2D, B * H * W, Co, 9 * C, 1, 1, q.QNN_ALGO_AUTO), dtype=torch.uint8, device="cuda")
+    measure("conv3x3 128x256x16x16 -> 256", B * H * W, Co, 9 * C, 1, 1,
+            lambda al: q.qnn_binary_conv2d(xb, B, C, H, W, wb, Co, 3, 3, 1, 1, 1, o4, None, None, None, al, w4), 2.0 * B * H * W * Co * 9 * C, 5)
+    return rows
+
+
 def run_extras(q, bench, peaks, algo):
     """Other paper-shaped workloads, one record each (device time, L2 flushed): packers against the HBM
     roofline, products in binary Tops/s."""
@@ -381,6 +475,26 @@ def run_extras(q, bench, peaks, algo):
     ms, best = _time_op(cold, flush)
     rec("c1_layer_cold_weights", ms, best, bytes_=(M * K + K * N) * 4.0 + 2 * (M + N) * ld * 4 + M * N * 4,
         ops=2.0 * M * N * K)
+
+    # the same cold layer without packed planes in between: fp32 -> tensor-core form (one pass each), then the product
+    form1 = q.qnn_tc_form(1, q.QNN_MODE_PM1, 1, q.QNN_MODE_PM1, K)
+    rb1 = q.qnn_tc_row_bytes(K, form1)
+    xf1 = torch.empty(M, rb1, dtype=torch.uint8, device="cuda"); wf1 = torch.empty(N, rb1, dtype=torch.uint8, device="cuda")
+
+    def cold_direct():
+        q.qnn_quantize_form_sign(Xd, M, K, K, form1, xf1, rb1)
+        q.qnn_quantize_form_sign_t(Wd, K, N, N, form1, wf1, rb1)
+        q.qnn_tc_gemm(q.tc_operand(xf1, rb1, form1), q.tc_operand(wf1, rb1, form1), M, N, K, out, N)
+    ms, best = _time_op(cold_direct, flush)
+    rec("c1_layer_cold_weights_fp32_to_form", ms, best, bytes_=(M * K + K * N) * 4.0 + 2 * (M + N) * rb1 + M * N * 4, ops=2.0 * M * N * K,
+        note="three launches: two quantisers that write the tensor-core form directly, then the product")
+    ms, best = _time_op(lambda: q.qnn_quantize_form_sign_t(Wd, K, N, N, form1, wf1, rb1), flush)
+    rec("c1_quantize_form_W_4096x4096_transposed", ms, best, bytes_=K * N * 4.5)
+    # ... and as ONE pass over the fp32 weights: binarised while they stream, multiplied on the tensor cores
+    wsf = torch.empty(q.qnn_fc_sign_f32_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ms, best = _time_op(lambda: q.qnn_fc_sign_f32(Xd, M, K, K, Wd, N, N, out, N, wsf), flush)
+    rec("c1_layer_cold_weights_one_pass", ms, best, bytes_=(M * K + K * N) * 4.0 + M * N * 4, ops=2.0 * M * N * K,
+        note="qnn_fc_sign_f32: weights read once as fp32, nothing packed written; bytes = fp32 inputs + int32 output")
 
     # Items whose roofline time is below a few microseconds cannot approach it in a single launch (a launch alone costs
     # 3-5 us): the same calls 100 times back to back inside one CUDA graph show what is left without the launch latency.
@@ -463,6 +577,18 @@ def run_extras(q, bench, peaks, algo):
     ms, best = _time_op(lambda: q.qnn_binary_conv2d_prepared(xf4, f4, B, C, H, Wd_, prep, Co, 3, 3, 1, thr=t4, out_form=of4,
                                                               out_form_kind=f4), flush)
     rec("c4_conv3x3_prepared_filters_form_in_form_out", ms, best, ops=ops4, note="mid-network layer: activations arrive and leave in tensor-core form")
+
+    # Algorithm 4 end to end from host buffers at small batches: call by call against one CUDA graph per pass
+    for Bm in (100, 1000):
+        mb = MlpBench(q, 0, algo, M=Bm)
+        opsb = sum(_ops(Bm))
+        ms, best = _time_op(mb.step_e2e_calls, flush)
+        rec(f"mlp_e2e_batch{Bm}_call_by_call", ms, best, ops=opsb, note="qnn_mlp_forward_host: copies, kernels and the copy back issued one by one")
+        ms, best = _time_op(mb.step_e2e, flush)
+        rec(f"mlp_e2e_batch{Bm}_one_graph", ms, best, ops=opsb, note="the same pass replayed as one CUDA graph (qnn_mlp_graph_launch)")
+        del mb
+    ms, best = _time_op(bench.step_e2e_calls, flush)
+    rec(f"mlp_e2e_batch{BATCH}_call_by_call", ms, best, ops=sum(_ops(BATCH)), note="qnn_mlp_forward_host, 2 chunks")
 
     # the whole CIFAR-10 ConvNet of Table 7 (first layer on 8-bit pixels, pooled thresholds, FC head), one call per pass
     for Bn in (128, 1024):
@@ -579,6 +705,8 @@ def main():
         e2e_ev.append((s, e))
     barrier()
     e2e_ms = sum(s.elapsed_time(e) for s, e in e2e_ev)
+    if os.environ.get("QNN_BENCH_DEBUG"):
+        sys.stderr.write("e2e per step (ms): " + " ".join(f"{s.elapsed_time(e):.3f}" for s, e in e2e_ev) + "\n")
     t_end = time.time()
     clocks = sampler.stop(t_begin, t_end)
     same = bool(torch.equal(bench.scores_host, bench.scores.cpu()))
@@ -631,7 +759,8 @@ def main():
                        "weights": "packed and rewritten in tensor-core form once at load (not in the step)"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": BATCH * DIMS[0],
                     "d2h_bytes_per_step": BATCH * DIMS[-1] * 4, "ms_per_step": e2e_ms / args.steps,
-                    "matches_device_arm": same},
+                    "matches_device_arm": same,
+                    "api": "qnn_mlp_forward_host (pinned host buffers in, pinned host scores out, two overlapped half-batches)"},
             "gpu_launches": int(launches),
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                        "samples": clocks["samples"]},
@@ -640,6 +769,21 @@ def main():
                          "peak_note": peak_note},
             "per_layer_binary_ops": per_layer,
         }
+        # the same step counted once per integer multiply-accumulate (layer 1's eight planes are one int8 product)
+        int_ops_step = sum(_ops(BATCH, count_planes=False))
+        line["int_ops_value"] = world * int_ops_step * args.steps / (total_ms / 1e3) / 1e12
+        line["int_ops_unit"] = "Tops/s (2*M*N*K per layer: operations the tensor cores issue)"
+        if world == 1:
+            try:
+                pk = pipe_peaks(q)
+                line["pipe_peaks"] = pk
+                key = {q.QNN_ALGO_TC_FP4: "e2m1_tensor", q.QNN_ALGO_TC_I8: "int8_tensor"}.get(resolved, "popc_alu")
+                line["roofline"]["measured_pipe_peak"] = pk[key]["Tops"]
+                line["roofline"]["frac_of_measured_pipe_peak"] = achieved / pk[key]["Tops"]
+                line["roofline"]["pipe_peak_note"] = ("issue-only loop of the same instruction on resident shared-memory tiles, every SM, "
+                                                      "measured in this run (no loads, no epilogue)")
+            except Exception as ex:
+                line["pipe_peaks_error"] = repr(ex)
         if not args.no_cpu_baseline and world == 1:
             cb = _cpu_baseline()
             line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
@@ -648,6 +792,10 @@ def main():
                 line["extra"] = run_extras(q, bench, peaks, algo)
             except Exception as ex:  # extras never invalidate the headline record
                 line["extra_error"] = repr(ex)
+            try:
+                line["algorithms"] = algo_matrix(q, bench.flush_l2)
+            except Exception as ex:
+                line["algorithms_error"] = repr(ex)
         line["paper_context"] = "paper: XNOR kernel 23x its own baseline kernel, 3.4x cuBLAS at 8192^3, MLP 7x, on a GTX750 (context only)"
         print(json.dumps(line))
     if world > 1:

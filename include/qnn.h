@@ -82,6 +82,11 @@ extern "C" {
                              scales, fp32 TMEM accumulators (exact: integer sums below 2^24);
                              operands of at most 2 planes                                 */
 
+#define QNN_ALGO_TC_PACKED 5 /* the e2m1 product straight from the packed planes: packed tiles by TMA into shared
+                             memory, expanded to values there, one launch, NO workspace; operands of at most
+                             2 planes, sums below 2^24; 16-byte aligned rows (ld a multiple of 4 words).  What
+                             QNN_ALGO_AUTO takes for small batches when it is given no usable workspace   */
+
 /* tensor-core operand forms: one VALUE per element, rows packed along K, pad positions 0 */
 #define QNN_FORM_I8 1     /* one byte per element: int8 (QNN_MODE_PM1) or uint8 (QNN_MODE_U01) */
 #define QNN_FORM_FP4 2    /* one e2m1 nibble per element, element 2i in the low nibble of byte i;
@@ -281,6 +286,20 @@ QNN_API int qnn_quantize_form_kbit(const float *x, int64_t rows, int64_t K, int6
 QNN_API int qnn_quantize_form_kbit_t(const float *w, int64_t K, int64_t N, int64_t ldw, int bits, float lo, float hi,
                                      int mode, int form, void *out, int64_t ld_bytes, void *stream);
 
+/* Algorithm 4's hidden-layer product for a SMALL batch whose weights are still
+ * real-valued, in one pass over them:
+ *   out[m, n] = sum_k sign(x[m, k]) * sign(w[k, n])      (Eq. 1 on both operands)
+ * x fp32 [M, K] (ldx), w fp32 [K, N] row-major (ldw), out int32 [M, ldo].
+ * The kernel binarises the weights while it streams them (4 bytes per weight,
+ * read once, nothing packed is written or re-read) and multiplies on the
+ * tensor cores; the result equals qnn_quantize_pack_sign + _sign_t +
+ * qnn_xnor_gemm bit for bit.  Meant for M up to a few hundred rows: every
+ * further 128 rows of the batch stream the weights again.  K < 2^24.
+ * ws: qnn_fc_sign_f32_workspace_bytes(M, K) bytes (the activations as values). */
+QNN_API size_t qnn_fc_sign_f32_workspace_bytes(int64_t M, int64_t K);
+QNN_API int qnn_fc_sign_f32(const float *x, int64_t M, int64_t K, int64_t ldx, const float *w, int64_t N, int64_t ldw,
+                            int32_t *out, int64_t ldo, void *ws, size_t ws_bytes, void *stream);
+
 /* Size of the scratch array built into the library for qnn_xnor_gemm_noalloc. */
 #define QNN_NOALLOC_SCRATCH_BYTES (8u << 20)
 
@@ -449,6 +468,25 @@ QNN_API int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, 
                          int L, int32_t *scores_host, int algo, void *ws, size_t ws_bytes,
                          void *stream);
 
+/* The same pass from HOST buffers as one CUDA graph (Algorithm 4 end to end:
+ * input copies, every layer, the copy of the scores back).  _create runs the
+ * pass once, captures a second issue of it on `stream` (which must not be the
+ * default stream) and instantiates the graph; _launch replays it with one
+ * launch, asynchronously on the given stream -- synchronise that stream before
+ * reading scores_host.  The graph refers to x_host, scores_host (both must be
+ * pinned host memory and stay valid), the layers' buffers and ws as they were
+ * at creation: write new inputs into the same x_host buffer between launches.
+ * chunks (1..8): pieces the batch is cut into so that input copies overlap the
+ * previous piece's layers; with the launch overhead gone, 3-4 pays for large
+ * batches.  The handle is a small host object the caller owns; the library
+ * allocates no device memory for it (the CUDA runtime keeps the graph). */
+typedef struct qnn_mlp_graph qnn_mlp_graph;
+QNN_API int qnn_mlp_graph_create(const uint8_t *x_host, int64_t M, int in_bits, const qnn_mlp_layer *layers, int L,
+                                 int32_t *scores_host, int algo, void *ws, size_t ws_bytes, int chunks, void *stream,
+                                 qnn_mlp_graph **out);
+QNN_API int qnn_mlp_graph_launch(qnn_mlp_graph *g, void *stream);
+QNN_API int qnn_mlp_graph_destroy(qnn_mlp_graph *g);
+
 QNN_API size_t qnn_mlp_workspace_bytes(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int algo,
                                int host_io);
 
@@ -583,6 +621,20 @@ QNN_API int qnn_set_kernel_events(void *start, void *stop);
 /* Same, but the events go around the (nth + 1)-th matrix-product kernel this thread launches from now on
  * (nth = 0 is the next one): lets one layer inside qnn_mlp_forward be timed. */
 QNN_API int qnn_set_kernel_events_nth(void *start, void *stop, int nth);
+
+/* Measurement aid (the paper has no counterpart): launches one kernel that
+ * keeps a pipe busy with nothing else in the way -- every SM multiplies one
+ * resident shared-memory tile pair `iters` times with the tensor-core
+ * instruction the product kernels use (128 x 256 x 32 bytes of K, e2m1 with
+ * unit block scales or int8; no loads, no epilogue), or runs Eq. 11's xor /
+ * popc / add on registers.  *ops_host receives the operations one launch
+ * performs (2 per multiply-accumulate; 64 per 32-bit xor/popc/add); the caller
+ * times the launch with its own events.  The product kernels' speed is quoted
+ * against these figures as well as against the library-GEMM proxy. */
+#define QNN_PIPE_TENSOR_FP4 1
+#define QNN_PIPE_TENSOR_I8 2
+#define QNN_PIPE_POPC 3
+QNN_API int qnn_pipe_peak_launch(int pipe, int iters, double *ops_host, void *stream);
 
 /* Number of kernels this library has launched in this process so far (all
  * threads, all streams); a monotonically increasing bookkeeping counter. */

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libqnn.so")
 QNN_OK = 0
 QNN_ERR_INVALID_ARG, QNN_ERR_ALIGNMENT, QNN_ERR_UNSUPPORTED, QNN_ERR_OVERFLOW = 1, 2, 3, 4
 QNN_ERR_WORKSPACE, QNN_ERR_CUDA, QNN_ERR_TIMEOUT = 5, 6, 7
-QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA, QNN_ALGO_TC_FP4 = 0, 1, 2, 3, 4
+QNN_ALGO_AUTO, QNN_ALGO_POPC, QNN_ALGO_TC_I8, QNN_ALGO_B1_MMA, QNN_ALGO_TC_FP4, QNN_ALGO_TC_PACKED = 0, 1, 2, 3, 4, 5
 QNN_FORM_I8, QNN_FORM_FP4 = 1, 2
 QNN_MODE_U01, QNN_MODE_PM1 = 0, 1
 QNN_OP_XNOR_GEMM, QNN_OP_BITPLANE_GEMM, QNN_OP_CONV2D, QNN_OP_MLP = 1, 2, 3, 4
@@ -91,6 +91,8 @@ _SIGS = {
     "qnn_quantize_form_sign_nchw": (i32, [vp, i32, i32, i32, i32, i32, vp, i64, vp]),
     "qnn_quantize_form_kbit": (i32, [vp, i64, i64, i64, i32, ctypes.c_float, ctypes.c_float, i32, i32, vp, i64, vp]),
     "qnn_quantize_form_kbit_t": (i32, [vp, i64, i64, i64, i32, ctypes.c_float, ctypes.c_float, i32, i32, vp, i64, vp]),
+    "qnn_fc_sign_f32_workspace_bytes": (sz, [i64, i64]),
+    "qnn_fc_sign_f32": (i32, [vp, i64, i64, i64, vp, i64, i64, vp, i64, vp, sz, vp]),
     "qnn_tc_form": (i32, [i32, i32, i32, i32, i64]),
     "qnn_tc_row_bytes": (i64, [i64, i32]),
     "qnn_tc_operand_bytes": (sz, [i64, i64, i32]),
@@ -116,12 +118,16 @@ _SIGS = {
     "qnn_convnet_forward": (i32, [vp, i32, i32, i32, ctypes.POINTER(qnn_net_layer), i32, vp, vp, vp, sz, vp]),
     "qnn_mlp_forward": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
     "qnn_mlp_forward_host": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, vp]),
+    "qnn_mlp_graph_create": (i32, [vp, i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, vp, i32, vp, sz, i32, vp, ctypes.POINTER(vp)]),
+    "qnn_mlp_graph_launch": (i32, [vp, vp]),
+    "qnn_mlp_graph_destroy": (i32, [vp]),
     "qnn_mlp_layer_form": (i32, [ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
     "qnn_mlp_workspace_bytes": (sz, [i64, i32, ctypes.POINTER(qnn_mlp_layer), i32, i32, i32]),
     "qnn_workspace_bytes": (sz, [i32, i64, i64, i64, i32, i32, i32]),
     "qnn_select_algo": (i32, [i64, i64, i64, i32, i32, i32, i32]),
     "qnn_device_status": (i32, [vp]),
     "qnn_selftest_wait_timeout": (i32, [vp]),
+    "qnn_pipe_peak_launch": (i32, [i32, i32, ctypes.POINTER(ctypes.c_double), vp]),
     "qnn_launch_count": (ctypes.c_uint64, []),
     "qnn_set_kernel_events": (i32, [vp, vp]),
     "qnn_set_kernel_events_nth": (i32, [vp, vp, i32]),
@@ -266,6 +272,16 @@ def qnn_quantize_form_kbit_t(w, K, N, ldw, bits, lo, hi, mode, form, out, ld_byt
         "qnn_quantize_form_kbit_t")
 
 
+def qnn_fc_sign_f32_workspace_bytes(M, K) -> int:
+    return int(_lib.qnn_fc_sign_f32_workspace_bytes(M, K))
+
+
+def qnn_fc_sign_f32(x, M, K, ldx, w, N, ldw, out, ldo, ws):
+    """out = sign(x) . sign(w) from fp32 activations [M, K] and fp32 weights [K, N], weights read once (small batches)."""
+    wp, wb = _ws(ws)
+    _ck(_lib.qnn_fc_sign_f32(_p(x), M, K, ldx, _p(w), N, ldw, _p(out), ldo, wp, wb, _stream()), "qnn_fc_sign_f32")
+
+
 def tc_operand(data, ld_bytes, form, planes=1, mode=QNN_MODE_PM1) -> qnn_tc_operand:
     return qnn_tc_operand(_p(data), ld_bytes, form, planes, mode)
 
@@ -372,6 +388,33 @@ def qnn_mlp_forward_host(x_host, M, in_bits, layers, scores_host, algo=QNN_ALGO_
     wp, wb = _ws(ws)
     _ck(_lib.qnn_mlp_forward_host(_p(x_host), M, in_bits, layers, len(layers), _p(scores_host), algo, wp, wb,
                                   _stream()), "qnn_mlp_forward_host")
+
+
+class MlpGraph:
+    """One Algorithm-4 pass from pinned host buffers as a CUDA graph (argument marshalling only)."""
+
+    def __init__(self, x_host, M, in_bits, layers, scores_host, algo, ws, chunks=3):
+        wp, wb = _ws(ws)
+        self.handle = vp()
+        self.keep = (x_host, scores_host, layers, ws)
+        self.stream = torch.cuda.Stream()
+        self.stream.wait_stream(torch.cuda.current_stream())
+        _ck(_lib.qnn_mlp_graph_create(_p(x_host), M, in_bits, layers, len(layers), _p(scores_host), algo, wp, wb, chunks,
+                                      self.stream.cuda_stream, ctypes.byref(self.handle)), "qnn_mlp_graph_create")
+
+    def launch(self):
+        _ck(_lib.qnn_mlp_graph_launch(self.handle, _stream()), "qnn_mlp_graph_launch")
+
+    def close(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.qnn_mlp_graph_destroy(self.handle)
+        self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:       # interpreter shutdown: the library may already be gone
+            pass
 
 
 def qnn_logquant_pack_i8(x, rows, K, ldx, emin, emax, out, ld_bytes):
@@ -502,6 +545,16 @@ def qnn_device_status() -> int:
 def qnn_selftest_wait_timeout():
     """Launches the diagnostic kernel whose bounded wait runs out; the next qnn_device_status() reports it once."""
     _ck(_lib.qnn_selftest_wait_timeout(_stream()), "qnn_selftest_wait_timeout")
+
+
+QNN_PIPE_TENSOR_FP4, QNN_PIPE_TENSOR_I8, QNN_PIPE_POPC = 1, 2, 3
+
+
+def qnn_pipe_peak_launch(pipe: int, iters: int) -> float:
+    """Launches the issue-only measurement kernel of `pipe`; returns the operations that launch performs."""
+    ops = ctypes.c_double(0.0)
+    _ck(_lib.qnn_pipe_peak_launch(pipe, iters, ctypes.byref(ops), _stream()), "qnn_pipe_peak_launch")
+    return float(ops.value)
 
 
 def qnn_launch_count() -> int:

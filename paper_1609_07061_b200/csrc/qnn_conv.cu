@@ -219,7 +219,7 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
     const int64_t M = (int64_t)B * Ho * Wo;
     const int64_t kwords = (int64_t)KH * KW * Cw;
     cudaStream_t st = as_stream(stream);
-    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_FP4, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: unknown algo %d", algo);
+    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_PACKED, QNN_ERR_INVALID_ARG, "qnn_binary_conv2d: unknown algo %d", algo);
 
     GemmArgs g{};
     g.b = w; g.ldb = kwords; g.ka = g.kb = 1; g.a_mode = g.b_mode = QNN_MODE_PM1;

@@ -63,7 +63,7 @@ static int forced_algo()
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st)
 {
     if (int rc = validate_gemm(g)) return rc;
-    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_FP4, QNN_ERR_INVALID_ARG, "gemm: unknown algo %d", algo);
+    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_PACKED, QNN_ERR_INVALID_ARG, "gemm: unknown algo %d", algo);
     if (g.M == 0 || g.N == 0) return QNN_OK;
     if (algo == QNN_ALGO_AUTO) {
         algo = forced_algo();
@@ -79,14 +79,18 @@ int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_
             if (!fits || kw == 0) {
                 algo = QNN_ALGO_POPC;
             } else if (need > 0 && (ws == nullptr || !aligned(ws, 256) || ws_bytes < need)) {
-                // the result is the same, the speed is not: leave word of it where the caller can find it
-                note("gemm: QNN_ALGO_AUTO ran the CUDA-core kernel instead of the tensor-core one: it needs a 256-byte "
-                     "aligned workspace of %zu bytes (got %zu at %p)", need, ws_bytes, ws);
-                algo = QNN_ALGO_POPC;
+                // The result is the same, the speed is not: leave word of it where the caller can find it.  Small batches
+                // still run on the tensor cores, straight from the packed planes; the rest on the CUDA cores.
+                const bool packed_ok = g.M <= 1024 && gemm_smallm_supported(g);
+                note("gemm: QNN_ALGO_AUTO ran the %s instead of the tensor-core kernel on rewritten operands: that one needs a "
+                     "256-byte aligned workspace of %zu bytes (got %zu at %p)",
+                     packed_ok ? "tensor-core kernel on packed tiles" : "CUDA-core kernel", need, ws_bytes, ws);
+                algo = packed_ok ? QNN_ALGO_TC_PACKED : QNN_ALGO_POPC;
             }
         }
         if (algo == QNN_ALGO_B1_MMA && !(g.ka == 1 && g.kb == 1)) algo = QNN_ALGO_POPC;
     }
+    if (algo == QNN_ALGO_TC_PACKED) return launch_gemm_smallm(g, st);
     if (algo == QNN_ALGO_POPC || algo == QNN_ALGO_B1_MMA)
         QNN_REQUIRE(g.a && g.b && !g.out_form, QNN_ERR_INVALID_ARG, "gemm: the CUDA-core paths take packed planes and write no form output");
     switch (algo) {

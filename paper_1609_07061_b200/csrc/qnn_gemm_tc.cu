@@ -26,18 +26,13 @@
 #include <atomic>
 #include <cstdlib>
 #include "qnn_internal.cuh"
+#include "qnn_tc_ptx.cuh"
 
 namespace qnn {
 namespace {
 
-constexpr int BM = 128;              // rows of A per tile (UMMA M)
-constexpr int BKB = 128;             // bytes of K per pipeline stage = one 128-byte swizzle row
 constexpr int EPI_GROUPS = 2;        // epilogue warps per quarter of the accumulator's lanes
 constexpr int TC_THREADS = 64 + 128 * EPI_GROUPS;   // warp 0: TMA, warp 1: MMA + TMEM owner, the rest: epilogue
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
-constexpr int SMEM_LIMIT = 232448;   // 227 KB of dynamic shared memory per CTA
-
-__device__ int g_tc_status = 0;      // 0 = fine; otherwise the code of the first wait that ran out
 
 struct TcParams {
     int64_t M, N;
@@ -61,106 +56,6 @@ struct TcParams {
     int64_t corr_ld;                 // row length of the correction table: N rounded up to 32, pad zero
 };
 
-// ---- PTX wrappers -----------------------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the block is aborting (this wait ran out, or another one did).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int code,
-                                          const uint32_t limit = WAIT_LIMIT)
-{
-    for (uint32_t it = 0; it < limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it > 4096) __nanosleep(64);
-        if ((it & 63) == 63 && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    atomicCAS(&g_tc_status, 0, code);
-    return false;
-}
-
-
-// bulk tensor stores (shared -> global); rows / columns past the tensor's extents are clipped by the hardware
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, int32_t y, uint32_t src)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, int32_t x, int32_t y, int32_t z, uint32_t src)
-{
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// waits until the shared-memory side of all but the N most recent store groups has been read
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// CTAS = 1: a CTA works alone.  CTAS = 2: two CTAs of a cluster share 256 x BN tiles (cta_group::2); the same
-// warp of both CTAs allocates / frees.
-template <int CTAS>
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols)
-{
-    if (CTAS == 2) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    } else {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-}
-template <int CTAS>
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    if (CTAS == 2) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// shared::cluster address of the same shared-memory location in CTA `rank` of this cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 // One pipeline stage of the MMA warp as ONE instruction stream: poll the NEXT stage's full barrier, issue the
 // four K steps of this stage (+32 bytes of K = +2 in the descriptors' address field), commit them to this
 // stage's empty barrier, and only then read the poll's result -- the poll's latency hides behind the issue.
@@ -390,44 +285,6 @@ __device__ __forceinline__ uint32_t tma_stage_conv(uint32_t next_empty_bar, uint
           "r"(c3), "r"(dst_b), "l"(map_b), "r"(bx), "r"(by)
         : "memory");
     return ready;
-}
-
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-// this warp's 32 lanes x 8 columns, all set to `val`
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, uint32_t val)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr), "r"(val) : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are KB = 128 (or 64) bytes, swizzled over 128 (64)
-// bytes -- the layout a TMA box of KB bytes x rows produces: 8-row groups are 8*KB bytes apart.
-template <int KB>
-__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t saddr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3ffffu) >> 4);          // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                            // leading-dimension offset (unused with swizzle) = 1
-    d |= (uint64_t)((8 * KB) >> 4) << 32;              // stride between 8-row groups
-    d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
-    d |= (uint64_t)(KB == 128 ? 2 : 4) << 61;          // 128-byte / 64-byte swizzle
-    return d;
 }
 
 // Diagnostic: one CTA waits, with a short limit, on a barrier that nothing ever arrives on.  No copy and no MMA is in
@@ -1069,23 +926,6 @@ __global__ void __launch_bounds__(256) expand_fp4_kernel(const uint32_t *__restr
 
 // ---- tensor maps -------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
 // 2-D byte matrix [rows, row_bytes] with rows ld_bytes apart; box = 128 bytes x box_rows; reads past either extent give 0
 int make_map_2d(CUtensorMap *map, const void *base, int64_t rows, int64_t row_bytes, int64_t ld_bytes, int box_rows, int kblk = BKB)
 {
@@ -1464,10 +1304,16 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
     static const bool pairs_off = [] { const char *e = getenv("QNN_TC_PAIRS"); return e && e[0] == '0'; }();
     const int pairs_resident = pairs_off ? 0 : pairs_resident_on_current_device();
     const int64_t tiles_m2 = ceil_div(g.M, 2 * BM);
-    const bool pairs = !g.conv && pairs_resident >= 8 && p.num_kb >= 12 && tiles_m2 * ceil_div(g.N, 224) >= pairs_resident;
+    static const int pair_min_kb = [] { const char *e = getenv("QNN_TC_PAIR_MIN_KB"); return e ? atoi(e) : 12; }();
+    const bool pairs = !g.conv && pairs_resident >= 8 && p.num_kb >= pair_min_kb && tiles_m2 * ceil_div(g.N, 224) >= pairs_resident;
     if (pairs) {
         p.tiles_m = (int32_t)tiles_m2;
-        const int bn = pick_bn(tiles_m2, g.N, pairs_resident, 64);
+        int bn = pick_bn(tiles_m2, g.N, pairs_resident, 64);
+        if (form == QNN_FORM_I8 && bn == 224) {
+            // (int8 has no scale columns in tensor memory: two 256-column accumulator stages fit)
+            const int64_t w224 = ceil_div(tiles_m2 * ceil_div(g.N, 224), pairs_resident), w256 = ceil_div(tiles_m2 * ceil_div(g.N, 256), pairs_resident);
+            if (w256 * (256 + 900) < w224 * (224 + 900)) bn = 256;
+        }
         if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, bn / 2)) return rc;
         if (form == QNN_FORM_FP4) {
             switch (bn) {
@@ -1478,6 +1324,7 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
             }
         }
         switch (bn) {
+            case 256: return launch_tc_cfg<QNN_FORM_I8, 256, 2>(ma, mb, p, pairs_resident, st);
             case 224: return launch_tc_cfg<QNN_FORM_I8, 224, 2>(ma, mb, p, pairs_resident, st);
             case 192: return launch_tc_cfg<QNN_FORM_I8, 192, 2>(ma, mb, p, pairs_resident, st);
             case 128: return launch_tc_cfg<QNN_FORM_I8, 128, 2>(ma, mb, p, pairs_resident, st);
@@ -1522,6 +1369,130 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
 
 }  // namespace qnn
 
+// ---- issue-only pipe measurements ------------------------------------------------------------------------------
+//
+// What the pipes can do when nothing else is in the way: every CTA multiplies ONE resident shared-memory tile pair
+// over and over (no loads, no epilogue), or runs xor / popc / add on registers.  The bench divides the operations by
+// the device time of such a launch and reports the product kernels against that figure as well.
+namespace qnn {
+namespace {
+
+constexpr int PEAK_N = 256;             // instruction shape of the tensor measurement: 128 x 256 x (32 bytes of K)
+
+template <int FORM>
+__global__ void __launch_bounds__(128, 1) tc_peak_kernel(int iters, uint32_t idesc, int *ok_out)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *gen = smem_raw + (base - raw);
+    constexpr int A_BYTES = BM * BKB, B_BYTES = PEAK_N * BKB;
+    uint64_t *bar = reinterpret_cast<uint64_t *>(gen + A_BYTES + B_BYTES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar + 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5;
+    // operand values: A all +1, B +1 / -1 alternating along K, so that every K step adds zero to the accumulators
+    const uint32_t a_word = FORM == QNN_FORM_FP4 ? 0x22222222u : 0x01010101u;
+    const uint32_t b_word = FORM == QNN_FORM_FP4 ? 0xA2A2A2A2u : 0xFF01FF01u;
+    for (int i = threadIdx.x; i < A_BYTES / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(gen)[i] = a_word;
+    for (int i = threadIdx.x; i < B_BYTES / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(gen + A_BYTES)[i] = b_word;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(bar), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    fence_async_shared();
+    if (warp == 0) tmem_alloc<1>(smem_u32(tmem_slot), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (FORM == QNN_FORM_FP4) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_st8(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(PEAK_N + 8 * c), 0x7f7f7f7fu);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+    if (threadIdx.x == 0) {
+        const uint64_t da = make_kmajor_desc<BKB>(base), db = make_kmajor_desc<BKB>(base + A_BYTES);
+        const uint32_t sf = tmem_base + (uint32_t)PEAK_N;
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const uint64_t a = da + (uint64_t)(2 * ks), b = db + (uint64_t)(2 * ks);
+                const uint32_t acc = (it | ks) != 0;
+                if (FORM == QNN_FORM_FP4)
+                    asm volatile("{\n.reg .pred P;\nsetp.ne.b32 P, %4, 0;\n"
+                                 "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%5], P;\n}\n"
+                                 ::"r"(tmem_base), "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(sf) : "memory");
+                else
+                    asm volatile("{\n.reg .pred P;\nsetp.ne.b32 P, %4, 0;\n"
+                                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, P;\n}\n"
+                                 ::"r"(tmem_base), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+            }
+        }
+        umma_commit(smem_u32(bar));
+        const bool done = mbar_wait(smem_u32(bar), 0, abort_flag, 8);
+        if (blockIdx.x == 0 && ok_out != nullptr) *ok_out = done ? 1 : 0;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0) tmem_dealloc<1>(tmem_base, 512);
+}
+
+// xor, popc, add on registers: eight independent chains per thread (Eq. 11's three instructions, nothing else)
+__global__ void __launch_bounds__(1024) popc_peak_kernel(int iters, uint32_t seed, uint32_t *sink)
+{
+    uint32_t x[8], acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { x[i] = seed * (threadIdx.x + 1) + i * 0x9e3779b9u; acc[i] = 0; }
+    uint32_t y = seed ^ blockIdx.x;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] += __popc(x[i] ^ y);
+        y = y * 1664525u + 1013904223u;
+    }
+    uint32_t t = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t += acc[i];
+    if (t == 0xffffffffu) *sink = t;         // (never true for these counts; keeps the loop alive)
+}
+
+}  // namespace
+}  // namespace qnn
+
+extern "C" int qnn_pipe_peak_launch(int pipe, int iters, double *ops_host, void *stream)
+{
+    using namespace qnn;
+    QNN_REQUIRE(iters >= 1 && iters <= (1 << 20), QNN_ERR_INVALID_ARG, "qnn_pipe_peak_launch: iters must be in 1..2^20");
+    QNN_REQUIRE(ops_host != nullptr, QNN_ERR_INVALID_ARG, "qnn_pipe_peak_launch: ops_host is NULL");
+    cudaStream_t st = as_stream(stream);
+    const int sms = sm_count();
+    if (pipe == QNN_PIPE_POPC) {
+        const int blocks = 2 * sms;
+        popc_peak_kernel<<<blocks, 1024, 0, st>>>(iters, 0x12345u, nullptr);
+        *ops_host = 64.0 * 8.0 * (double)iters * 1024.0 * blocks;          // one 32-bit xor/popc/add = 32 products = 64 operations
+        return check_launch("qnn_pipe_peak_launch");
+    }
+    QNN_REQUIRE(pipe == QNN_PIPE_TENSOR_FP4 || pipe == QNN_PIPE_TENSOR_I8, QNN_ERR_INVALID_ARG, "qnn_pipe_peak_launch: unknown pipe %d", pipe);
+    const size_t smem = (size_t)BM * BKB + (size_t)PEAK_N * BKB + 64 + 1024;
+    const int kstep = pipe == QNN_PIPE_TENSOR_FP4 ? 64 : 32;               // elements of K per instruction (32 bytes)
+    *ops_host = 2.0 * BM * PEAK_N * kstep * 4.0 * (double)iters * sms;
+    if (pipe == QNN_PIPE_TENSOR_FP4) {
+        const uint32_t idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((uint32_t)(BM >> 4) << 24) | ((uint32_t)(PEAK_N >> 3) << 17);
+        QNN_CUDA(cudaFuncSetAttribute(tc_peak_kernel<QNN_FORM_FP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        tc_peak_kernel<QNN_FORM_FP4><<<sms, 128, smem, st>>>(iters, idesc, nullptr);
+    } else {
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24) | ((uint32_t)(PEAK_N >> 3) << 17);
+        QNN_CUDA(cudaFuncSetAttribute(tc_peak_kernel<QNN_FORM_I8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        tc_peak_kernel<QNN_FORM_I8><<<sms, 128, smem, st>>>(iters, idesc, nullptr);
+    }
+    return check_launch("qnn_pipe_peak_launch");
+}
+
 extern "C" int qnn_selftest_wait_timeout(void *stream)
 {
     using namespace qnn;
@@ -1533,12 +1504,12 @@ extern "C" int qnn_device_status(void *stream)
 {
     using namespace qnn;
     QNN_CUDA(cudaStreamSynchronize(as_stream(stream)));
-    int code = 0;
-    QNN_CUDA(cudaMemcpyFromSymbol(&code, g_tc_status, sizeof(int)));
-    if (code != 0) {
-        const int zero = 0;
-        QNN_CUDA(cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int)));
-        return fail(QNN_ERR_TIMEOUT, "a bounded device-side wait ran out (wait site %d)", code);
-    }
+    int code = 0, code_fc = 0, code_sm = 0;
+    QNN_CUDA(status_read_clear(&code));
+    if (int rc = fc_f32_status(&code_fc)) return rc;
+    if (int rc = smallm_status(&code_sm)) return rc;
+    if (code == 0) code = code_fc;
+    if (code == 0) code = code_sm;
+    if (code != 0) return fail(QNN_ERR_TIMEOUT, "a bounded device-side wait ran out (wait site %d)", code);
     return QNN_OK;
 }

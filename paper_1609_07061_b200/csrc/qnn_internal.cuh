@@ -112,6 +112,12 @@ bool conv_prep_layout(int Cout, int C, int KH, int KW, int pad, int want_form, C
 int tc_expand(const uint32_t *src, int planes, int mode, int64_t ld, int64_t plane_stride, int64_t rows, int64_t kwords,
               int64_t pad_period, int pad_tail, int form, uint8_t *dst, int64_t dst_ld, cudaStream_t st);
 int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_t st);
+// Small-batch product straight from packed planes (packed tiles by TMA, expanded in shared memory): no workspace.
+bool gemm_smallm_supported(const GemmArgs &g);
+int launch_gemm_smallm(const GemmArgs &g, cudaStream_t st);
+int smallm_status(int *code);
+// status word of the real-valued-weights layer kernel's bounded waits (its own translation unit): reads and clears it
+int fc_f32_status(int *code);
 
 #ifdef __CUDACC__
 // Programmatic dependent launch.  A kernel launched through launch_pdl may be scheduled while the kernel before it in the

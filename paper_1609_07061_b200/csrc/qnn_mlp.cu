@@ -4,6 +4,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <new>
 #include "qnn_internal.cuh"
 
 namespace qnn {
@@ -44,6 +45,7 @@ int resolve_env_algo()
     if (!strcmp(e, "TC_I8") || !strcmp(e, "2")) return QNN_ALGO_TC_I8;
     if (!strcmp(e, "B1_MMA") || !strcmp(e, "3")) return QNN_ALGO_B1_MMA;
     if (!strcmp(e, "TC_FP4") || !strcmp(e, "4")) return QNN_ALGO_TC_FP4;
+    if (!strcmp(e, "TC_PACKED") || !strcmp(e, "5")) return QNN_ALGO_TC_PACKED;
     return QNN_ALGO_AUTO;
 }
 
@@ -60,6 +62,7 @@ LayerChoice choose_layer(int64_t M, int in_bits, const qnn_mlp_layer *layers, in
     LayerChoice c{algo, 0};
     if (algo == QNN_ALGO_AUTO) c.algo = qnn_select_algo(M, ly.N, ly.K, ka, 1, a_mode, QNN_MODE_PM1);
     if (c.algo == QNN_ALGO_B1_MMA && ka != 1) c.algo = QNN_ALGO_POPC;
+    if (c.algo == QNN_ALGO_TC_PACKED && best_form != QNN_FORM_FP4) c.algo = QNN_ALGO_POPC;     // (more than two planes, or sums beyond 2^24)
     if (c.algo == QNN_ALGO_TC_FP4 && best_form != QNN_FORM_FP4) c.algo = best_form ? QNN_ALGO_TC_I8 : QNN_ALGO_POPC;
     if (c.algo == QNN_ALGO_TC_I8 && !(tc_form_holds(QNN_FORM_I8, ka, a_mode))) c.algo = QNN_ALGO_POPC;
     if (c.algo == QNN_ALGO_TC_FP4) c.form = QNN_FORM_FP4;
@@ -71,7 +74,7 @@ int plan_mlp(int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int alg
 {
     QNN_REQUIRE(layers != nullptr && L >= 1, QNN_ERR_INVALID_ARG, "mlp: need at least one layer");
     QNN_REQUIRE(M >= 0 && in_bits >= 1 && in_bits <= 8, QNN_ERR_INVALID_ARG, "mlp: bad batch or input bit-width");
-    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_FP4, QNN_ERR_INVALID_ARG, "mlp: unknown algo %d", algo);
+    QNN_REQUIRE(algo >= QNN_ALGO_AUTO && algo <= QNN_ALGO_TC_PACKED, QNN_ERR_INVALID_ARG, "mlp: unknown algo %d", algo);
     for (int l = 0; l < L; ++l) {
         QNN_REQUIRE(layers[l].K >= 1 && layers[l].N >= 1 && layers[l].w != nullptr, QNN_ERR_INVALID_ARG,
                     "mlp: layer %d has a bad shape or NULL weights", l);
@@ -215,6 +218,63 @@ cudaStream_t copy_stream()
 }  // namespace
 }  // namespace qnn
 
+namespace qnn {
+namespace {
+
+// One pass from host buffers, queued on `st` (and on the library's copy stream for the overlapped input chunks):
+// input copies, the layers chunk by chunk, the copy of the scores back.  Does not synchronise.  Also runs under
+// stream capture: the copy stream is forked from `st` by an event and joined back by the chunks' events.
+int issue_host_pass(const uint8_t *x_host, int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int32_t *scores_host,
+                    int algo, char *base, const MlpPlan &p, int chunks, cudaStream_t st)
+{
+    uint8_t *x_dev = reinterpret_cast<uint8_t *>(base + p.off_x);
+    int32_t *s_dev = reinterpret_cast<int32_t *>(base + p.off_scores);
+    const int64_t K0 = layers[0].K, NL = layers[L - 1].N;
+    if (chunks > 8) chunks = 8;
+    cudaStream_t cs = chunks > 1 ? copy_stream() : nullptr;
+    if (chunks == 1 || cs == nullptr) {
+        QNN_CUDA(cudaMemcpyAsync(x_dev, x_host, (size_t)M * (size_t)K0, cudaMemcpyHostToDevice, st));
+        if (int rc = run_mlp(x_dev, M, in_bits, layers, L, s_dev, algo, base, p, st)) return rc;
+    } else {
+        const int64_t rows_c = (int64_t)round_up((size_t)ceil_div(M, chunks), 256);   // whole 256-row tiles per chunk
+        cudaEvent_t ev[9] = {};
+        int rc = QNN_OK;
+        for (int c = 0; c <= chunks && rc == QNN_OK; ++c)
+            if (cudaEventCreateWithFlags(&ev[c], cudaEventDisableTiming) != cudaSuccess) rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: cudaEventCreate failed");
+        if (rc == QNN_OK) {
+            // the copies start after whatever the caller already queued on its stream
+            if (cudaEventRecord(ev[chunks], st) != cudaSuccess || cudaStreamWaitEvent(cs, ev[chunks], 0) != cudaSuccess)
+                rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: stream ordering failed");
+        }
+        for (int c = 0; c < chunks && rc == QNN_OK; ++c) {
+            const int64_t r0 = c * rows_c, rows = (r0 + rows_c <= M ? rows_c : M - r0);
+            if (rows <= 0) break;
+            if (cudaMemcpyAsync(x_dev + r0 * K0, x_host + r0 * K0, (size_t)rows * (size_t)K0, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+                cudaEventRecord(ev[c], cs) != cudaSuccess)
+                rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: chunk copy failed");
+        }
+        for (int c = 0; c < chunks && rc == QNN_OK; ++c) {
+            const int64_t r0 = c * rows_c, rows = (r0 + rows_c <= M ? rows_c : M - r0);
+            if (rows <= 0) break;
+            if (cudaStreamWaitEvent(st, ev[c], 0) != cudaSuccess) { rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: stream wait failed"); break; }
+            rc = run_mlp(x_dev + r0 * K0, rows, in_bits, layers, L, s_dev + r0 * NL, algo, base, p, st);
+        }
+        if (rc != QNN_OK) {
+            cudaStreamSynchronize(cs);
+            cudaStreamSynchronize(st);
+        }
+        // (events may be destroyed while work that uses them is pending: the runtime frees them when it is done)
+        for (int c = 0; c <= chunks; ++c)
+            if (ev[c]) cudaEventDestroy(ev[c]);
+        if (rc != QNN_OK) return rc;
+    }
+    QNN_CUDA(cudaMemcpyAsync(scores_host, s_dev, sizeof(int32_t) * (size_t)M * (size_t)NL, cudaMemcpyDeviceToHost, st));
+    return QNN_OK;
+}
+
+}  // namespace
+}  // namespace qnn
+
 using namespace qnn;
 
 extern "C" {
@@ -255,52 +315,78 @@ int qnn_mlp_forward_host(const uint8_t *x_host, int64_t M, int in_bits, const qn
                 "qnn_mlp_forward_host: workspace of at least %zu bytes (256-byte aligned) required", p.total);
     cudaStream_t st = as_stream(stream);
     char *base = static_cast<char *>(ws);
-    uint8_t *x_dev = reinterpret_cast<uint8_t *>(base + p.off_x);
-    int32_t *s_dev = reinterpret_cast<int32_t *>(base + p.off_scores);
-    const int64_t K0 = layers[0].K, NL = layers[L - 1].N;
 
     // Batch rows are independent, so the batch is cut into chunks whose host-to-device copies (on a copy stream
     // of the library's own) run while the previous chunk is being computed on the caller's stream.
-    const int chunks = M >= 4096 ? 2 : 1;      // (more chunks cost more in launches than they hide in copies)
-    cudaStream_t cs = chunks > 1 ? copy_stream() : nullptr;
-    if (chunks == 1 || cs == nullptr) {
-        QNN_CUDA(cudaMemcpyAsync(x_dev, x_host, (size_t)M * (size_t)K0, cudaMemcpyHostToDevice, st));
-        if (int rc = run_mlp(x_dev, M, in_bits, layers, L, s_dev, algo, base, p, st)) return rc;
-    } else {
-        const int64_t rows_c = (int64_t)round_up((size_t)ceil_div(M, chunks), 256);   // whole 256-row tiles per chunk
-        cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-        int rc = QNN_OK;
-        for (int c = 0; c <= chunks && rc == QNN_OK; ++c)
-            if (cudaEventCreateWithFlags(&ev[c], cudaEventDisableTiming) != cudaSuccess) rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: cudaEventCreate failed");
-        if (rc == QNN_OK) {
-            // the copies start after whatever the caller already queued on its stream
-            if (cudaEventRecord(ev[chunks], st) != cudaSuccess || cudaStreamWaitEvent(cs, ev[chunks], 0) != cudaSuccess)
-                rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: stream ordering failed");
-        }
-        for (int c = 0; c < chunks && rc == QNN_OK; ++c) {
-            const int64_t r0 = c * rows_c, rows = (r0 + rows_c <= M ? rows_c : M - r0);
-            if (rows <= 0) break;
-            if (cudaMemcpyAsync(x_dev + r0 * K0, x_host + r0 * K0, (size_t)rows * (size_t)K0, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
-                cudaEventRecord(ev[c], cs) != cudaSuccess)
-                rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: chunk copy failed");
-        }
-        for (int c = 0; c < chunks && rc == QNN_OK; ++c) {
-            const int64_t r0 = c * rows_c, rows = (r0 + rows_c <= M ? rows_c : M - r0);
-            if (rows <= 0) break;
-            if (cudaStreamWaitEvent(st, ev[c], 0) != cudaSuccess) { rc = fail(QNN_ERR_CUDA, "qnn_mlp_forward_host: stream wait failed"); break; }
-            rc = run_mlp(x_dev + r0 * K0, rows, in_bits, layers, L, s_dev + r0 * NL, algo, base, p, st);
-        }
-        if (rc != QNN_OK) {
-            cudaStreamSynchronize(cs);
-            cudaStreamSynchronize(st);
-        }
-        // (events may be destroyed while work that uses them is pending: the runtime frees them when it is done)
-        for (int c = 0; c <= chunks; ++c)
-            if (ev[c]) cudaEventDestroy(ev[c]);
-        if (rc != QNN_OK) return rc;
-    }
-    QNN_CUDA(cudaMemcpyAsync(scores_host, s_dev, sizeof(int32_t) * (size_t)M * (size_t)NL, cudaMemcpyDeviceToHost, st));
+    const int chunks = M >= 4096 ? 2 : 1;      // (issued call by call, more chunks cost more in launches than they hide in copies)
+    if (int rc = issue_host_pass(x_host, M, in_bits, layers, L, scores_host, algo, base, p, chunks, st)) return rc;
     QNN_CUDA(cudaStreamSynchronize(st));
+    return QNN_OK;
+}
+
+}  // extern "C"
+
+// A whole pass from host buffers as ONE CUDA graph: built once (stream capture of the same calls
+// qnn_mlp_forward_host issues), replayed with a single launch per pass.
+struct qnn_mlp_graph {
+    cudaGraphExec_t exec;
+    int device;
+};
+
+extern "C" {
+
+int qnn_mlp_graph_create(const uint8_t *x_host, int64_t M, int in_bits, const qnn_mlp_layer *layers, int L, int32_t *scores_host,
+                         int algo, void *ws, size_t ws_bytes, int chunks, void *stream, qnn_mlp_graph **out)
+{
+    QNN_REQUIRE(out != nullptr, QNN_ERR_INVALID_ARG, "qnn_mlp_graph_create: out is NULL");
+    *out = nullptr;
+    MlpPlan p;
+    if (int rc = plan_mlp(M, in_bits, layers, L, algo, 1, &p)) return rc;
+    QNN_REQUIRE(M >= 1, QNN_ERR_INVALID_ARG, "qnn_mlp_graph_create: empty batch");
+    QNN_REQUIRE(x_host && scores_host, QNN_ERR_INVALID_ARG, "qnn_mlp_graph_create: NULL input or output");
+    QNN_REQUIRE(chunks >= 1 && chunks <= 8, QNN_ERR_INVALID_ARG, "qnn_mlp_graph_create: chunks must be in 1..8");
+    QNN_REQUIRE(ws && aligned(ws, 256) && ws_bytes >= p.total, QNN_ERR_WORKSPACE,
+                "qnn_mlp_graph_create: workspace of at least %zu bytes (256-byte aligned) required", p.total);
+    cudaStream_t st = as_stream(stream);
+    QNN_REQUIRE(st != nullptr, QNN_ERR_INVALID_ARG, "qnn_mlp_graph_create: a stream other than the default stream is required for capture");
+    char *base = static_cast<char *>(ws);
+    // one eager pass first: one-time kernel attributes are set outside the capture, and argument errors surface here
+    if (int rc = issue_host_pass(x_host, M, in_bits, layers, L, scores_host, algo, base, p, chunks, st)) return rc;
+    QNN_CUDA(cudaStreamSynchronize(st));
+    QNN_CUDA(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    const int rc = issue_host_pass(x_host, M, in_bits, layers, L, scores_host, algo, base, p, chunks, st);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+    if (rc != QNN_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return rc;
+    }
+    if (ce != cudaSuccess || graph == nullptr) return fail(QNN_ERR_CUDA, "qnn_mlp_graph_create: stream capture failed: %s", cudaGetErrorString(ce));
+    cudaGraphExec_t exec = nullptr;
+    const cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess) return fail(QNN_ERR_CUDA, "qnn_mlp_graph_create: cudaGraphInstantiate failed: %s", cudaGetErrorString(ie));
+    qnn_mlp_graph *g = new (std::nothrow) qnn_mlp_graph;
+    if (g == nullptr) { cudaGraphExecDestroy(exec); return fail(QNN_ERR_CUDA, "qnn_mlp_graph_create: out of host memory"); }
+    g->exec = exec;
+    g->device = 0;
+    cudaGetDevice(&g->device);
+    *out = g;
+    return QNN_OK;
+}
+
+int qnn_mlp_graph_launch(qnn_mlp_graph *g, void *stream)
+{
+    QNN_REQUIRE(g != nullptr && g->exec != nullptr, QNN_ERR_INVALID_ARG, "qnn_mlp_graph_launch: NULL graph");
+    QNN_CUDA(cudaGraphLaunch(g->exec, as_stream(stream)));
+    return QNN_OK;
+}
+
+int qnn_mlp_graph_destroy(qnn_mlp_graph *g)
+{
+    if (g == nullptr) return QNN_OK;
+    if (g->exec) cudaGraphExecDestroy(g->exec);
+    delete g;
     return QNN_OK;
 }
 

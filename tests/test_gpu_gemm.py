@@ -17,7 +17,7 @@ def q():
 
 
 def _algos(q):
-    return [q.QNN_ALGO_POPC, q.QNN_ALGO_B1_MMA, q.QNN_ALGO_TC_I8, q.QNN_ALGO_AUTO, q.QNN_ALGO_TC_FP4]
+    return [q.QNN_ALGO_POPC, q.QNN_ALGO_B1_MMA, q.QNN_ALGO_TC_I8, q.QNN_ALGO_AUTO, q.QNN_ALGO_TC_FP4, q.QNN_ALGO_TC_PACKED]
 
 
 def _ws(q, op, M, N, K, ka=1, kb=1, algo=0):
@@ -216,3 +216,86 @@ def test_padding_invariance(q):
         out = torch.empty(M, N, dtype=torch.int32, device="cuda")
         q.qnn_xnor_gemm(as_i32_words(a).cuda(), ld, as_i32_words(b).cuda(), ld, M, N, K, out, N, q.QNN_ALGO_POPC)
         np.testing.assert_array_equal(out.cpu().numpy(), want)
+
+
+# ---- QNN_ALGO_TC_PACKED: the tensor-core product straight from packed tiles (no workspace) ---------------------------
+
+def _ld4(K):
+    return (words_per_row(K) + 3) // 4 * 4          # rows TMA can address: a multiple of 16 bytes apart
+
+
+@pytest.mark.parametrize("ka,a_mode,kb,b_mode", [(1, 1, 1, 1), (2, 0, 1, 1), (2, 1, 1, 1), (1, 0, 1, 1), (2, 0, 2, 1), (1, 1, 2, 0)])
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (5, 7, 31), (100, 130, 1000), (128, 32, 256), (129, 33, 257), (300, 70, 2048), (37, 257, 2049),
+                                   (64, 96, 4500)])
+def test_tc_packed_bitplane_products(q, ka, a_mode, kb, b_mode, M, N, K):
+    """Packed planes in, int32 out, nothing in between: ragged M / N / K, several row tiles, more than one packed tile along
+    K (2048 elements each), one- and two-plane operands in both value modes; every output against the oracle."""
+    rng = np.random.default_rng(ka * 100 + kb * 10 + a_mode + M + N + K)
+    qa = rng.integers(0, 1 << ka, (M, K)).astype(np.int32)
+    qb = rng.integers(0, 1 << kb, (K, N)).astype(np.int32)
+    ld = _ld4(K) + 4
+    ap = _planes_ref(qa, ka, ld)
+    bp = _planes_ref(qb.T, kb, ld)
+    out = Guarded((M, N + 1), torch.int32, fill=-7)
+    q.qnn_bitplane_gemm(as_i32_words(ap).cuda(), ka, a_mode, ld, M * ld, as_i32_words(bp).cuda(), kb, b_mode, ld, N * ld, M, N, K,
+                        out.t, N + 1, q.QNN_ALGO_TC_PACKED, None)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    got = out.t.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :N], oracle.int_gemm(_values(qa, ka, a_mode), _values(qb, kb, b_mode)))
+    assert (got[:, N:] == -7).all()
+    out.check()
+
+
+@pytest.mark.parametrize("M,N,K", [(100, 4096, 4096), (130, 300, 1000), (3, 40, 96)])
+def test_tc_packed_threshold_bits(q, M, N, K):
+    """Thresholded bits out of the packed-tile kernel, with exact equalities planted and flips."""
+    rng = np.random.default_rng(M + N + K)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    W = rng.uniform(-1, 1, (K, N)).astype(np.float32)
+    s = oracle.xnor_gemm(X, W)
+    T = rng.integers(-40, 41, N).astype(np.int32)
+    T[::3] = s[M // 2, ::3]
+    flip = rng.integers(0, 2, N).astype(np.uint8)
+    ld = _ld4(K)
+    a = as_i32_words(pack_bits_ref((X >= 0).astype(np.uint8), ld)).cuda()
+    b = as_i32_words(pack_bits_ref((W >= 0).astype(np.uint8).T, ld)).cuda()
+    ldw = words_per_row(N) + 1
+    bits = Guarded((M, ldw), torch.int32, fill=0x77777777)
+    q.qnn_xnor_gemm_threshold(a, ld, b, ld, M, N, K, dev(T), dev(flip), bits.t, ldw, q.QNN_ALGO_TC_PACKED, None)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    np.testing.assert_array_equal(unpack_words(words_np(bits.t), N), oracle.threshold(s, T, flip))
+    assert (words_np(bits.t)[:, words_per_row(N):] == 0x77777777).all()
+    bits.check()
+
+
+def test_tc_packed_refuses_what_it_cannot_run(q):
+    fake = torch.zeros(4096, dtype=torch.int32, device="cuda")
+    out = torch.zeros(64, dtype=torch.int32, device="cuda")
+    with pytest.raises(q.QnnError) as e:           # rows 20 bytes apart: not addressable by TMA
+        q.qnn_xnor_gemm(fake, 5, fake, 5, 8, 8, 160, out, 8, q.QNN_ALGO_TC_PACKED, None)
+    assert e.value.status == q.QNN_ERR_UNSUPPORTED
+    with pytest.raises(q.QnnError) as e:           # 4 planes do not fit e2m1
+        q.qnn_bitplane_gemm(fake, 4, 1, 8, 64, fake, 1, 1, 8, 0, 8, 8, 256, out, 8, q.QNN_ALGO_TC_PACKED, None)
+    assert e.value.status == q.QNN_ERR_UNSUPPORTED
+
+
+def test_auto_without_workspace_stays_on_the_tensor_cores_for_small_batches(q):
+    """QNN_ALGO_AUTO with no workspace: small batches take the packed-tile kernel (and say so), bit-exact."""
+    wl = workloads.fc_single()
+    X, W = wl.X.numpy(), wl.W.numpy()
+    M, K = X.shape
+    N = W.shape[1]
+    ld = K // 32
+    a = as_i32_words(pack_bits_ref((X >= 0).astype(np.uint8), ld)).cuda()
+    b = as_i32_words(pack_bits_ref((W >= 0).astype(np.uint8).T, ld)).cuda()
+    out = Guarded((M, N), torch.int32, fill=-7)
+    before = q.qnn_launch_count()
+    q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, out.t, N, q.QNN_ALGO_AUTO, None)
+    assert q.qnn_launch_count() == before + 1          # one launch, nothing rewritten
+    assert "packed tiles" in q.qnn_last_error()
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0
+    np.testing.assert_array_equal(out.t.cpu().numpy(), oracle.xnor_gemm(X, W))
+    out.check()

@@ -395,3 +395,68 @@ def test_conv2d_prepared_chain_two_layers(q):
     torch.cuda.synchronize()
     assert q.qnn_device_status() == 0
     np.testing.assert_array_equal(out.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("M,K,N,ldx,ldw", [(100, 4096, 4096, 4096, 4096), (1, 1, 1, 1, 1), (5, 31, 7, 33, 9), (37, 300, 130, 300, 132),
+                                           (128, 256, 32, 256, 32), (129, 1000, 257, 1000, 260), (64, 513, 96, 516, 97), (300, 2048, 1000, 2048, 1000)])
+def test_fc_sign_f32_weights_read_once(q, M, K, N, ldx, ldw):
+    """The small-batch layer straight from fp32 activations and fp32 weights (config 1's shape first; then ragged M, N, K,
+    unaligned leading dimensions, several row tiles): every output against the oracle's sign-then-multiply."""
+    if (M, K, N) == (100, 4096, 4096):
+        wl = workloads.fc_single()
+        X, W = wl.X.numpy(), wl.W.numpy()
+    else:
+        rng = np.random.default_rng(M * 3 + K * 5 + N)
+        X = rng.standard_normal((M, ldx)).astype(np.float32)
+        W = rng.uniform(-1, 1, (K, ldw)).astype(np.float32)
+        sp = np.array([0.0, -0.0, np.nan, np.inf, -np.inf, 1e-45, -1e-45], np.float32)
+        W.reshape(-1)[:min(W.size, sp.size)] = sp[:min(W.size, sp.size)]
+        X.reshape(-1)[:min(X.size, sp.size)] = sp[::-1][:min(X.size, sp.size)]
+    out = Guarded((M, N + 3), torch.int32, fill=-7)
+    ws = torch.empty(q.qnn_fc_sign_f32_workspace_bytes(M, K), dtype=torch.uint8, device="cuda")
+    q.qnn_fc_sign_f32(dev(X), M, K, X.shape[1], dev(W), N, W.shape[1], out.t, N + 3, ws)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    got = out.t.cpu().numpy()
+    np.testing.assert_array_equal(got[:, :N], oracle.xnor_gemm(X[:, :K], W[:, :N]))
+    assert (got[:, N:] == -7).all()
+    out.check()
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_fc_sign_f32(dev(X), M, K, X.shape[1], dev(W), N, W.shape[1], out.t, N + 3, None)
+    assert e.value.status == q.QNN_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("M,dims,chunks", [(2100, (784, 1024, 1024, 10), 3), (300, (784, 512, 256, 10), 1), (5000, (784, 1024, 1024, 10), 4)])
+def test_mlp_graph_from_host_buffers(q, M, dims, chunks):
+    """The end-to-end pass (pinned host input -> scores in pinned host memory) as one CUDA graph: every replay, also
+    with new inputs written into the same host buffer, must give the oracle's Algorithm-4 scores."""
+    wl = workloads.mnist_mlp(M=M, dims=dims, seed=1)
+    packed, ldws = [], []
+    for W in wl.Ws:
+        K, N = W.shape
+        ld = (words_per_row(K) + 3) // 4 * 4
+        o = torch.zeros(N, ld, dtype=torch.int32, device="cuda")
+        q.qnn_quantize_pack_sign_t(W.cuda(), K, N, N, o, ld)
+        packed.append(o); ldws.append(ld)
+    thr = [t.cuda() for t in wl.Ts]
+    layers = q.make_mlp_layers(packed, ldws, dims[:-1], dims[1:], thr, [None] * len(thr))
+    keep = q.prepack_mlp_weights(layers, packed, 8)                                   # noqa: F841
+    ws = torch.empty(q.qnn_mlp_workspace_bytes(M, 8, layers, q.QNN_ALGO_AUTO, 1), dtype=torch.uint8, device="cuda")
+    xh = wl.X.contiguous().pin_memory()
+    sh = torch.full((M, dims[-1]), -7, dtype=torch.int32).pin_memory()
+    g = q.MlpGraph(xh, M, 8, layers, sh, q.QNN_ALGO_AUTO, ws, chunks=chunks)
+    Ws = [oracle.sign(w.numpy()) for w in wl.Ws]
+    Ts = [t.numpy() for t in wl.Ts]
+    want = oracle.mlp_forward(wl.X.numpy().astype(np.int32), Ws, Ts)
+    for _ in range(2):
+        sh.fill_(-7)
+        g.launch()
+        torch.cuda.synchronize()
+        assert q.qnn_device_status() == 0, q.qnn_last_error()
+        np.testing.assert_array_equal(sh.numpy(), want)
+    # new inputs through the same host buffer
+    x2 = workloads.mnist_mlp(M=M, dims=dims, seed=1, stream=1).X
+    xh.copy_(x2)
+    g.launch()
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(sh.numpy(), oracle.mlp_forward(x2.numpy().astype(np.int32), Ws, Ts))

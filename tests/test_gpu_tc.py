@@ -354,7 +354,7 @@ def test_bounded_wait_that_runs_out_is_reported_once_and_leaves_the_context_usab
 
 
 def test_auto_leaves_a_note_when_it_cannot_use_the_workspace(q):
-    """QNN_ALGO_AUTO with no (or a misaligned) workspace still gives the right integers on the CUDA-core kernel, and says so."""
+    """QNN_ALGO_AUTO with no (or a misaligned) workspace still gives the right integers on another kernel, and says so."""
     M, N, K = 300, 4096, 4096
     assert q.qnn_select_algo(M, N, K) in (q.QNN_ALGO_TC_FP4, q.QNN_ALGO_TC_I8)
     g = torch.Generator(device="cuda").manual_seed(1)
@@ -369,6 +369,6 @@ def test_auto_leaves_a_note_when_it_cannot_use_the_workspace(q):
     for ws in (None, raw[off + 16: off + 16 + need]):
         got = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
         q.qnn_xnor_gemm(a, ld, b, ld, M, N, K, got, N, q.QNN_ALGO_AUTO, ws)
-        assert "CUDA-core kernel instead" in q.qnn_last_error()
+        assert "instead of the tensor-core kernel on rewritten operands" in q.qnn_last_error()
         torch.cuda.synchronize()
         assert torch.equal(got, want)
