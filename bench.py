@@ -394,7 +394,8 @@ def algo_matrix(q, flush):
         rows.append(r)
 
     g = torch.Generator(device="cuda").manual_seed(4)
-    for (M, N, K) in ((100, 4096, 4096), (1024, 1024, 1024), (4096, 4096, 4096), (8192, 8192, 8192)):
+    for (M, N, K) in ((64, 256, 1024), (128, 256, 1024), (128, 512, 2048), (256, 1024, 1024), (512, 1024, 2048), (100, 4096, 4096),
+                      (1024, 1024, 1024), (4096, 4096, 4096), (8192, 8192, 8192)):
         ld = K // 32
         a = torch.randint(-2**31, 2**31 - 1, (M, ld), dtype=torch.int32, device="cuda", generator=g)
         b = torch.randint(-2**31, 2**31 - 1, (N, ld), dtype=torch.int32, device="cuda", generator=g)
@@ -495,6 +496,25 @@ def run_extras(q, bench, peaks, algo):
     ms, best = _time_op(lambda: q.qnn_fc_sign_f32(Xd, M, K, K, Wd, N, N, out, N, wsf), flush)
     rec("c1_layer_cold_weights_one_pass", ms, best, bytes_=(M * K + K * N) * 4.0 + M * N * 4, ops=2.0 * M * N * K,
         note="qnn_fc_sign_f32: weights read once as fp32, nothing packed written; bytes = fp32 inputs + int32 output")
+
+    # ... and 40 such passes back to back on four copies of the weights (268 MB, more than twice the L2: every pass reads
+    # its weights from HBM) -- what the kernel sustains once the launch and the quantiser before it overlap the previous pass
+    Wcopies = [Wd] + [Wd.clone() for _ in range(3)]
+
+    def cold_many():
+        for i in range(40):
+            q.qnn_fc_sign_f32(Xd, M, K, K, Wcopies[i % 4], N, N, out, N, wsf)
+    cold_many()
+    torch.cuda.synchronize()
+    tsm = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); cold_many(); e1.record()
+        e1.synchronize()
+        tsm.append(e0.elapsed_time(e1) / 40)
+    rec("c1_layer_cold_weights_one_pass_x40_back_to_back", statistics.median(tsm), min(tsm), bytes_=(M * K + K * N) * 4.0 + M * N * 4,
+        ops=2.0 * M * N * K, note="per pass; 40 passes in a row, weights rotating over four copies (268 MB) so that each pass reads them from HBM")
+    del Wcopies
 
     # Items whose roofline time is below a few microseconds cannot approach it in a single launch (a launch alone costs
     # 3-5 us): the same calls 100 times back to back inside one CUDA graph show what is left without the launch latency.

@@ -230,11 +230,11 @@ int qnn_binary_conv2d(const uint32_t *x, int B, int C, int H, int W, const uint3
 
     // ---- implicit GEMM on the tensor cores: no im2col matrix ------------------------------------
     ConvPrep lay{};
-    bool implicit = stride == 1 && W <= 128 && algo != QNN_ALGO_POPC && algo != QNN_ALGO_B1_MMA &&
+    bool implicit = stride == 1 && W <= 128 && algo != QNN_ALGO_POPC && algo != QNN_ALGO_B1_MMA && algo != QNN_ALGO_TC_PACKED &&
                     conv_prep_layout(Cout, C, KH, KW, pad, algo == QNN_ALGO_TC_I8 ? QNN_FORM_I8 : (algo == QNN_ALGO_TC_FP4 ? QNN_FORM_FP4 : 0), &lay);
     if (implicit && algo == QNN_ALGO_AUTO) {
         const int pick = qnn_select_algo(M, Cout, g.K, 1, 1, QNN_MODE_PM1, QNN_MODE_PM1);
-        implicit = pick == QNN_ALGO_TC_FP4 || pick == QNN_ALGO_TC_I8;
+        implicit = pick == QNN_ALGO_TC_FP4 || pick == QNN_ALGO_TC_I8 || pick == QNN_ALGO_TC_PACKED;
     }
     if (implicit) {
         const int64_t cbytes = tc_row_bytes(Cw, lay.form);

@@ -10,7 +10,7 @@
 //   warp 0        TMA: A tiles (128 rows x 128 bytes of K per stage)
 //   warp 1        tcgen05.mma issue, tensor-memory owner
 //   warps 2..5    epilogue: tcgen05.ld -> int32 rows
-//   warps 6..13   converters: fp32 weights -> e2m1 B tile (32 output units x 256 k per stage)
+//   warps 6..     converters (16 warps; 8 on the register path): fp32 weights -> e2m1 B tile (32 output units x 256 k per stage)
 //
 // Every device-side wait is bounded (status word, clean exit), as in the product kernel.
 #include <atomic>
@@ -22,8 +22,9 @@ namespace {
 
 constexpr int FC_BN = 32;                      // output units per CTA
 constexpr int FC_KB = 256;                     // k per pipeline stage (128 bytes of e2m1)
-constexpr int FC_CONV_WARPS = 8;
-constexpr int FC_THREADS = 32 * (6 + FC_CONV_WARPS);
+// converter warps: 16 when the weights arrive as TMA tiles (four k per thread; the kernel is bound by the converters'
+// instruction stream, and twice the warps hide twice the latency), 8 on the register path (eight k per thread)
+constexpr int fc_threads(int cw) { return 32 * (6 + cw); }
 constexpr int FC_A_BYTES = BM * BKB;           // 16 KB
 constexpr int FC_B_BYTES = FC_BN * BKB;        // 4 KB
 constexpr int FC_STAGE_BYTES = FC_A_BYTES + FC_B_BYTES;
@@ -46,7 +47,8 @@ struct FcParams {
 
 __device__ __forceinline__ uint32_t sign_nibble(float v) { return v >= 0.0f ? 0x2u : 0xAu; }   // +1 / -1 as e2m1
 
-__global__ void __launch_bounds__(FC_THREADS, 1)
+template <int CW, bool WTMA>
+__global__ void __launch_bounds__(fc_threads(CW), 1)
 fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w, const FcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -71,9 +73,9 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
 
     if (threadIdx.x == 0) {
         // a stage is full when the TMA bytes have landed AND every converter warp has written its part
-        for (int s = 0; s < FC_STAGES; ++s) { mbar_init(full_bar(s), 1 + FC_CONV_WARPS); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < FC_STAGES; ++s) { mbar_init(full_bar(s), 1 + CW); mbar_init(empty_bar(s), 1); }
         mbar_init(tfull_bar, 1);
-        for (int s = 0; s < FC_W_STAGES; ++s) { mbar_init(wfull_bar(s), 1); mbar_init(wempty_bar(s), FC_CONV_WARPS); }
+        for (int s = 0; s < FC_W_STAGES; ++s) { mbar_init(wfull_bar(s), 1); mbar_init(wempty_bar(s), CW); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -118,7 +120,7 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 return true;
             };
             bool ok = true;
-            if (p.w_tma)
+            if (WTMA)
                 while (ok && wkb < p.num_kb && wkb < FC_W_STAGES) ok = issue_w();
             griddep_wait();
             int stage = 0; uint32_t phase = 0;
@@ -130,7 +132,7 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                     ::"r"(full_bar(stage)), "r"((uint32_t)FC_A_BYTES), "r"(base + (uint32_t)(stage * FC_STAGE_BYTES)), "l"(&tmap_a),
                       "r"(kb * BKB), "r"(m0) : "memory");
                 if (++stage == FC_STAGES) { stage = 0; phase ^= 1u; }
-                if (p.w_tma && wkb < p.num_kb) ok = issue_w();
+                if (WTMA && wkb < p.num_kb) ok = issue_w();
             }
         }
     } else if (warp == 1) {
@@ -190,8 +192,9 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             }
         }
     } else {
-        // ---- converters: thread (cw, lane) owns columns n0 + 4*(lane & 7) .. +3 and the eight k of group
+        // ---- converters: thread (cw, lane) owns columns n0 + 4*(lane & 7) .. +3 and the KPT consecutive k of group
         // kq = cw*4 + (lane >> 3) in every K block; a warp's load of one k row set is 4 rows x 128 contiguous bytes.
+        constexpr int KPT = FC_KB / (4 * CW);                    // k per thread and block: 8 or 4
         const int cw = warp - 6;
         const int n4 = lane & 7;
         const int kq = cw * 4 + (lane >> 3);
@@ -199,18 +202,32 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         const bool cols_ok = ncol + 4 <= p.N;
         int stage = 0; uint32_t phase = 0;
         const bool ragged_cols = n0 + FC_BN > p.N;
-        // eight k x four columns of fp32 weights -> four 32-bit words of e2m1 nibbles; what lies outside the matrix -> 0
-        auto convert = [&](const float4 (&t)[8], int32_t kb, uint32_t (&wv)[4]) {
-            wv[0] = wv[1] = wv[2] = wv[3] = 0u;
-            const bool ragged = ragged_cols || ((int64_t)(kb + 1) * FC_KB > p.K);
+        // KPT k x four columns of fp32 weights -> four words of KPT e2m1 nibbles; what lies outside the matrix -> 0
+        auto convert = [&](const float4 (&t)[KPT], int32_t kb, uint32_t (&wv)[4]) {
+            const bool ragged = ragged_cols || ((int64_t)(kb + 1) * FC_KB > p.K);       // (uniform over the CTA)
+            if (!ragged) {
+                // the common case, kept free of any index test: a compare, a select and a shifted OR per element
+                // (0xA = -1, flipped to 0x2 = +1 where x >= 0)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+                for (int c = 0; c < 4; ++c) wv[c] = KPT == 8 ? 0xAAAAAAAAu : 0xAAAAu;
+#pragma unroll
+                for (int j = 0; j < KPT; ++j) {
+                    wv[0] ^= (t[j].x >= 0.0f ? 8u : 0u) << (4 * j);
+                    wv[1] ^= (t[j].y >= 0.0f ? 8u : 0u) << (4 * j);
+                    wv[2] ^= (t[j].z >= 0.0f ? 8u : 0u) << (4 * j);
+                    wv[3] ^= (t[j].w >= 0.0f ? 8u : 0u) << (4 * j);
+                }
+                return;
+            }
+            wv[0] = wv[1] = wv[2] = wv[3] = 0u;
+#pragma unroll
+            for (int j = 0; j < KPT; ++j) {
                 const float e[4] = {t[j].x, t[j].y, t[j].z, t[j].w};
-                const bool k_in = !ragged || ((int64_t)kb * FC_KB + kq * 8 + j < p.K);
+                const bool k_in = (int64_t)kb * FC_KB + kq * KPT + j < p.K;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t nib = sign_nibble(e[c]);
-                    if (ragged && !(k_in && ncol + c < p.N)) nib = 0u;
+                    if (!(k_in && ncol + c < p.N)) nib = 0u;
                     wv[c] |= nib << (4 * j);
                 }
             }
@@ -223,9 +240,11 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int row = 4 * n4 + c;
-                // 128-byte swizzle: 16-byte chunk index XOR (row mod 8); this thread's 4 bytes sit at byte kq*4 of the row
-                const int chunk = (kq >> 2) ^ (row & 7);
-                *reinterpret_cast<uint32_t *>(bt + row * 128 + chunk * 16 + (kq & 3) * 4) = wv[c];
+                // 128-byte swizzle: 16-byte chunk index XOR (row mod 8); this thread's KPT/2 bytes sit at byte kq*KPT/2 of the row
+                const int off = kq * (KPT / 2);
+                uint8_t *dstp = bt + row * 128 + (((off >> 4) ^ (row & 7)) << 4) + (off & 15);
+                if (KPT == 8) *reinterpret_cast<uint32_t *>(dstp) = wv[c];
+                else *reinterpret_cast<uint16_t *>(dstp) = (uint16_t)wv[c];
             }
             fence_async_shared();                                  // generic-proxy writes -> visible to the tensor core
             __syncwarp();
@@ -233,7 +252,7 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
             if (++stage == FC_STAGES) { stage = 0; phase ^= 1u; }
             return true;
         };
-        if (p.w_tma) {
+        if (WTMA) {
             // weights arrive as [256 k][32 columns] fp32 tiles in shared memory
             int ws = 0; uint32_t wphase = 0;
             bool ok = true;
@@ -243,9 +262,9 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 landed = __shfl_sync(0xffffffffu, landed, 0);
                 if (!landed) { ok = false; break; }
                 const float *wt = reinterpret_cast<const float *>(gen + FC_W_OFFSET + ws * FC_W_BYTES);
-                float4 t[8];
+                float4 t[KPT];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) t[j] = *reinterpret_cast<const float4 *>(wt + (kq * 8 + j) * FC_BN + 4 * n4);
+                for (int j = 0; j < KPT; ++j) t[j] = *reinterpret_cast<const float4 *>(wt + (kq * KPT + j) * FC_BN + 4 * n4);
                 uint32_t wv[4];
                 convert(t, kb, wv);
                 __syncwarp();                                        // every lane holds its values in registers: the tile may be refilled
@@ -258,11 +277,11 @@ fc_sign_f32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         // Three K blocks of this thread's weights are in flight at any time (24 x 16 bytes per thread, 96 KB per SM):
         // the kernel lives on the bytes it keeps in flight, a block's registers are refilled as soon as they are consumed.
         constexpr int DEPTH = 3;
-        float4 buf[DEPTH][8];
-        auto load_block = [&](int32_t kb, float4 (&t)[8]) {
-            const int64_t k0 = (int64_t)kb * FC_KB + kq * 8;
+        float4 buf[DEPTH][KPT];
+        auto load_block = [&](int32_t kb, float4 (&t)[KPT]) {
+            const int64_t k0 = (int64_t)kb * FC_KB + kq * KPT;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
+            for (int j = 0; j < KPT; ++j) {
                 const int64_t k = k0 + j;
                 if (p.vec && cols_ok && k < p.K) {
                     t[j] = __ldcs(reinterpret_cast<const float4 *>(p.w + k * p.ldw + ncol));
@@ -380,10 +399,15 @@ int qnn_fc_sign_f32(const float *x, int64_t M, int64_t K, int64_t ldx, const flo
     int dev = 0;
     QNN_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !opted_in[dev].load(std::memory_order_acquire)) {
-        QNN_CUDA(cudaFuncSetAttribute(fc_sign_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FC_SMEM));
+        QNN_CUDA(cudaFuncSetAttribute(fc_sign_f32_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, FC_SMEM));
+        QNN_CUDA(cudaFuncSetAttribute(fc_sign_f32_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, FC_SMEM));
         if (dev >= 0 && dev < 64) opted_in[dev].store(true, std::memory_order_release);
     }
-    QNN_CUDA(launch_pdl(fc_sign_f32_kernel, dim3((unsigned)ceil_div(N, FC_BN), (unsigned)ceil_div(M, BM)), dim3(FC_THREADS), (size_t)FC_SMEM, st, ma, mw, p));
+    const dim3 grid((unsigned)ceil_div(N, FC_BN), (unsigned)ceil_div(M, BM));
+    if (p.w_tma)
+        QNN_CUDA(launch_pdl(fc_sign_f32_kernel<16, true>, grid, dim3(fc_threads(16)), (size_t)FC_SMEM, st, ma, mw, p));
+    else
+        QNN_CUDA(launch_pdl(fc_sign_f32_kernel<8, false>, grid, dim3(fc_threads(8)), (size_t)FC_SMEM, st, ma, mw, p));
     return check_launch(what);
 }
 

@@ -68,6 +68,7 @@ int run_gemm(const GemmArgs &g, int algo, void *ws, size_t ws_bytes, cudaStream_
     if (algo == QNN_ALGO_AUTO) {
         algo = forced_algo();
         if (algo == QNN_ALGO_AUTO) algo = qnn_select_algo(g.M, g.N, g.K, g.ka, g.kb, g.a_mode, g.b_mode);
+        if (algo == QNN_ALGO_TC_PACKED && !gemm_smallm_supported(g)) algo = QNN_ALGO_TC_FP4;      // (prepared operands, unaligned rows, ...)
         // AUTO never fails for want of a workspace or of a fitting form: fall back to the CUDA-core path
         if (algo == QNN_ALGO_TC_I8 || algo == QNN_ALGO_TC_FP4) {
             const int form = algo == QNN_ALGO_TC_FP4 ? QNN_FORM_FP4 : QNN_FORM_I8;
@@ -228,16 +229,23 @@ int qnn_tc_gemm(const qnn_tc_operand *a, const qnn_tc_operand *b, int64_t M, int
 
 int qnn_select_algo(int64_t M, int64_t N, int64_t K, int ka, int kb, int a_mode, int b_mode)
 {
-    // Measured on B200: the 1-bit mma.sync path never beats xor+popc on the CUDA cores, so it is never picked.
-    // A tensor-core path costs one pass whatever the plane counts; with its two operand-rewriting launches it
-    // overtakes the CUDA-core path once the equivalent plane-pair work M*N*K*ka*kb reaches about 2^30
-    // (100 x 4096 x 4096: 26 us against 33 us; 256 x 1000 x 4096 with 2 planes: 21 us against 86 us;
-    // 1024^3: level).
+    // Measured on B200 (whole call from packed planes, L2 flushed; see the bench's `algorithms` block):
+    //  - the 1-bit mma.sync path never beats xor+popc on the CUDA cores, so it is never picked;
+    //  - a tensor-core path costs one pass whatever the plane counts and overtakes the CUDA-core path once the
+    //    equivalent plane-pair work M*N*K*ka*kb reaches about 2 * 10^7 (128 x 512 x 2048: 15.4 us against 19.4 us;
+    //    64 x 256 x 1024: 11.3 us against 13.3 us; below that every path is one launch of 11-13 us);
+    //  - the kernel that expands packed tiles itself (one launch, no operand rewriting) wins while its 128 x 32 tiles
+    //    fit one wave of CTAs and K is short (512 x 1024 x 2048: 14.3 us against 15.4 us; at K = 4096 the two are level,
+    //    beyond one wave it re-expands too much: 1024^3 18.4 us against 13.5 us).
+    // The answer assumes operands the chosen kernel accepts (alignment, a workspace for the rewritten operands);
+    // QNN_ALGO_AUTO falls back at call time where they are not.
     if (M <= 0 || N <= 0 || K <= 0) return QNN_ALGO_POPC;
     const int form = tc_pick_form(ka, a_mode, kb, b_mode, K);
     if (form == 0) return QNN_ALGO_POPC;
     const double work = (double)M * (double)N * (double)K * (double)ka * (double)kb;
-    if (work < 1073741824.0) return QNN_ALGO_POPC;
+    if (work < 16777216.0) return QNN_ALGO_POPC;
+    if (form == QNN_FORM_FP4 && ka == 1 && kb == 1 && K <= 2048 && ceil_div(M, 128) * ceil_div(N, 32) <= sm_count())
+        return QNN_ALGO_TC_PACKED;
     return form == QNN_FORM_FP4 ? QNN_ALGO_TC_FP4 : QNN_ALGO_TC_I8;
 }
 

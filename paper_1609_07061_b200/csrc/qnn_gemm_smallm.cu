@@ -11,7 +11,7 @@
 //   warp 0        TMA: packed A and B tiles
 //   warp 1        tcgen05.mma issue, tensor-memory owner
 //   warps 2..5    epilogue
-//   warps 6..13   converters
+//   warps 6..21   converters
 //
 // Operands: up to 2 planes each, {0,1} codes or +-1 values (the value sets e2m1 holds).  Every device-side wait is bounded.
 #include <atomic>
@@ -24,7 +24,9 @@ namespace {
 constexpr int SM_BN = 32;                       // output columns per CTA
 constexpr int SM_KB = 256;                      // k per operand stage (128 bytes of e2m1)
 constexpr int SM_SB_WORDS = 64;                 // packed words of K per row in one packed tile (2048 elements); 32 when four planes have to fit
-constexpr int SM_CONV_WARPS = 8;
+constexpr int SM_CONV_WARPS = 16;               // (the kernel is bound by the converters' instruction stream: 16 warps hide more latency than 8)
+constexpr int SM_CONV_THREADS = 32 * SM_CONV_WARPS;
+constexpr int SM_A_ITEMS = BM * 8 / SM_CONV_THREADS;   // packed A words a converter thread expands per operand stage: 2
 constexpr int SM_THREADS = 32 * (6 + SM_CONV_WARPS);
 constexpr int SM_A_BYTES = BM * BKB;            // 16 KB
 constexpr int SM_B_BYTES = SM_BN * BKB;         // 4 KB
@@ -233,20 +235,21 @@ gemm_smallm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
         }
     } else {
         // ---- converters: per operand stage (256 k) the A tile is 128 rows x 8 packed words, the B tile 32 rows x 8 words;
-        // item i of a tile is (row i / 8, word i % 8): thread t expands A items t, t + 256, t + 512, t + 768 and B item t.
+        // item i of a tile is (row i / 8, word i % 8): thread t expands A items t, t + 512 and, if t < 256, B item t.
         // Where an item sits never changes, so its offsets are worked out once; a block that lies wholly inside K and
         // rows inside the matrix take the mask-free path.
         const int t = threadIdx.x - 6 * 32;
         const int word = t & 7;
-        int a_src[4], a_dst[4]; bool a_row_ok[4];
+        int a_src[SM_A_ITEMS], a_dst[SM_A_ITEMS]; bool a_row_ok[SM_A_ITEMS];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int row = (t + 256 * i) >> 3;
+        for (int i = 0; i < SM_A_ITEMS; ++i) {
+            const int row = (t + SM_CONV_THREADS * i) >> 3;
             a_src[i] = row * p.sbw + word;
             a_dst[i] = row * 128 + ((word ^ (row & 7)) << 4);
             a_row_ok[i] = m0 + row < p.M;
         }
-        const int b_row = t >> 3;
+        const bool has_b = t < SM_BN * 8;                         // the B tile has 256 words per stage
+        const int b_row = (t >> 3) & (SM_BN - 1);
         const int b_src = b_row * p.sbw + word;
         const int sb_blocks = p.sbw * 32 / SM_KB;                // operand stages per packed tile
         const int b_dst = SM_A_BYTES + b_row * 128 + ((word ^ (b_row & 7)) << 4);
@@ -269,15 +272,15 @@ gemm_smallm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 const int64_t left = p.K - (kblock * SM_KB + word * 32);
                 const uint32_t kvalid = left >= 32 ? 0xffffffffu : (left > 0 ? ((1u << (int)left) - 1u) : 0u);
                 // expand first (registers), then wait for the operand stage
-                uint4 ea[4], eb;
+                uint4 ea[SM_A_ITEMS], eb = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
+                for (int i = 0; i < SM_A_ITEMS; ++i) {
                     const uint32_t w0 = pa[a_src[i] + kbi * 8];
                     if (!a_row_ok[i]) ea[i] = make_uint4(0u, 0u, 0u, 0u);
                     else if (a_signs && kvalid == 0xffffffffu) ea[i] = signs_to_fp4_full(w0);
                     else ea[i] = planes_to_fp4(w0, p.ka > 1 ? pa[BM * p.sbw + a_src[i] + kbi * 8] : 0u, p.ka, p.a_pm1, kvalid);
                 }
-                {
+                if (has_b) {
                     const uint32_t w0 = pb[b_src + kbi * 8];
                     if (!b_row_ok) eb = make_uint4(0u, 0u, 0u, 0u);
                     else if (b_signs && kvalid == 0xffffffffu) eb = signs_to_fp4_full(w0);
@@ -287,8 +290,8 @@ gemm_smallm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_cons
                 if (!__all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 25))) { ok = false; break; }
                 uint8_t *at = gen + stage * SM_STAGE_BYTES;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4 *>(at + a_dst[i]) = ea[i];       // (128-byte swizzle in a_dst)
-                *reinterpret_cast<uint4 *>(at + b_dst) = eb;
+                for (int i = 0; i < SM_A_ITEMS; ++i) *reinterpret_cast<uint4 *>(at + a_dst[i]) = ea[i];       // (128-byte swizzle in a_dst)
+                if (has_b) *reinterpret_cast<uint4 *>(at + b_dst) = eb;
                 fence_async_shared();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(full_bar(stage));

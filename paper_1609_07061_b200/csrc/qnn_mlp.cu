@@ -60,7 +60,12 @@ LayerChoice choose_layer(int64_t M, int in_bits, const qnn_mlp_layer *layers, in
     const int best_form = tc_pick_form(ka, a_mode, 1, QNN_MODE_PM1, ly.K);
     if (algo == QNN_ALGO_AUTO) algo = resolve_env_algo();
     LayerChoice c{algo, 0};
-    if (algo == QNN_ALGO_AUTO) c.algo = qnn_select_algo(M, ly.N, ly.K, ka, 1, a_mode, QNN_MODE_PM1);
+    if (algo == QNN_ALGO_AUTO) {
+        c.algo = qnn_select_algo(M, ly.N, ly.K, ka, 1, a_mode, QNN_MODE_PM1);
+        // (inside a network the layers hand their activations over in tensor-core form and the weights may be prepared:
+        // the packed-tile kernel, which takes packed planes only, is left to single products)
+        if (c.algo == QNN_ALGO_TC_PACKED) c.algo = QNN_ALGO_TC_FP4;
+    }
     if (c.algo == QNN_ALGO_B1_MMA && ka != 1) c.algo = QNN_ALGO_POPC;
     if (c.algo == QNN_ALGO_TC_PACKED && best_form != QNN_FORM_FP4) c.algo = QNN_ALGO_POPC;     // (more than two planes, or sums beyond 2^24)
     if (c.algo == QNN_ALGO_TC_FP4 && best_form != QNN_FORM_FP4) c.algo = best_form ? QNN_ALGO_TC_I8 : QNN_ALGO_POPC;
