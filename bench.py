@@ -39,8 +39,8 @@ UNIT = "Tops/s (2*M*N*K per 1-bit plane product)"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from
 # the ncu capture of that kernel; None until a capture exists for the kernel the run selects.
 NCU_TRAFFIC_BYTES = {
-    # hidden layer 2 (the launch the live timing brackets): 28.97 MB read + 0.25 MB written per launch
-    "tcgen05 kind::mxf4 xnor product 10000x4096x4096, threshold epilogue (gemm_tc_kernel<FP4>)": 29.22e6,
+    # hidden layer 2 (the launch the live timing brackets): 28.96 MB read + 0.23 MB written per launch
+    "tcgen05 kind::mxf4 xnor product 10000x4096x4096, threshold epilogue (gemm_tc_kernel<FP4>)": 29.20e6,
 }
 
 
