@@ -44,6 +44,9 @@ struct TcParams {
     const int32_t *thr; const uint8_t *flip; uint32_t *out_bits; int64_t ld_bits;
     uint8_t *out_form; int64_t ld_form; int out_form_kind;
     uint32_t idesc;
+    // The last column block may be narrower than the tile: its instructions then multiply only n_last columns
+    // (a multiple of 16), described by idesc_last, and a pair's second CTA loads its B rows n_last / 2 further on.
+    uint32_t idesc_last; int32_t n_last;
     int32_t thr_clamp;               // int8 form: max |sum| + 1 when that is below 2^30 (else 0: plain compares)
     // asynchronous (TMA) stores through the per-warp staging buffers: 0 = plain stores from registers
     int tma_out;                     // 1: int32 row-major [M, N]; 2: int32 NCHW [img, n, pix]
@@ -408,13 +411,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // destination, barriers and the K coordinate are carried from stage to stage (see the MMA warp)
             const uint32_t fb0 = (CTAS == 2) ? map_to_cta(full_bar(0), 0) : full_bar(0), eb0 = empty_bar(0);
             uint32_t sa = base, fb = fb0, eb = eb0;
+            // tile coordinates advance by additions: one division per role, before its loop
+            const uint32_t step_n = (gridDim.x / CTAS) / tiles_m, step_m = (gridDim.x / CTAS) - step_n * tiles_m;
+            int32_t tn = (int32_t)((blockIdx.x / CTAS) / tiles_m), tm = (int32_t)((blockIdx.x / CTAS) - (uint32_t)tn * tiles_m);
             for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS) {
-                const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
                 int32_t img = 0, y0 = 0;
                 if (p.conv) { img = tm / p.tiles_per_img; y0 = (tm - img * p.tiles_per_img) * p.cR; img *= p.cG; }
                 int32_t cx = 0, kx = 0, tx = -p.cpad, ty = y0 - p.cpad;   // conv: channel byte, K byte, tap column and row of kb
                 const int32_t a_row = (CTAS == 2) ? (tm * 2 + (int32_t)rank) * BM : tm * BM;
-                const int32_t b_row = (CTAS == 2) ? tn * BN + (int32_t)rank * (BN / 2) : tn * BN;
+                const int32_t b_row = (CTAS == 2) ? tn * BN + (int32_t)rank * ((tn == p.tiles_n - 1 ? p.n_last : BN) / 2) : tn * BN;
                 const int32_t cx_end = p.cblocks * KB, tx_end = p.cKW - p.cpad;
                 // (the convolution's loop is unrolled, the plain one is not: measured best for each)
                 if (p.conv) {
@@ -453,6 +458,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         sa = sa_n; fb = fb_n; eb = eb_n; phase = phase_n;
                     }
                 }
+                tm += (int32_t)step_m; tn += (int32_t)step_n;
+                if (tm >= (int32_t)tiles_m) { tm -= (int32_t)tiles_m; ++tn; }
             }
         }
     } else if (warp == 1) {
@@ -469,8 +476,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
             const uint32_t a_lo0 = (uint32_t)desc0, fb0 = full_bar(0), eb0 = empty_bar(0);
             uint32_t a_lo = a_lo0, fb = fb0, eb = eb0;
+            const uint32_t step_n = (gridDim.x / CTAS) / tiles_m, step_m = (gridDim.x / CTAS) - step_n * tiles_m;
+            uint32_t tn = (blockIdx.x / CTAS) / tiles_m, tm = (blockIdx.x / CTAS) - tn * tiles_m;
             for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS, ++iter) {
                 const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
+                const uint32_t idesc = (tn == (uint32_t)p.tiles_n - 1u) ? p.idesc_last : p.idesc;
+                tm += step_m; tn += step_n;
+                if (tm >= tiles_m) { tm -= tiles_m; ++tn; }
                 if (!mbar_wait(tempty_bar(as), aphase ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + as * (uint32_t)BN;
@@ -485,11 +497,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     const uint32_t phase_n = wrap ? phase ^ 1u : phase;
                     const uint32_t b_lo = a_lo + (uint32_t)(S::A_BYTES >> 4);
                     if (CTAS == 2)
-                        ready = umma_stage_pair<FORM>(fb_n, phase_n, d_tmem, a_lo, b_lo, desc_hi, p.idesc, (uint32_t)(kb != 0), sf, eb) != 0;
+                        ready = umma_stage_pair<FORM>(fb_n, phase_n, d_tmem, a_lo, b_lo, desc_hi, idesc, (uint32_t)(kb != 0), sf, eb) != 0;
                     else if (KB == 64)
-                        ready = umma_stage_half(fb_n, phase_n, d_tmem, a_lo, b_lo, desc_hi, p.idesc, (uint32_t)(kb != 0), sf, eb) != 0;
+                        ready = umma_stage_half(fb_n, phase_n, d_tmem, a_lo, b_lo, desc_hi, idesc, (uint32_t)(kb != 0), sf, eb) != 0;
                     else
-                        ready = umma_stage<FORM>(fb_n, phase_n, d_tmem, a_lo, b_lo, desc_hi, p.idesc, (uint32_t)(kb != 0), sf, eb) != 0;
+                        ready = umma_stage<FORM>(fb_n, phase_n, d_tmem, a_lo, b_lo, desc_hi, idesc, (uint32_t)(kb != 0), sf, eb) != 0;
                     stage = wrap ? 0 : stage + 1;
                     a_lo = a_lo_n; fb = fb_n; eb = eb_n; phase = phase_n;
                 }
@@ -546,12 +558,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             r_y = rem / p.cW;
             r_x = rem - r_y * p.cW;
         }
+        const uint32_t step_n = (gridDim.x / CTAS) / tiles_m, step_m = (gridDim.x / CTAS) - step_n * tiles_m;
+        int32_t tn = (int32_t)((blockIdx.x / CTAS) / tiles_m), tm = (int32_t)((blockIdx.x / CTAS) - (uint32_t)tn * tiles_m);
         if (want_sign && blockIdx.x / CTAS < num_tiles) {
-            tn_fetched = (int32_t)((blockIdx.x / CTAS) / tiles_m);
+            tn_fetched = tn;
             fetch_thresholds((int64_t)tn_fetched * BN);
         }
         for (uint32_t t = blockIdx.x / CTAS; t < num_tiles && ok; t += gridDim.x / CTAS, ++iter) {
-            const int32_t tm = (int32_t)(t % tiles_m), tn = (int32_t)(t / tiles_m);
+            // the next tile's coordinates
+            int32_t tm_next = tm + (int32_t)step_m, tn_next = tn + (int32_t)step_n;
+            if (tm_next >= (int32_t)tiles_m) { tm_next -= (int32_t)tiles_m; ++tn_next; }
             const uint32_t as = iter & 1u, aphase = (iter >> 1) & 1u;
             const int64_t ntile = (int64_t)tn * BN;
 
@@ -585,7 +601,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (want_sign) {
                 const uint32_t tnext = t + gridDim.x / CTAS;
                 if (tnext < num_tiles) {
-                    const int32_t tn_next = (int32_t)(tnext / tiles_m);
                     if (tn_next != tn_fetched) { tn_fetched = tn_next; fetch_thresholds((int64_t)tn_next * BN); }
                 }
             }
@@ -807,6 +822,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (CTAS == 2) mbar_arrive_cluster(map_to_cta(tempty_bar(as), 0));
                 else mbar_arrive(tempty_bar(as));
             }
+            tm = tm_next; tn = tn_next;
         }
         // stores still reading shared memory must finish before the block's shared memory goes away
         if (STG) {
@@ -1062,6 +1078,11 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, int 
     p.tiles_n = (int32_t)ceil_div(p.N, BN);
     p.idesc |= (uint32_t)(BN >> 3) << 17;
     if (CTAS == 2) p.idesc = (p.idesc & ~(0x1fu << 24)) | ((uint32_t)((2 * BM) >> 4) << 24);   // the pair's instruction is 256 rows tall
+    {
+        const int64_t rest = p.N - (int64_t)(p.tiles_n - 1) * BN;       // columns of the last block, 1..BN
+        p.n_last = (int32_t)(rest >= BN ? BN : ((rest + 15) / 16) * 16);
+        p.idesc_last = (p.idesc & ~(0x3fu << 17)) | ((uint32_t)(p.n_last >> 3) << 17);
+    }
     const bool conv_full_tiles = p.conv && p.cR * p.cW == BM && p.cG == 1;
     if (p.out != nullptr && aligned(p.out, 16)) {
         // (the bulk store clips the innermost extent in 16-byte units, so N must be a whole number of them)
