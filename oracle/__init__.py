@@ -20,6 +20,9 @@ Pins (what each routine is checked against, other than itself) live in
   mlp_forward     Algorithm 4 step by step with the routines above
   ap2 / log_quant float64 round(log2|x|) away from ties, exact powers of two, the factor-sqrt(2)
                   bound, monotonicity, clipping, zero / infinities / NaN
+  log_gemm        exact rational arithmetic (fractions) on small inputs built from the literal
+                  sign * 2^round(log2|x|), closed forms (constant rows, clipping at both ends, the
+                  31-exponent range beyond int32), additivity in w
   maxpool2x2      library max_pool2d in float64; the identity that pooling the
                   integer sums and then thresholding equals OR (AND where the
                   comparison is flipped) of the thresholded bits, by brute force
@@ -215,6 +218,17 @@ def log_quant(x, emin: int, emax: int) -> np.ndarray:
     _check(_load().qo_log_quant(_ptr(x), ctypes.c_int64(x.size), ctypes.c_int(emin), ctypes.c_int(emax), _ptr(v)),
            "log_quant")
     return v
+
+
+def log_gemm(x, w, emin: int, emax: int) -> np.ndarray:
+    """The backward products of Algorithm 1 with logarithmically quantised gradients (Eq. 10; Sec. 4.1 quantises
+    them to 6 bits: a sign and up to 31 exponents): out[m,n] = sum_k LogQuant(x)[m,k] * w[k,n], exact, as int64 in
+    units of 2^emin.  x: float [M,K]; w: integers [K,N] (the +-1 weights, or +-1 activations for the weight
+    gradient).  The definition written out: quantise, then an integer matrix product (a library matmul on int64)."""
+    if emax - emin > 30:
+        raise ValueError("log_gemm: at most 31 exponents")
+    v = log_quant(x, emin, emax).astype(np.int64)
+    return v @ np.ascontiguousarray(w).astype(np.int64)
 
 
 def maxpool2x2(x) -> np.ndarray:

@@ -175,3 +175,43 @@ def test_log_quant_pins():
     assert set(mags.tolist()) <= {1, 2, 4, 8, 16, 32, 64}
     with pytest.raises(ValueError):
         oracle.log_quant(y, 2, 1)
+
+
+def test_log_gemm_pins():
+    """Algorithm 1's backward products on Eq. 10 codes: out = sum_k sign(x) 2^clamp(round(log2|x|)) w, in units of 2^emin."""
+    from fractions import Fraction
+    import math
+    rng = np.random.default_rng(11)
+    # (i) exact rational arithmetic on inputs away from the rounding ties
+    M, K, N, emin, emax = 5, 23, 4, -12, 3
+    x = (rng.standard_normal((M, K)) * np.exp2(rng.integers(-14, 5, (M, K)))).astype(np.float32)
+    l2 = np.log2(np.abs(x.astype(np.float64)))
+    assert np.all(np.abs(l2 - np.floor(l2) - 0.5) > 1e-6)
+    w = rng.integers(0, 2, (K, N)) * 2 - 1
+    got = oracle.log_gemm(x, w, emin, emax)
+    assert got.dtype == np.int64
+    for m in range(M):
+        for n in range(N):
+            acc = Fraction(0)
+            for k in range(K):
+                e = min(max(round(math.log2(abs(float(x[m, k])))), emin), emax)
+                acc += (1 if x[m, k] >= 0 else -1) * Fraction(2) ** e * int(w[k, n])
+            assert Fraction(int(got[m, n])) * Fraction(2) ** emin == acc
+    # (ii) constant rows: every element 2^e0 gives 2^(e0 - emin) * sum(w); clipping at both ends
+    ones = np.full((2, K), 0.25, np.float32)
+    np.testing.assert_array_equal(oracle.log_gemm(ones, w, -4, 2), np.tile(4 * w.sum(axis=0), (2, 1)))
+    tiny, huge = np.full((1, K), 1e-30, np.float32), np.full((1, K), -1e30, np.float32)
+    np.testing.assert_array_equal(oracle.log_gemm(tiny, w, -4, 2), w.sum(axis=0)[None, :])
+    np.testing.assert_array_equal(oracle.log_gemm(huge, w, -4, 2), -64 * w.sum(axis=0)[None, :])
+    # (iii) the full 31-exponent range of a 6-bit code: sums beyond int32 stay exact
+    big = np.full((1, 8), 1.0, np.float32)
+    np.testing.assert_array_equal(oracle.log_gemm(big, np.ones((8, 1), np.int64), -30, 0), [[8 * 2 ** 30]])
+    mixed = np.array([[1.0, 2.0 ** -30, -(2.0 ** -15)]], np.float32)
+    np.testing.assert_array_equal(oracle.log_gemm(mixed, np.array([[1], [1], [1]]), -30, 0), [[2 ** 30 + 1 - 2 ** 15]])
+    # (iv) additivity in w, oddness in x
+    w2 = rng.integers(-3, 4, (K, N))
+    np.testing.assert_array_equal(oracle.log_gemm(x, w + w2, emin, emax), oracle.log_gemm(x, w, emin, emax) + oracle.log_gemm(x, w2, emin, emax))
+    nz = np.where(x == 0, np.float32(1.0), x)
+    np.testing.assert_array_equal(oracle.log_gemm(-nz, w, emin, emax), -oracle.log_gemm(nz, w, emin, emax))
+    with pytest.raises(ValueError):
+        oracle.log_gemm(x, w, -31, 0)
