@@ -238,6 +238,41 @@ class MlpBench:
         self.q.qnn_mlp_forward_host(self.x_host, self.M, IN_BITS, self.layers, self.scores_host, self.algo, self.ws)
 
 
+def backward_records(q, flush, rec):
+    M, Nu, K = BATCH, 4096, 4096                       # batch, units of the layer, its inputs
+    emin, emax = -30, 0
+    G = q.qnn_logquant_groups(emin, emax)
+    g = torch.Generator(device="cuda").manual_seed(6)
+    gs = torch.randn(M, Nu, device="cuda", generator=g) * torch.exp2(torch.randint(emin, emax + 1, (M, Nu), device="cuda", generator=g).float())
+    for name, transposed, rows, kdim, ncols in (("g_a = LogQuant(g_s) W", 0, M, Nu, K), ("g_W = a^T LogQuant(g_s)", 1, Nu, M, K)):
+        kz = (kdim + 31) // 32 * 32
+        ld = (kz + 127) // 128 * 128
+        a8 = torch.empty(G * rows, ld, dtype=torch.uint8, device="cuda")
+        bits = torch.randint(-2**31, 2**31 - 1, (ncols, (kdim + 31) // 32), dtype=torch.int32, device="cuda", generator=g)
+        if kdim % 32:
+            bits[:, -1] &= (1 << (kdim % 32)) - 1
+        b8 = torch.empty(ncols, ld, dtype=torch.uint8, device="cuda")
+        q.qnn_tc_prepack(bits, 1, q.QNN_MODE_PM1, (kdim + 31) // 32, 0, ncols, kdim, q.QNN_FORM_I8, b8, ld)
+        part = torch.empty(G * rows, ncols, dtype=torch.int32, device="cuda")
+        out = torch.empty(rows, ncols, dtype=torch.int64, device="cuda")
+        A = q.tc_operand(a8, ld, q.QNN_FORM_I8, planes=7, mode=q.QNN_MODE_PM1)
+        Bo = q.tc_operand(b8, ld, q.QNN_FORM_I8, planes=1, mode=q.QNN_MODE_PM1)
+        tag = "g_a" if not transposed else "g_W"
+        ms, best = _time_op(lambda: q.qnn_logquant_pack_groups(gs, rows, kdim, Nu, transposed, emin, emax, a8, ld), flush, reps=5)
+        rec(f"alg1_backward_{tag}_pack_groups", ms, best, bytes_=4.0 * M * Nu + float(G) * rows * ld,
+            note=f"{name}: fp32 gradient -> {G} int8 group matrices ({'transposed' if transposed else 'row-major'})")
+
+        def whole():
+            q.qnn_logquant_pack_groups(gs, rows, kdim, Nu, transposed, emin, emax, a8, ld)
+            q.qnn_tc_gemm(A, Bo, G * rows, ncols, kdim, out=part, ldo=ncols)
+            q.qnn_logquant_combine(part, G, rows, ncols, ncols, out, ncols)
+        ms, best = _time_op(whole, flush, reps=5)
+        rec(f"alg1_backward_{tag}_{rows}x{ncols}x{kdim}_6bit_log_gradients", ms, best, ops=2.0 * rows * ncols * kdim * G,
+            note=f"{name}: pack, one int8 product of {G} stacked groups, int64 combine; rate counted per int8 multiply-accumulate issued "
+                 f"({2.0 * rows * ncols * kdim / ms / 1e9:.0f} Top/s counted once per 6-bit product)")
+        del a8, bits, b8, part, out
+
+
 def _cpu_baseline(sample_rows: int = 0, budget_s: float = 15.0):
     """The oracle as it stands, on the host cores, on a bounded sample of batch rows of the same workload."""
     import oracle
@@ -613,6 +648,10 @@ def run_extras(q, bench, peaks, algo):
     # the whole CIFAR-10 ConvNet of Table 7 (first layer on 8-bit pixels, pooled thresholds, FC head), one call per pass
     for Bn in (128, 1024):
         convnet_record(q, Bn, flush, rec)
+
+    # Algorithm 1's backward products of a 4096-unit hidden layer at batch 10000 with 6-bit logarithmic gradients
+    # (Eq. 10, 31 exponents = 5 int8 groups): gradient x +-1 weights, and +-1 activations^T x gradient
+    backward_records(q, flush, rec)
 
     # config 5: LSTM gate 4b x 4b and the square sweep
     wl5 = workloads.lstm_gate()

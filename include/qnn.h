@@ -509,6 +509,34 @@ QNN_API size_t qnn_mlp_workspace_bytes(int64_t M, int in_bits, const qnn_mlp_lay
 QNN_API int qnn_logquant_pack_i8(const float *x, int64_t rows, int64_t K, int64_t ldx, int emin, int emax, void *out,
                                  int64_t ld_bytes, void *stream);
 
+/* Eq. 10 with up to 31 exponents (a 6-bit code: a sign and 5 bits of exponent), for the
+ * backward products of Algorithm 1 with quantised gradients (Sec. 4.4: of the gradient
+ * quantisers tried only the logarithmic one worked, at 6 bits; end of Sec. 5: quantised
+ * gradients let the backward pass use the binary kernel): gradient x +-1 weights, and +-1 activations x gradient.
+ * A code sign * 2^(e - emin) with e - emin up to 30 has one set bit; the exponents are cut
+ * into groups of seven, group g holding sign * 2^(e - emin - 7g) where e falls into it and
+ * 0 elsewhere.  qnn_logquant_groups = the number of groups G = (emax - emin) / 7 + 1
+ * (0 when the range is not 0..30).  qnn_logquant_pack_groups writes the G group matrices
+ * stacked row-wise, int8 [G * rows, ld_bytes] (group g at rows g*rows ..): ONE operand of
+ * the int8 tensor-core form (qnn_tc_gemm, QNN_FORM_I8, QNN_MODE_PM1, 7 planes) whose
+ * product with a +-1 matrix is int32 [G * rows, N]; qnn_logquant_combine then gives
+ *     out[m, n] = sum_g 2^(7g) * p[g * M + m, n]
+ * the exact sum of code x weight in int64, in units of 2^emin.
+ *   x           device, float; transposed = 0: [rows, ldx], a row of x is a row of the
+ *               operand (K elements); transposed = 1: [K, ldx >= rows], a COLUMN of x is a
+ *               row of the operand (the weight gradient contracts over the batch)
+ *   out         device, int8 [G * rows, ld_bytes]; ld_bytes >= K rounded up to 32, a multiple
+ *               of 4 (of 16 to serve as a tensor-core operand); bytes K .. roundup(K, 32) of
+ *               every row are written as zero
+ *   p, out(i64) device; ldp, ldo in elements
+ * Rounding, zero, infinities, NaN and the sign as in qnn_logquant_pack_i8.
+ * Errors: INVALID_ARG, UNSUPPORTED (more than 31 exponents), ALIGNMENT, CUDA. */
+QNN_API int qnn_logquant_groups(int emin, int emax);
+QNN_API int qnn_logquant_pack_groups(const float *x, int64_t rows, int64_t K, int64_t ldx, int transposed, int emin, int emax,
+                                     void *out, int64_t ld_bytes, void *stream);
+QNN_API int qnn_logquant_combine(const int32_t *p, int groups, int64_t M, int64_t N, int64_t ldp, int64_t *out, int64_t ldo,
+                                 void *stream);
+
 /* ------------------------------------------------------------------------- */
 /* The ConvNet of Table 7                                                     */
 /* ------------------------------------------------------------------------- */

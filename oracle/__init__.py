@@ -221,7 +221,7 @@ def log_quant(x, emin: int, emax: int) -> np.ndarray:
 
 
 def log_gemm(x, w, emin: int, emax: int) -> np.ndarray:
-    """The backward products of Algorithm 1 with logarithmically quantised gradients (Eq. 10; Sec. 4.1 quantises
+    """The backward products of Algorithm 1 with logarithmically quantised gradients (Eq. 10; Sec. 4.4 quantises
     them to 6 bits: a sign and up to 31 exponents): out[m,n] = sum_k LogQuant(x)[m,k] * w[k,n], exact, as int64 in
     units of 2^emin.  x: float [M,K]; w: integers [K,N] (the +-1 weights, or +-1 activations for the weight
     gradient).  The definition written out: quantise, then an integer matrix product (a library matmul on int64)."""

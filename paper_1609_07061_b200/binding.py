@@ -106,6 +106,9 @@ _SIGS = {
     "qnn_conv_form": (i32, [i32]),
     "qnn_conv_can_pool": (i32, [i32, i32]),
     "qnn_conv_prepared_bytes": (sz, [i32, i32, i32, i32, i32]),
+    "qnn_logquant_groups": (i32, [i32, i32]),
+    "qnn_logquant_pack_groups": (i32, [vp, i64, i64, i64, i32, i32, i32, vp, i64, vp]),
+    "qnn_logquant_combine": (i32, [vp, i32, i64, i64, i64, vp, i64, vp]),
     "qnn_conv_prepare": (i32, [vp, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
     "qnn_binary_conv2d_prepared": (i32, [ctypes.POINTER(qnn_conv_io), i32, i32, i32, i32, vp, i32, i32, i32, i32, vp, sz, vp]),
     "qnn_logquant_pack_i8": (i32, [vp, i64, i64, i64, i32, i32, vp, i64, vp]),
@@ -319,6 +322,19 @@ def qnn_binary_conv2d(x, B, C, H, W, w, Cout, KH, KW, stride, pad, pad_bit, out_
 
 def qnn_conv_form(C) -> int:
     return int(_lib.qnn_conv_form(C))
+
+
+def qnn_logquant_groups(emin, emax) -> int:
+    return int(_lib.qnn_logquant_groups(emin, emax))
+
+
+def qnn_logquant_pack_groups(x, rows, K, ldx, transposed, emin, emax, out, ld_bytes):
+    _ck(_lib.qnn_logquant_pack_groups(_p(x), rows, K, ldx, int(transposed), emin, emax, _p(out), ld_bytes, _stream()),
+        "qnn_logquant_pack_groups")
+
+
+def qnn_logquant_combine(p, groups, M, N, ldp, out, ldo):
+    _ck(_lib.qnn_logquant_combine(_p(p), groups, M, N, ldp, _p(out), ldo, _stream()), "qnn_logquant_combine")
 
 
 def qnn_conv_prepared_bytes(Cout, C, KH, KW, pad) -> int:

@@ -286,6 +286,78 @@ def test_logquant_products(q, M, N, K, la, lb):
     out.check()
 
 
+def _log_backward_product(q, G_f32, transposed, rows, K, W_pm1_rows, emin, emax):
+    """LogQuant(gradient) [rows, K] times +-1 rows [N, K] -> int64 [rows, N] through the group operand, one int8 product and
+    the combine step.  G_f32: the gradient as stored ([rows, K], or [K, rows] when `transposed`)."""
+    N = W_pm1_rows.shape[0]
+    groups = q.qnn_logquant_groups(emin, emax)
+    kz = (K + 31) // 32 * 32
+    ld = (kz + 15) // 16 * 16
+    a8 = Guarded((groups * rows, ld), torch.uint8, fill=0x5C)
+    q.qnn_logquant_pack_groups(dev(G_f32), rows, K, G_f32.shape[1], transposed, emin, emax, a8.t, ld)
+    bits = torch.zeros(N, (K + 31) // 32, dtype=torch.int32, device="cuda")
+    q.qnn_quantize_pack_sign(dev(W_pm1_rows.astype(np.float32)), N, K, K, bits, (K + 31) // 32)
+    b8 = torch.zeros(N, ld, dtype=torch.uint8, device="cuda")
+    q.qnn_tc_prepack(bits, 1, q.QNN_MODE_PM1, (K + 31) // 32, 0, N, K, q.QNN_FORM_I8, b8, ld)
+    part = torch.empty(groups * rows, N, dtype=torch.int32, device="cuda")
+    A = q.tc_operand(a8.t, ld, q.QNN_FORM_I8, planes=7, mode=q.QNN_MODE_PM1)
+    Bo = q.tc_operand(b8, ld, q.QNN_FORM_I8, planes=1, mode=q.QNN_MODE_PM1)
+    q.qnn_tc_gemm(A, Bo, groups * rows, N, K, out=part, ldo=N)
+    out = Guarded((rows, N), torch.int64, fill=-7)
+    q.qnn_logquant_combine(part, groups, rows, N, N, out.t, N)
+    torch.cuda.synchronize()
+    assert q.qnn_device_status() == 0, q.qnn_last_error()
+    a8.check(); out.check()
+    return a8.t.cpu().numpy().view(np.int8), out.t.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,Nu,K,emin,emax", [(70, 40, 96, -30, 0), (300, 130, 1000, -20, -3), (129, 257, 515, -6, 0), (33, 5, 31, -14, 0)])
+def test_alg1_backward_products_log_gradients(q, M, Nu, K, emin, emax):
+    """Algorithm 1's backward pass with logarithmically quantised gradients (Eq. 10, up to 31 exponents: the 6-bit code of
+    Sec. 4.4): g_a = LogQuant(g_s) W^b (batch x units times units x inputs) and g_W = a^b^T LogQuant(g_s), the second one
+    contracting over the batch through the transposed packer.  Exact int64 sums against the oracle; the group operand's
+    bytes against the oracle's codes."""
+    rng = np.random.default_rng(M + Nu + K)
+    gs = (rng.standard_normal((M, Nu)) * np.exp2(rng.integers(emin - 2, emax + 3, (M, Nu)))).astype(np.float32)   # gradient of the layer's sums
+    gs.reshape(-1)[:7] = np.array([0.0, -0.0, np.nan, np.inf, -np.inf, 1e-45, -1e-45], np.float32)
+    Wb = rng.integers(0, 2, (K, Nu)).astype(np.int32) * 2 - 1          # the layer's +-1 weights [inputs, units]
+    ab = rng.integers(0, 2, (M, K)).astype(np.int32) * 2 - 1           # its +-1 input activations
+    # g_a[m, k] = sum_n LogQuant(g_s)[m, n] W[k, n]: contraction over the units; the gradient's rows are operand rows
+    codes, got_a = _log_backward_product(q, gs, 0, M, Nu, Wb, emin, emax)
+    np.testing.assert_array_equal(got_a, oracle.log_gemm(gs, Wb.T, emin, emax))
+    v = oracle.log_quant(gs, emin, emax).astype(np.int64)
+    groups = q.qnn_logquant_groups(emin, emax)
+    rebuilt = sum(codes[g * M:(g + 1) * M, :Nu].astype(np.int64) << (7 * g) for g in range(groups))
+    np.testing.assert_array_equal(rebuilt, v)
+    assert (codes[:, Nu:(Nu + 31) // 32 * 32] == 0).all()
+    # g_W[n, k] = sum_m LogQuant(g_s)[m, n] a[m, k]: contraction over the batch; the gradient's COLUMNS are operand rows
+    _, got_w = _log_backward_product(q, gs, 1, Nu, M, np.ascontiguousarray(ab.T), emin, emax)
+    np.testing.assert_array_equal(got_w, oracle.log_gemm(np.ascontiguousarray(gs.T), ab, emin, emax))
+
+
+def test_logquant_groups_argument_errors(q):
+    x = torch.zeros(4, 32, device="cuda")
+    out = torch.zeros(5 * 4, 32, dtype=torch.uint8, device="cuda")
+    assert q.qnn_logquant_groups(-30, 0) == 5 and q.qnn_logquant_groups(-6, 0) == 1 and q.qnn_logquant_groups(-7, 0) == 2
+    assert q.qnn_logquant_groups(-31, 0) == 0 and q.qnn_logquant_groups(1, 0) == 0
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_pack_groups(x, 4, 32, 32, 0, -31, 0, out, 32)
+    assert e.value.status == q.QNN_ERR_UNSUPPORTED
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_pack_groups(x, 4, 32, 16, 0, -3, 0, out, 32)          # ldx below K
+    assert e.value.status == q.QNN_ERR_INVALID_ARG
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_pack_groups(x, 4, 32, 32, 0, -3, 0, out, 30)          # row stride below K rounded up
+    assert e.value.status == q.QNN_ERR_INVALID_ARG
+    p = torch.zeros(8, 4, dtype=torch.int32, device="cuda")
+    o = torch.zeros(4, 4, dtype=torch.int64, device="cuda")
+    with pytest.raises(q.QnnError) as e:
+        q.qnn_logquant_combine(p, 6, 4, 4, 4, o, 4)
+    assert e.value.status == q.QNN_ERR_INVALID_ARG
+    q.qnn_logquant_pack_groups(x, 0, 32, 32, 0, -3, 0, out, 32)              # empty: nothing to do
+    q.qnn_logquant_combine(p, 2, 0, 4, 4, o, 4)
+
+
 @pytest.mark.parametrize("K", [256, 512, 200])
 @pytest.mark.parametrize("a_rows", ["zeros", "mixed"])
 def test_fp4_zero_sum_against_zero_threshold(q, K, a_rows):
