@@ -83,15 +83,37 @@ __global__ void __launch_bounds__(256) log_groups_t_kernel(const float *__restri
     }
 }
 
+// four consecutive columns per thread where the rows allow 16-byte accesses (the pass is a stream: 20 bytes in and 8 out
+// per element)
+template <bool VEC>
 __global__ void __launch_bounds__(256) log_combine_kernel(const int32_t *__restrict__ p, int groups, int64_t M, int64_t N, int64_t ldp,
                                                           int64_t *__restrict__ out, int64_t ldo)
 {
-    const int64_t total = M * N;
+    const int64_t nq = VEC ? N / 4 : N;
+    const int64_t total = M * nq;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t m = i / N, n = i - m * N;
-        int64_t acc = 0;
-        for (int g = 0; g < groups; ++g) acc += (int64_t)__ldcs(p + ((int64_t)g * M + m) * ldp + n) << (LOG_GROUP * g);
-        out[m * ldo + n] = acc;
+        const int64_t m = i / nq, n = (i - m * nq) * (VEC ? 4 : 1);
+        if (VEC) {
+            int64_t acc[4] = {0, 0, 0, 0};
+            int4 v[5];
+#pragma unroll
+            for (int g = 0; g < 5; ++g)
+                if (g < groups) v[g] = __ldcs(reinterpret_cast<const int4 *>(p + ((int64_t)g * M + m) * ldp + n));
+#pragma unroll
+            for (int g = 0; g < 5; ++g) {
+                if (g < groups) {
+                    acc[0] += (int64_t)v[g].x << (LOG_GROUP * g); acc[1] += (int64_t)v[g].y << (LOG_GROUP * g);
+                    acc[2] += (int64_t)v[g].z << (LOG_GROUP * g); acc[3] += (int64_t)v[g].w << (LOG_GROUP * g);
+                }
+            }
+            longlong2 *dst = reinterpret_cast<longlong2 *>(out + m * ldo + n);
+            __stcs(dst, make_longlong2(acc[0], acc[1]));
+            __stcs(dst + 1, make_longlong2(acc[2], acc[3]));
+        } else {
+            int64_t acc = 0;
+            for (int g = 0; g < groups; ++g) acc += (int64_t)__ldcs(p + ((int64_t)g * M + m) * ldp + n) << (LOG_GROUP * g);
+            out[m * ldo + n] = acc;
+        }
     }
 }
 
@@ -146,8 +168,10 @@ int qnn_logquant_combine(const int32_t *p, int groups, int64_t M, int64_t N, int
     QNN_REQUIRE(p && out, QNN_ERR_INVALID_ARG, "%s: NULL pointer", what);
     QNN_REQUIRE(ldp >= N && ldo >= N, QNN_ERR_INVALID_ARG, "%s: leading dimension below N", what);
     QNN_REQUIRE(aligned(p, 4) && aligned(out, 8), QNN_ERR_ALIGNMENT, "%s: p must be 4-byte, out 8-byte aligned", what);
-    const int64_t need = ceil_div(M * N, 256), cap = (int64_t)sm_count() * 16;
-    log_combine_kernel<<<(int)(need < cap ? need : cap), 256, 0, as_stream(stream)>>>(p, groups, M, N, ldp, out, ldo);
+    const bool vec = N % 4 == 0 && ldp % 4 == 0 && ldo % 2 == 0 && aligned(p, 16) && aligned(out, 16);
+    const int64_t need = ceil_div(M * (vec ? N / 4 : N), 256), cap = (int64_t)sm_count() * 32;
+    if (vec) log_combine_kernel<true><<<(int)(need < cap ? need : cap), 256, 0, as_stream(stream)>>>(p, groups, M, N, ldp, out, ldo);
+    else log_combine_kernel<false><<<(int)(need < cap ? need : cap), 256, 0, as_stream(stream)>>>(p, groups, M, N, ldp, out, ldo);
     return check_launch(what);
 }
 
