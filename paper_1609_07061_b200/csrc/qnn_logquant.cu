@@ -74,13 +74,14 @@ __global__ void __launch_bounds__(256) log_groups_t_kernel(const float *__restri
         tile[ty + 8 * i][tx] = (k < K && n < rows) ? log_code(__ldcs(x + k * ldx + n), emin, emax) : 0xffu;
     }
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int64_t n = n0 + ty + 8 * i;
-        if (n >= rows) continue;
-        const uint32_t c = tile[tx][ty + 8 * i];
-        for (int g = 0; g < groups; ++g) out[((int64_t)g * rows + n) * ld_bytes + k0 + tx] = (uint8_t)group_byte(c, g);
-    }
+    // one thread per (operand row, four consecutive k) of the tile: a 4-byte store per group, eight threads to a 32-byte run
+    const int nl = threadIdx.x >> 3, kq = threadIdx.x & 7;
+    const int64_t n = n0 + nl;
+    if (n >= rows) return;
+    const uint32_t c0 = tile[4 * kq][nl], c1 = tile[4 * kq + 1][nl], c2 = tile[4 * kq + 2][nl], c3 = tile[4 * kq + 3][nl];
+    for (int g = 0; g < groups; ++g)
+        *reinterpret_cast<uint32_t *>(out + ((int64_t)g * rows + n) * ld_bytes + k0 + 4 * kq) =
+            group_byte(c0, g) | (group_byte(c1, g) << 8) | (group_byte(c2, g) << 16) | (group_byte(c3, g) << 24);
 }
 
 // four consecutive columns per thread where the rows allow 16-byte accesses (the pass is a stream: 20 bytes in and 8 out
