@@ -238,7 +238,7 @@ class MlpBench:
         self.q.qnn_mlp_forward_host(self.x_host, self.M, IN_BITS, self.layers, self.scores_host, self.algo, self.ws)
 
 
-def backward_records(q, flush, rec):
+def backward_records(q, flush, rec, reps=5):
     M, Nu, K = BATCH, 4096, 4096                       # batch, units of the layer, its inputs
     emin, emax = -30, 0
     G = q.qnn_logquant_groups(emin, emax)
@@ -258,7 +258,7 @@ def backward_records(q, flush, rec):
         A = q.tc_operand(a8, ld, q.QNN_FORM_I8, planes=7, mode=q.QNN_MODE_PM1)
         Bo = q.tc_operand(b8, ld, q.QNN_FORM_I8, planes=1, mode=q.QNN_MODE_PM1)
         tag = "g_a" if not transposed else "g_W"
-        ms, best = _time_op(lambda: q.qnn_logquant_pack_groups(gs, rows, kdim, Nu, transposed, emin, emax, a8, ld), flush, reps=5)
+        ms, best = _time_op(lambda: q.qnn_logquant_pack_groups(gs, rows, kdim, Nu, transposed, emin, emax, a8, ld), flush, reps=reps)
         rec(f"alg1_backward_{tag}_pack_groups", ms, best, bytes_=4.0 * M * Nu + float(G) * rows * ld,
             note=f"{name}: fp32 gradient -> {G} int8 group matrices ({'transposed' if transposed else 'row-major'})")
 
@@ -266,7 +266,7 @@ def backward_records(q, flush, rec):
             q.qnn_logquant_pack_groups(gs, rows, kdim, Nu, transposed, emin, emax, a8, ld)
             q.qnn_tc_gemm(A, Bo, G * rows, ncols, kdim, out=part, ldo=ncols)
             q.qnn_logquant_combine(part, G, rows, ncols, ncols, out, ncols)
-        ms, best = _time_op(whole, flush, reps=5)
+        ms, best = _time_op(whole, flush, reps=reps)
         rec(f"alg1_backward_{tag}_{rows}x{ncols}x{kdim}_6bit_log_gradients", ms, best, ops=2.0 * rows * ncols * kdim * G,
             note=f"{name}: pack, one int8 product of {G} stacked groups, int64 combine; rate counted per int8 multiply-accumulate issued "
                  f"({2.0 * rows * ncols * kdim / ms / 1e9:.0f} Top/s counted once per 6-bit product)")
@@ -690,6 +690,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--convnet-only", type=int, default=0, metavar="BATCH",
                     help="time only the Table 7 ConvNet forward at this batch and print its record (one GPU)")
+    ap.add_argument("--backward-only", action="store_true",
+                    help="time only Algorithm 1's backward products with 6-bit logarithmic gradients and print their records (one GPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -711,6 +713,25 @@ def main():
             {"name": name, "ms": round(ms, 5), "ms_best": round(best, 5), "binary_Tops": round(ops / ms / 1e9, 2), "note": note}),
             reps=max(args.steps if args.steps != 200 else 7, 1))
         print(json.dumps(out[0]))
+        return
+    if args.backward_only:
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+        def flush():
+            flush_buf.fill_(1)
+            flush_buf.sum()
+        out = []
+
+        def rec(name, ms, best, bytes_=None, ops=None, note=None):
+            r = {"name": name, "ms": round(ms, 5), "ms_best": round(best, 5)}
+            if bytes_ is not None:
+                r["GBps"] = round(bytes_ / ms / 1e6, 1)
+            if ops is not None:
+                r["int8_Tops"] = round(ops / ms / 1e9, 2)
+            r["note"] = note
+            out.append(r)
+        backward_records(q, flush, rec, reps=max(args.steps if args.steps != 200 else 5, 1))
+        print(json.dumps(out))
         return
     rank, world, local = _dist_setup(args.gpus)
     algo = {"auto": q.QNN_ALGO_AUTO, "popc": q.QNN_ALGO_POPC, "tc_i8": q.QNN_ALGO_TC_I8, "b1_mma": q.QNN_ALGO_B1_MMA,
