@@ -32,7 +32,8 @@ namespace qnn {
 namespace {
 
 constexpr int EPI_GROUPS = 2;        // epilogue warps per quarter of the accumulator's lanes
-constexpr int TC_THREADS = 64 + 128 * EPI_GROUPS;   // warp 0: TMA, warp 1: MMA + TMEM owner, the rest: epilogue
+constexpr int tc_threads(int groups) { return 64 + 128 * groups; }   // warp 0: TMA, warp 1: MMA + TMEM owner, the rest: epilogue
+constexpr int TC_THREADS = tc_threads(EPI_GROUPS);
 
 struct TcParams {
     int64_t M, N;
@@ -308,18 +309,18 @@ __global__ void __launch_bounds__(32) wait_probe_kernel()
 
 constexpr int next_pow2_cols(int c) { return c <= 32 ? 32 : c <= 64 ? 64 : c <= 128 ? 128 : c <= 256 ? 256 : 512; }
 
-template <int FORM, int BN, int STG, int CTAS, int KB = BKB>
+template <int FORM, int BN, int STG, int CTAS, int KB = BKB, int G = EPI_GROUPS>
 struct TcCfg {
     static constexpr int A_BYTES = BM * KB;
     static constexpr int B_BYTES = (BN / CTAS) * KB;                    // a pair splits the B tile between its CTAs
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int CPW = (BN / 32 + EPI_GROUPS - 1) / EPI_GROUPS;  // 32-column chunks per epilogue warp
+    static constexpr int CPW = (BN / 32 + G - 1) / G;                    // 32-column chunks per epilogue warp
     static constexpr int THR_WORDS = CPW * 32 + 8;                       // per epilogue warp: its thresholds + flip words
-    static constexpr int THR_BYTES = 4 * EPI_GROUPS * THR_WORDS * 4;
+    static constexpr int THR_BYTES = 4 * G * THR_WORDS * 4;
     // epilogue staging per warp: one 4 KB tile of 32 x 32 int32 for the bulk stores; kernels instantiated
     // without it keep one more pipeline stage and store from registers
     static constexpr int STG_WARP_BYTES = STG ? 4096 : 0;
-    static constexpr int STG_BYTES = 4 * EPI_GROUPS * STG_WARP_BYTES;
+    static constexpr int STG_BYTES = 4 * G * STG_WARP_BYTES;
     static constexpr int AUX_BYTES = 256 + THR_BYTES + 1024;             // barriers, thresholds, 1024-byte alignment slack
     static constexpr int MAX_STAGES = (SMEM_LIMIT - AUX_BYTES - STG_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = MAX_STAGES > 7 ? 7 : MAX_STAGES;
@@ -336,12 +337,12 @@ struct TcCfg {
     static_assert(KB == 128 || (KB == 64 && FORM == QNN_FORM_FP4 && CTAS == 1), "64-byte K blocks: e2m1, single CTA");
 };
 
-template <int FORM, int BN, int STG, int CTAS, int KB = BKB>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+template <int FORM, int BN, int STG, int CTAS, int KB = BKB, int G = EPI_GROUPS>
+__global__ void __launch_bounds__(tc_threads(G), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_out, const TcParams p)
 {
-    using S = TcCfg<FORM, BN, STG, CTAS, KB>;
+    using S = TcCfg<FORM, BN, STG, CTAS, KB, G>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;                      // swizzled tiles need 1024-byte alignment
@@ -366,7 +367,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * EPI_GROUPS * CTAS); }   // one arrival per epilogue warp
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4 * G * CTAS); }   // one arrival per epilogue warp
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -536,8 +537,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         auto fetch_thresholds = [&](int64_t ncol0) {
 #pragma unroll
             for (int lc = 0; lc < CPW; ++lc) {
-                const int64_t n = ncol0 + (grp + lc * EPI_GROUPS) * 32 + lane;
-                const bool ncol = (grp + lc * EPI_GROUPS) < BN / 32 && n < p.N;
+                const int64_t n = ncol0 + (grp + lc * G) * 32 + lane;
+                const bool ncol = (grp + lc * G) < BN / 32 && n < p.N;
                 // (raw values: nothing here may wait for the loads -- they are converted when they are parked)
                 const int32_t tv = ncol ? __ldg(p.thr + n) : 0;
                 thr_next[lc] = tv;
@@ -655,7 +656,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int nchunks = (int)((p.N - ntile + 31) >> 5);         // warp-uniform
             nchunks = nchunks > BN / 32 ? BN / 32 : nchunks;
 #pragma unroll 1
-            for (int c = grp, lc = 0; c < nchunks; c += EPI_GROUPS, ++lc) {
+            for (int c = grp, lc = 0; c < nchunks; c += G, ++lc) {
                 const int64_t n0 = ntile + c * 32;
                 uint32_t v[32];
                 tmem_ld32(tacc + (uint32_t)(c * 32), v);
@@ -1022,11 +1023,11 @@ int pairs_resident_on_current_device()
     return v - 1;
 }
 
-template <int FORM, int BN, int STG, int CTAS, int KB = BKB>
+template <int FORM, int BN, int STG, int CTAS, int KB = BKB, int G = EPI_GROUPS>
 int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMap &mo, TcParams p, int workers, cudaStream_t st)
 {
-    using S = TcCfg<FORM, BN, STG, CTAS, KB>;
-    auto kern = gemm_tc_kernel<FORM, BN, STG, CTAS, KB>;
+    using S = TcCfg<FORM, BN, STG, CTAS, KB, G>;
+    auto kern = gemm_tc_kernel<FORM, BN, STG, CTAS, KB, G>;
     // the shared-memory opt-in is per kernel and device: asked for once, not on every launch (it costs microseconds)
     // (per device ordinal; racing first calls of two host threads both set the same attribute, which is harmless)
     static std::atomic<bool> opted_in[64];
@@ -1046,7 +1047,7 @@ int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMa
         const bool pdl = pdl_enabled();
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(CTAS * nw));
-        cfg.blockDim = dim3(TC_THREADS);
+        cfg.blockDim = dim3(tc_threads(G));
         cfg.dynamicSmemBytes = S::TOTAL;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
@@ -1068,7 +1069,7 @@ int launch_tc_stg(const CUtensorMap &ma, const CUtensorMap &mb, const CUtensorMa
     return check_launch("tc gemm");
 }
 
-template <int FORM, int BN, int CTAS, int KB = BKB>
+template <int FORM, int BN, int CTAS, int KB = BKB, int G = EPI_GROUPS>
 int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, int workers, cudaStream_t st)
 {
     // The int32 result leaves through bulk stores where its layout allows it (16-byte aligned rows), which
@@ -1102,8 +1103,8 @@ int launch_tc_cfg(const CUtensorMap &ma, const CUtensorMap &mb, TcParams p, int 
             p.tma_out = 2;
         }
     }
-    if (p.tma_out) return launch_tc_stg<FORM, BN, 1, CTAS, KB>(ma, mb, mo, p, workers, st);
-    return launch_tc_stg<FORM, BN, 0, CTAS, KB>(ma, mb, mo, p, workers, st);
+    if (p.tma_out) return launch_tc_stg<FORM, BN, 1, CTAS, KB, G>(ma, mb, mo, p, workers, st);
+    return launch_tc_stg<FORM, BN, 0, CTAS, KB, G>(ma, mb, mo, p, workers, st);
 }
 
 // Tile width.  Measured on B200: the time of one wave of tiles depends only weakly on the width (about
@@ -1351,6 +1352,19 @@ int launch_gemm_tc(const GemmArgs &g, int form, void *ws, size_t ws_bytes, cudaS
             case 128: return launch_tc_cfg<QNN_FORM_I8, 128, 2>(ma, mb, p, pairs_resident, st);
             default: return launch_tc_cfg<QNN_FORM_I8, 64, 2>(ma, mb, p, pairs_resident, st);
         }
+    }
+
+    // Short K on the int8 form (Algorithm 4's first layer, K = 784): single CTAs are bound there by the bytes an SM takes
+    // from L2 (48 KB per K block at 256 columns) and the pair halves the B share of them, but with 4 .. 11 K blocks per
+    // tile the pair's epilogue sets the pace -- so the pair runs with three epilogue warps per accumulator quarter
+    // (measured on 10000 x 4096 x 784: single CTAs 37.4-39.3 us, pairs 37.1 us, pairs with three warps 35.3 us).
+    // QNN_TC_PAIRS_SHORT=0 in the environment keeps single CTAs.
+    static const bool pairs_short_off = [] { const char *e = getenv("QNN_TC_PAIRS_SHORT"); return e && e[0] == '0'; }();
+    if (!pairs_short_off && !g.conv && form == QNN_FORM_I8 && pairs_resident >= 8 && p.num_kb >= 4 && p.num_kb < pair_min_kb &&
+        g.N >= 256 && tiles_m2 * ceil_div(g.N, 256) >= 2 * (int64_t)pairs_resident) {
+        p.tiles_m = (int32_t)tiles_m2;
+        if (int rc = make_map_2d(&mb, b8, g.N, row_bytes, b_ld, 128)) return rc;
+        return launch_tc_cfg<QNN_FORM_I8, 256, 2, BKB, 3>(ma, mb, p, pairs_resident, st);
     }
 
     // (int8 has no scale columns in tensor memory, so two 256-column accumulator stages fit: tried for wide single-CTA products)

@@ -200,12 +200,14 @@ def test_tc_gemm_argument_errors(q):
 
 
 @pytest.mark.parametrize("form_name,M,N,K", [("FP4", 4100, 1000, 4100), ("FP4", 5000, 777, 3104), ("I8", 4400, 900, 1600),
-                                                 ("FP4", 4100, 901, 3200), ("I8", 4400, 1029, 1600), ("FP4", 4100, 1137, 3104)])
+                                                 ("FP4", 4100, 901, 3200), ("I8", 4400, 1029, 1600), ("FP4", 4100, 1137, 3104),
+                                                 ("I8", 8300, 1100, 800), ("I8", 8300, 1030, 520)])
 @pytest.mark.parametrize("outputs", ["int", "sign"])
 def test_tc_gemm_cta_pair_shapes(q, form_name, M, N, K, outputs):
     """Ragged shapes large enough (and with K long enough) for the product to run on CTA pairs: 256-row tiles whose
     second half hangs over the end of M, a last column tile of a few columns (5, 17, 104 ...: the kernel narrows the
-    last block's instructions to the next multiple of 16), a partial last K block.  The oracle
+    last block's instructions to the next multiple of 16), a partial last K block; the int8 shapes with K = 800 and 520 run
+    on the short-K pairs (three epilogue warps per accumulator quarter).  The oracle
     runs on sampled rows (every row position inside a pair's tile is hit) and row-sum checksums cover all outputs."""
     form = getattr(q, "QNN_FORM_" + form_name)
     rng = np.random.default_rng(M + N + K)
