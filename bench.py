@@ -380,6 +380,19 @@ def convnet_record(q, Bn, flush, rec, reps=7):
     ms, best = _time_op(lambda: net.forward(xn, sn, wsn), flush, reps=reps)
     rec(f"table7_convnet_forward_batch{Bn}", ms, best, ops=opsn,
         note=f"{Bn / ms * 1e3:.0f} images/s; 6 conv + 3 FC layers in one qnn_convnet_forward call, weights prepared once")
+    # the same call replayed from a CUDA graph (the runner allocates nothing and never synchronises)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        net.forward(xn, sn, wsn)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            net.forward(xn, sn, wsn)
+    torch.cuda.synchronize()
+    ms, best = _time_op(graph.replay, flush, reps=reps)
+    rec(f"table7_convnet_forward_batch{Bn}_one_graph", ms, best, ops=opsn, note=f"{Bn / ms * 1e3:.0f} images/s; the call captured once, one launch per pass")
+    del graph
 
 
 def pipe_peaks(q):
